@@ -1,0 +1,454 @@
+"""Pins for the fp64 oracle: every check here compares the oracle with something that is NOT
+the oracle -- a closed form, a limit, an invariant of the mathematics, an independent solver,
+a library routine, or values the paper prints.  All CPU.
+
+Coverage map (what a mistake would break):
+  rank-1 closed form ........ dropped term / wrong sign in K, transposed operand (x != y),
+                              u-then-v order, <P,C>
+  large-eps limit ........... scaling of the exponent by eps
+  scaling == log ............ the log-domain formulas (sign of C, eps factors, log a term)
+  protocol == centralized ... Algorithm 1 block indexing, Allgather, column-block access (Prop. 1)
+  fixed point / duality ..... marginals, objective values, gauge/shift invariance
+  half-step invariants ...... each pass alone; dual ascent; Hilbert-metric contraction
+  2x2 quadratic ............. converged plan against an explicit root
+  Newton on the dual ........ converged plan and cost against an independent convex solve
+  scipy logsumexp ........... LSE rows vs columns (a transposed LSE fails here)
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+from scipy.special import logsumexp
+
+import oracle
+from paper_2502_07021_b200 import workloads
+
+K_, C_ = oracle.KIND_KERNEL, oracle.KIND_COST
+SC, LG = oracle.DOMAIN_SCALING, oracle.DOMAIN_LOG
+
+
+def dyadic_additive(n, seed):
+    """C_il = x_i + y_l with x, y on a 1/64 grid, so C is exact in fp32 and K is exactly rank one."""
+    rng = np.random.default_rng(seed)
+    x = rng.integers(0, 64, n) / 64.0
+    y = rng.integers(0, 64, n) / 64.0
+    C = (x[:, None] + y[None, :]).astype(np.float32)
+    assert np.array_equal(C.astype(np.float64), x[:, None] + y[None, :])
+    return C, x, y
+
+
+def dirichlet_pair(n, seed):
+    a = workloads.dirichlet1(np.random.default_rng(seed), n).astype(np.float32)
+    b = workloads.dirichlet1(np.random.default_rng(seed + 1), n).astype(np.float32)
+    return a, b
+
+
+def random_cost(n, seed, scale=1.0):
+    rng = np.random.default_rng(seed)
+    return (scale * rng.random((n, n))).astype(np.float32)
+
+
+def hilbert(x, y):
+    r = np.asarray(x) / np.asarray(y)
+    return float(np.log(r.max()) - np.log(r.min()))
+
+
+# ------------------------------------------------------------------ P1 rank-1 closed form
+
+@pytest.mark.parametrize("n,eps", [(5, 0.3), (37, 0.11), (64, 1.0)])
+def test_rank1_closed_form_scaling(n, eps):
+    C, x, y = dyadic_additive(n, 11 + n)
+    a, b = dirichlet_pair(n, 100 + n)
+    a64, b64 = a.astype(np.float64), b.astype(np.float64)
+    p, q = np.exp(-x / eps), np.exp(-y / eps)
+    s = q.sum()
+    # one full iteration from u = v = 1:  u_i = a_i/(p_i s),  v_l = b_l / (q_l * sum_i p_i u_i)
+    u, v = oracle.sinkhorn_scaling(C, C_, eps, a, b, 1)
+    u_ref = a64 / (p * s)
+    v_ref = b64 / (q * (p * u_ref).sum())
+    np.testing.assert_allclose(u, u_ref, rtol=1e-13)
+    np.testing.assert_allclose(v, v_ref, rtol=1e-13)
+    P = oracle.plan(C, C_, eps, SC, u, v)
+    # P = a b^T / mass(a): rows scaled so that columns are exact after the v update
+    np.testing.assert_allclose(P, np.outer(a64, b64) / a64.sum(), rtol=1e-12)
+    obj = oracle.objectives(C, C_, eps, SC, u, v, C)
+    cost_ref = (np.outer(a64, b64) / a64.sum() * (x[:, None] + y[None, :])).sum()
+    assert obj["cost"] == pytest.approx(cost_ref, rel=1e-12)
+    # with a stored kernel instead of a stored cost: same iterates up to fp32 rounding of K
+    K32 = np.exp(-(x[:, None] + y[None, :]) / eps).astype(np.float32)
+    uk, vk = oracle.sinkhorn_scaling(K32, K_, eps, a, b, 1)
+    np.testing.assert_allclose(uk, u_ref, rtol=5e-7)
+    np.testing.assert_allclose(vk, v_ref, rtol=5e-7)
+    # the column error is zero from iteration 1 on, the row error too when masses agree
+    e = oracle.marginal_errors(C, C_, eps, SC, u, v, a, b)
+    assert e["col_l1"] < 1e-14
+    mass_gap = abs(a64.sum() - b64.sum())
+    assert e["row_l1"] <= mass_gap + 1e-14
+
+
+@pytest.mark.parametrize("n,eps", [(6, 0.25), (33, 0.07)])
+def test_rank1_closed_form_log(n, eps):
+    C, x, y = dyadic_additive(n, 21 + n)
+    a, b = dirichlet_pair(n, 200 + n)
+    a64, b64 = a.astype(np.float64), b.astype(np.float64)
+    f, g = oracle.sinkhorn_log(C, eps, a, b, 1)
+    # f_i = eps log a_i + x_i - eps log sum_l exp(-y_l/eps)   (from g = 0)
+    s = np.exp(-y / eps).sum()
+    f_ref = eps * np.log(a64) + x - eps * np.log(s)
+    # g_l = eps log b_l + y_l - eps log sum_i exp((f_i - x_i)/eps) = eps log b_l + y_l - eps log(sum a / s)
+    g_ref = eps * np.log(b64) + y - eps * np.log(a64.sum() / s)
+    np.testing.assert_allclose(f, f_ref, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(g, g_ref, rtol=0, atol=1e-13)
+    P = oracle.plan(C, C_, eps, LG, f, g)
+    np.testing.assert_allclose(P, np.outer(a64, b64) / a64.sum(), rtol=1e-11)
+
+
+def test_rank1_nonsymmetric_catches_transpose():
+    # x != y makes K non-symmetric: using K^T in the row pass would give p and q swapped
+    n, eps = 9, 0.2
+    C, x, y = dyadic_additive(n, 5)
+    assert not np.allclose(C, C.T)
+    a, b = dirichlet_pair(n, 55)
+    v0 = np.random.default_rng(3).random(n) + 0.5
+    u, qv = oracle.row_pass(C, C_, eps, a, v0)
+    np.testing.assert_allclose(qv, np.exp(-x / eps) * (np.exp(-y / eps) * v0).sum(), rtol=1e-13)
+    v, r = oracle.col_pass(C, C_, eps, b, u)
+    np.testing.assert_allclose(r, np.exp(-y / eps) * (np.exp(-x / eps) * u).sum(), rtol=1e-13)
+    np.testing.assert_allclose(u * qv, a, rtol=1e-15)
+    np.testing.assert_allclose(v * r, b, rtol=1e-15)
+
+
+# ------------------------------------------------------------------ P2 large-eps limit
+
+def test_large_eps_limit():
+    n = 24
+    C = random_cost(n, 31)
+    a, b = dirichlet_pair(n, 32)
+    ab = np.outer(a.astype(np.float64), b.astype(np.float64))
+    prev = None
+    for eps in (1e2, 1e4, 1e6):
+        u, v = oracle.sinkhorn_scaling(C, C_, eps, a, b, 50)
+        P = oracle.plan(C, C_, eps, SC, u, v)
+        dev = np.abs(P - ab).max() / ab.max()
+        assert dev < 3.0 * float(C.max()) / eps
+        f, g = oracle.sinkhorn_log(C, eps, a, b, 50)
+        Pl = oracle.plan(C, C_, eps, LG, f, g)
+        assert np.abs(Pl - ab).max() / ab.max() < 3.0 * float(C.max()) / eps
+        if prev is not None:
+            assert dev < prev / 50       # first order in 1/eps
+        prev = dev
+
+
+# ------------------------------------------------------------------ P3 scaling == log
+
+@pytest.mark.parametrize("n,eps,seed", [(17, 0.05, 1), (40, 0.02, 2), (8, 1.0, 3)])
+def test_domain_equivalence_every_iteration(n, eps, seed):
+    C = random_cost(n, seed)
+    a, b = dirichlet_pair(n, 40 + seed)
+    for t in (1, 2, 5, 13):
+        u, v = oracle.sinkhorn_scaling(C, C_, eps, a, b, t)
+        f, g = oracle.sinkhorn_log(C, eps, a, b, t)
+        np.testing.assert_allclose(f, eps * np.log(u), rtol=0, atol=1e-12)
+        np.testing.assert_allclose(g, eps * np.log(v), rtol=0, atol=1e-12)
+
+
+def test_log_domain_survives_underflow():
+    # exp(-C/eps) underflows fp64 for most entries here, the log form must not care
+    n, eps = 12, 1e-3
+    C = random_cost(n, 8, scale=4.0)
+    a, b = dirichlet_pair(n, 9)
+    assert (np.exp(-C.astype(np.float64) / eps) == 0).mean() > 0.5
+    f, g = oracle.sinkhorn_log(C, eps, a, b, 3000)
+    assert np.all(np.isfinite(f)) and np.all(np.isfinite(g))
+    e = oracle.marginal_errors(C, C_, eps, LG, f, g, a, b)
+    assert e["col_l1"] < 1e-12
+    # convergence is slow this close to the unregularised problem; it must still be monotone
+    f1, g1 = oracle.sinkhorn_log(C, eps, a, b, 300)
+    assert e["row_l1"] < oracle.marginal_errors(C, C_, eps, LG, f1, g1, a, b)["row_l1"] < 1.0
+
+
+# ------------------------------------------------------------------ P4 / P9 protocol == centralized
+
+def compositions(n, c):
+    for cuts in itertools.combinations(range(1, n), c - 1):
+        yield np.array((0,) + cuts + (n,), dtype=np.int64)
+
+
+def test_protocol_bit_identical_all_compositions():
+    n, eps = 7, 0.3
+    C = random_cost(n, 77)
+    assert not np.allclose(C, C.T)
+    a, b = dirichlet_pair(n, 78)
+    u0, v0 = oracle.sinkhorn_scaling(C, C_, eps, a, b, 4)
+    count = 0
+    for c in range(1, n + 1):
+        for off in compositions(n, c):
+            u, v, agree = oracle.sinkhorn_protocol(C, C_, eps, a, b, off, 4)
+            assert agree
+            assert np.array_equal(u, u0) and np.array_equal(v, v0), off
+            count += 1
+    assert count == 2 ** (n - 1)
+
+
+@pytest.mark.parametrize("offsets", [[0, 100, 101, 300, 512], [0, 512], list(range(0, 513, 64))])
+def test_protocol_bit_identical_config1(offsets):
+    w = workloads.make(1)
+    u0, v0 = oracle.sinkhorn_scaling(w.K, K_, w.eps, w.a, w.b, 3)
+    u, v, agree = oracle.sinkhorn_protocol(w.K, K_, w.eps, w.a, w.b, offsets, 3)
+    assert agree and np.array_equal(u, u0) and np.array_equal(v, v0)
+
+
+def test_rowpartition_equals_centralized_to_rounding():
+    w = workloads.make(2, n=300)
+    u0, v0 = oracle.sinkhorn_scaling(w.K, K_, w.eps, w.a, w.b, 6)
+    u, v = oracle.sinkhorn_rowpartition(w.K, K_, w.eps, w.a, w.b, [0, 7, 150, 151, 300], 6)
+    np.testing.assert_allclose(u, u0, rtol=1e-12)
+    np.testing.assert_allclose(v, v0, rtol=1e-12)
+    # a single block is the same association as the centralized sum
+    u1, v1 = oracle.sinkhorn_rowpartition(w.K, K_, w.eps, w.a, w.b, [0, 300], 6)
+    assert np.array_equal(u1, u0) and np.array_equal(v1, v0)
+
+
+def test_batched_is_loop_of_singles():
+    w = workloads.make(5, n=48, nbatch=5)
+    U, V = oracle.sinkhorn_batched(w.K, K_, w.eps, w.a, w.b, 7)
+    for p in range(5):
+        u, v = oracle.sinkhorn_scaling(w.K, K_, w.eps, w.a[p], w.b[p], 7)
+        assert np.array_equal(U[p], u) and np.array_equal(V[p], v)
+    # problems do not interact: permuting the batch permutes the answers
+    U2, V2 = oracle.sinkhorn_batched(w.K, K_, w.eps, w.a[::-1], w.b[::-1], 7)
+    assert np.array_equal(U2[::-1], U) and np.array_equal(V2[::-1], V)
+
+
+# ------------------------------------------------------------------ P5 fixed point, duality, invariance
+
+def test_fixed_point_marginals_and_strong_duality():
+    n, eps = 30, 0.08
+    C = random_cost(n, 91)
+    a, b = dirichlet_pair(n, 92)
+    # equal masses are needed for an exact fixed point: renormalise in fp64, round once
+    a = (a.astype(np.float64) / a.astype(np.float64).sum()).astype(np.float32)
+    b64 = b.astype(np.float64)
+    b = (b64 * (a.astype(np.float64).sum() / b64.sum())).astype(np.float32)
+    mass_gap = abs(a.astype(np.float64).sum() - b.astype(np.float64).sum())
+    u, v = oracle.sinkhorn_scaling(C, C_, eps, a, b, 4000)
+    e = oracle.marginal_errors(C, C_, eps, SC, u, v, a, b)
+    assert e["col_l1"] < 1e-13
+    assert e["row_l1"] < 1e-13 + 2 * mass_gap
+    f, g = eps * np.log(u), eps * np.log(v)
+    obj = oracle.objectives(C, C_, eps, SC, u, v, C)
+    D = oracle.dual_value(eps, f, g, a, b, obj["mass"])
+    assert obj["primal"] == pytest.approx(D, abs=1e-10 + 10 * mass_gap)
+    # log-domain run reaches the same plan
+    fl, gl = oracle.sinkhorn_log(C, eps, a, b, 4000)
+    np.testing.assert_allclose(oracle.plan(C, C_, eps, LG, fl, gl), oracle.plan(C, C_, eps, SC, u, v),
+                               rtol=1e-9, atol=1e-16)
+
+
+def test_plan_invariant_under_row_column_shifts():
+    # C_il -> C_il + alpha_i + beta_l only changes the duals, never P* (shifts on a dyadic grid so
+    # the shifted cost is exact in fp32)
+    n, eps = 16, 0.25
+    rng = np.random.default_rng(5)
+    C = (rng.integers(0, 256, (n, n)) / 256.0).astype(np.float32)
+    al = rng.integers(0, 32, n) / 32.0
+    be = rng.integers(0, 32, n) / 32.0
+    C2 = (C.astype(np.float64) + al[:, None] + be[None, :]).astype(np.float32)
+    assert np.array_equal(C2.astype(np.float64), C.astype(np.float64) + al[:, None] + be[None, :])
+    a, b = dirichlet_pair(n, 6)
+    u, v = oracle.sinkhorn_scaling(C, C_, eps, a, b, 3000)
+    u2, v2 = oracle.sinkhorn_scaling(C2, C_, eps, a, b, 3000)
+    np.testing.assert_allclose(oracle.plan(C2, C_, eps, SC, u2, v2), oracle.plan(C, C_, eps, SC, u, v), rtol=1e-10)
+
+
+# ------------------------------------------------------------------ P6 half-step invariants
+
+def test_half_step_invariants_dual_ascent_and_contraction():
+    n, eps = 25, 0.1
+    C = random_cost(n, 123)
+    a, b = dirichlet_pair(n, 124)
+    a64, b64 = a.astype(np.float64), b.astype(np.float64)
+    u, v = np.ones(n), np.ones(n)
+
+    def dual(u, v):
+        mass = oracle.objectives(C, C_, eps, SC, u, v, C)["mass"]
+        return oracle.dual_value(eps, eps * np.log(u), eps * np.log(v), a, b, mass)
+
+    last_D = dual(u, v)
+    last_dh = None
+    for t in range(12):
+        u_new, q = oracle.row_pass(C, C_, eps, a, v)
+        row, _ = oracle.marginals(C, C_, eps, SC, u_new, v)
+        np.testing.assert_allclose(row, a64, rtol=1e-14)            # after the u update P1 = a
+        D = dual(u_new, v)
+        assert D >= last_D - 1e-13
+        last_D = D
+        v_new, r = oracle.col_pass(C, C_, eps, b, u_new)
+        _, col = oracle.marginals(C, C_, eps, SC, u_new, v_new)
+        np.testing.assert_allclose(col, b64, rtol=1e-14)            # after the v update P^T 1 = b
+        D = dual(u_new, v_new)
+        assert D >= last_D - 1e-13
+        last_D = D
+        if t > 0:
+            dh = hilbert(u_new, u)
+            if last_dh is not None and last_dh > 1e-12:
+                assert dh < last_dh                                  # Birkhoff contraction
+            last_dh = dh
+        u, v = u_new, v_new
+
+
+def test_divide_is_hilbert_isometry():
+    n, eps = 10, 0.4
+    C = random_cost(n, 1)
+    a, _ = dirichlet_pair(n, 2)
+    rng = np.random.default_rng(3)
+    v1, v2 = rng.random(n) + 0.1, rng.random(n) + 0.1
+    u1, q1 = oracle.row_pass(C, C_, eps, a, v1)
+    u2, q2 = oracle.row_pass(C, C_, eps, a, v2)
+    assert hilbert(u1, u2) == pytest.approx(hilbert(q1, q2), rel=1e-12)
+    assert hilbert(q1, q2) < hilbert(v1, v2)
+
+
+# ------------------------------------------------------------------ P7 2x2 closed form
+
+@pytest.mark.parametrize("a1,b1,eps", [(0.3, 0.6, 0.5), (0.5, 0.5, 0.2), (0.85, 0.25, 1.5)])
+def test_two_by_two_closed_form(a1, b1, eps):
+    C = np.array([[0.0, 1.0], [0.75, 0.25]], dtype=np.float32)
+    a = np.array([a1, 1 - a1], dtype=np.float32)
+    b = np.array([b1, 1 - b1], dtype=np.float32)
+    a1, b1 = float(a[0]), float(b[0])
+    a2, b2 = float(a[1]), float(b[1])
+    m = 0.5 * ((a1 + a2) + (b1 + b2))
+    K = np.exp(-C.astype(np.float64) / eps)
+    theta = K[0, 0] * K[1, 1] / (K[0, 1] * K[1, 0])
+    # P11 = p, P12 = a1-p, P21 = b1-p, P22 = m-a1-b1+p ; cross ratio p*P22 = theta*P12*P21
+    A = 1 - theta
+    B = (m - a1 - b1) + theta * (a1 + b1)
+    Cq = -theta * a1 * b1
+    roots = np.roots([A, B, Cq]) if abs(A) > 1e-14 else np.array([-Cq / B])
+    lo, hi = max(0.0, a1 + b1 - m), min(a1, b1)
+    p = [float(r.real) for r in roots if abs(r.imag) < 1e-12 and lo - 1e-12 <= r.real <= hi + 1e-12]
+    assert len(p) == 1
+    u, v = oracle.sinkhorn_scaling(C, C_, eps, a, b, 2000)
+    P = oracle.plan(C, C_, eps, SC, u, v)
+    assert P[0, 0] == pytest.approx(p[0], abs=1e-7)   # 1e-7: fp32 a and b carry slightly different masses
+    assert P[0, 0] * P[1, 1] / (P[0, 1] * P[1, 0]) == pytest.approx(theta, rel=1e-12)
+
+
+# ------------------------------------------------------------------ P8 independent convex solve
+
+def newton_dual(C, a, b, eps, iters=200):
+    """Maximise D(f,g) = <f,a> + <g,b> - eps sum exp((f_i+g_l-C_il)/eps) with g_{n-1} = 0 by a
+    damped Newton method.  Written independently of the oracle (numpy only)."""
+    n = C.shape[0]
+    z = np.zeros(2 * n - 1)
+
+    def parts(z):
+        f, g = z[:n], np.append(z[n:], 0.0)
+        P = np.exp((f[:, None] + g[None, :] - C) / eps)
+        return f, g, P
+
+    def D(z):
+        f, g, P = parts(z)
+        return f @ a + g @ b - eps * P.sum()
+
+    for _ in range(iters):
+        f, g, P = parts(z)
+        grad = np.concatenate([a - P.sum(1), (b - P.sum(0))[:-1]])
+        if np.abs(grad).max() < 1e-15:
+            break
+        H = np.zeros((2 * n - 1, 2 * n - 1))
+        H[:n, :n] = np.diag(P.sum(1))
+        H[n:, n:] = np.diag(P.sum(0)[:-1])
+        H[:n, n:] = P[:, :-1]
+        H[n:, :n] = P[:, :-1].T
+        step = np.linalg.solve(H / eps, grad)
+        t, d0 = 1.0, D(z)
+        while D(z + t * step) < d0 and t > 1e-12:
+            t *= 0.5
+        z = z + t * step
+    f, g, P = parts(z)
+    return f, g, P
+
+
+@pytest.mark.parametrize("n,eps,seed", [(3, 0.5, 0), (5, 0.3, 1), (8, 0.2, 2), (8, 1.0, 3)])
+def test_against_newton_on_the_dual(n, eps, seed):
+    C32 = random_cost(n, 500 + seed)
+    a, b = dirichlet_pair(n, 600 + seed)
+    a64 = a.astype(np.float64)
+    b64 = b.astype(np.float64) * (a64.sum() / b.astype(np.float64).sum())   # exact equal mass in fp64
+    b = b64.astype(np.float32)
+    b64 = b.astype(np.float64)
+    gap = abs(a64.sum() - b64.sum())
+    C = C32.astype(np.float64)
+    f, g, P = newton_dual(C, a64, b64 * (a64.sum() / b64.sum()), eps)
+    u, v = oracle.sinkhorn_scaling(C32, C_, eps, a, b, 6000)
+    Po = oracle.plan(C32, C_, eps, SC, u, v)
+    np.testing.assert_allclose(Po, P, rtol=0, atol=1e-9 + 2 * gap)
+    assert oracle.objectives(C32, C_, eps, SC, u, v, C32)["cost"] == pytest.approx((P * C).sum(), abs=1e-9 + 2 * gap)
+    fl, gl = oracle.sinkhorn_log(C32, eps, a, b, 6000)
+    np.testing.assert_allclose(oracle.plan(C32, C_, eps, LG, fl, gl), P, rtol=0, atol=1e-9 + 2 * gap)
+    # duals agree up to the gauge (f + t, g - t)
+    # (1e-7: the fp32 a and b carry masses that differ by ~1e-8, which moves the duals by that much)
+    shift = (fl - f).mean()
+    np.testing.assert_allclose(fl - shift, f, atol=1e-7)
+    np.testing.assert_allclose(gl + shift, g, atol=1e-7)
+
+
+# ------------------------------------------------------------------ library-routine special case
+
+def test_lse_against_scipy():
+    n, eps = 50, 0.03
+    C = random_cost(n, 17, scale=2.0)
+    rng = np.random.default_rng(18)
+    g = rng.standard_normal(n) * 0.1
+    f = rng.standard_normal(n) * 0.1
+    C64 = C.astype(np.float64)
+    np.testing.assert_allclose(oracle.lse_rows(C, eps, g), logsumexp((g[None, :] - C64) / eps, axis=1), rtol=1e-13)
+    np.testing.assert_allclose(oracle.lse_cols(C, eps, f), logsumexp((f[:, None] - C64) / eps, axis=0), rtol=1e-13)
+
+
+def test_padded_leading_dimension():
+    n = 19
+    big = random_cost(32, 3)
+    view = big[:n, :n]                      # ld = 32 > n
+    dense = np.ascontiguousarray(view)
+    a, b = dirichlet_pair(n, 4)
+    u1, v1 = oracle.sinkhorn_scaling(view, C_, 0.2, a, b, 5)
+    u2, v2 = oracle.sinkhorn_scaling(dense, C_, 0.2, a, b, 5)
+    assert np.array_equal(u1, u2) and np.array_equal(v1, v2)
+
+
+# ------------------------------------------------------------------ the paper's printed toy example
+
+def read_golden(name):
+    path = os.path.join(os.path.dirname(__file__), "golden", name)
+    out, key = {}, None
+    for line in open(path):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        if line.startswith("["):
+            key = line.strip("[]")
+            out[key] = []
+        else:
+            out[key].append([float(t) for t in line.split()])
+    return {k: np.array(v) for k, v in out.items()}
+
+
+def test_toy_portfolio_printed_values():
+    gold = read_golden("toy_portfolio.txt")
+    a = gold["x_shifted"][0] / gold["x_shifted"][0].sum()
+    b = gold["xprime_shifted"][0] / gold["xprime_shifted"][0].sum()
+    P = gold["P"]
+    # what the printed plan does satisfy: its column sums are the stated b (to printed digits)
+    np.testing.assert_allclose(P.sum(0), b, atol=2e-3)
+    # what it does not: the row sums are not the stated a -- the example is inconsistent
+    assert np.abs(P.sum(1) - a).max() > 0.05
+    # the oracle on the printed C with the stated a, b and eps reaches the stated marginals
+    C = gold["C"].astype(np.float32)
+    u, v = oracle.sinkhorn_scaling(C, C_, 0.01, a.astype(np.float32), b.astype(np.float32), 5000)
+    row, col = oracle.marginals(C, C_, 0.01, SC, u, v)
+    np.testing.assert_allclose(col, b, atol=1e-7)
+    np.testing.assert_allclose(row, a, atol=1e-6)
