@@ -1,0 +1,185 @@
+/*
+ * fs.h -- C ABI of the B200 Sinkhorn hot-path library (libfs_b200.so).
+ *
+ * The library runs, on ONE GPU, the per-iteration kernel-operator passes of entropic optimal
+ * transport (paper Section 1, Eq. 1 and the display below it):
+ *
+ *        u <- a ./ (K v),      v <- b ./ (K^T u),      K = exp(-C/eps),
+ *
+ * started from u = v = 1 and applied in the order "u first, then v with the new u"
+ * (Algorithm 1), plus the stabilised log-domain form with duals f = eps log u, g = eps log v
+ * (named in Section 1 and Section 2.1; the update is the standard one)
+ *
+ *        f_i <- eps log a_i - eps LSE_l((g_l - C_il)/eps),
+ *        g_l <- eps log b_l - eps LSE_i((f_i - C_il)/eps),
+ *
+ * and the multi-target variant of Section 5.1.1 in which N problems share one K.
+ *
+ * The c row blocks I_j of the row-partitioned matrix (Section 3.1: client j holds a_j, b_j and the
+ * rows C_{I_j,:}) are kept as input structure: tiles of the column pass never straddle a block
+ * boundary and the marginal error is accumulated per block.  The iterates equal those of
+ * centralized Sinkhorn for every block layout (Proposition 1); they are bit-identical across
+ * layouts whose offsets are all multiples of the library's row-tile height.
+ *
+ * Conventions
+ *   - All `*_dev` pointers are DEVICE pointers on the current CUDA device; all other pointers
+ *     are HOST pointers.  `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - Matrices are fp32, row-major, n x n, with leading dimension ld >= n (in elements).
+ *   - Vectors are fp32.  With nbatch = N > 1 every vector argument is laid out [N][n]
+ *     (each problem's vector contiguous).
+ *   - Every function returns FS_OK (0) or a negative FS_ERR_* code and never throws.  On an
+ *     error no solver state is changed (fs_create leaves *out = NULL).
+ *   - Calls on one handle must not overlap in time (one stream at a time per handle).
+ *   - There is no CPU fallback: without a CUDA device every compute call fails with FS_ERR_CUDA.
+ */
+#ifndef FS_B200_H
+#define FS_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fs_solver fs_solver; /* opaque */
+
+enum { FS_DOMAIN_SCALING = 0, FS_DOMAIN_LOG = 1 };
+enum { FS_MATRIX_KERNEL = 0 /* the matrix is K */, FS_MATRIX_COST = 1 /* the matrix is C */ };
+
+enum {
+    FS_OK = 0,
+    FS_ERR_NULL = -1,                 /* a required pointer is NULL */
+    FS_ERR_BAD_N = -2,                /* n < 1, ld < n, nbatch < 1, k < 0, bad enum value */
+    FS_ERR_BAD_OFFSETS = -3,          /* offsets not 0 = o[0] < o[1] < ... < o[c] = n */
+    FS_ERR_BAD_EPS = -4,              /* eps not finite or <= 0 */
+    FS_ERR_NONPOSITIVE_MARGINAL = -5, /* some a_i or b_i is <= 0 or not finite (assumption A2) */
+    FS_ERR_MASS_MISMATCH = -6,        /* |sum a - sum b| > 1e-4 * sum a for some problem (A2) */
+    FS_ERR_DOMAIN = -7,               /* log domain requested with a kernel matrix (it needs C) */
+    FS_ERR_CUDA = -8,                 /* a CUDA runtime call failed; see fs_last_cuda_error() */
+    FS_ERR_NONFINITE = -9,            /* an update produced a non-finite or non-positive scaling */
+    FS_ERR_UNSUPPORTED = -10          /* combination not implemented (batched log domain) */
+};
+
+/* Options for fs_set_option. */
+enum {
+    FS_OPT_USE_GRAPH = 1,   /* 1 (default): fs_iterate replays a captured CUDA graph; 0: plain launches */
+    FS_OPT_BATCH_ENGINE = 2, /* batched passes: 0 = auto, 1 = fp32 FMA kernels, 2 = tensor-core kernels */
+    /* Tuning knobs for the single-problem passes (defaults are chosen from n at fs_create): */
+    FS_OPT_ROW_SHAPE = 3,   /* value = L*1000 + R: L threads sweep R rows at once; (32,1), (256,4), (256,8) */
+    FS_OPT_COL_SHAPE = 4    /* value = TX*1000 + H: TX in {32,64,256} threads across a column strip of 4*TX
+                               columns, row tiles of at most H <= 256 rows */
+};
+
+/*
+ * fs_create -- build a solver for one problem (nbatch = 1) or N problems sharing the matrix.
+ * Follows the problem statement of Section 3.1 / Algorithm 1 (inputs a_j, b_j, C_{I_j,:};
+ * start u = v = 1) and Section 5.1.1 (shared K, N marginal pairs).
+ *
+ *   out          receives the handle.
+ *   n            problem size; the matrix is n x n (square only).
+ *   c            number of row blocks, 1 <= c <= n.
+ *   row_offsets  HOST, c+1 entries, 0 = o[0] < o[1] < ... < o[c] = n; block j is rows o[j]..o[j+1]-1.
+ *                Copied.
+ *   M_dev, ld    DEVICE n x n fp32 row-major matrix, leading dimension ld.  BORROWED: it must stay
+ *                valid and unmodified until fs_destroy.  Never written.
+ *   matrix_kind  FS_MATRIX_KERNEL: M is K (entries > 0, assumption A1).  FS_MATRIX_COST: M is C;
+ *                in the scaling domain the library then materialises K = exp(-C/eps) once, in
+ *                fp32, into memory it owns; in the log domain C is streamed directly.
+ *   eps          entropic regularisation, > 0.
+ *   a_dev,b_dev  DEVICE [nbatch][n] marginals, strictly positive, equal mass per problem.  Copied.
+ *   nbatch       number of problems sharing the matrix (1 for the single-problem passes).
+ *   domain       FS_DOMAIN_SCALING or FS_DOMAIN_LOG (log needs FS_MATRIX_COST and nbatch = 1).
+ *   stream       stream for the set-up kernels; the call synchronises it before returning.
+ */
+int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets, const float *M_dev,
+              int64_t ld, int matrix_kind, double eps, const float *a_dev, const float *b_dev,
+              int32_t nbatch, int domain, void *stream);
+
+/*
+ * fs_iterate -- enqueue k full Sinkhorn iterations (row pass then column pass, Algorithm 1 loop
+ * body) on `stream`.  Asynchronous: returns after the launch.  k >= 0.  With FS_OPT_USE_GRAPH the
+ * k iterations are captured once into CUDA graphs (cached per handle) and replayed.
+ */
+int fs_iterate(fs_solver *s, int32_t k, void *stream);
+
+/* One half-step only: the row pass u <- a ./ (K v) (or its log form), resp. the column pass
+ * v <- b ./ (K^T u).  Asynchronous.  They do not advance the iteration counter. */
+int fs_row_pass(fs_solver *s, void *stream);
+int fs_col_pass(fs_solver *s, void *stream);
+
+/*
+ * fs_marginal_error -- marginal violation of the CURRENT state, err_a = ||P 1 - a|| and
+ * err_b = ||P^T 1 - b|| with P = diag(u) K diag(v) (Section 5.3 uses the 2-norm; norm = 1 gives the
+ * 1-norm).  Runs a fresh non-updating evaluation of both passes, synchronises `stream`.
+ *   row_err, col_err   HOST, [nbatch] each; either may be NULL.
+ * Returns FS_ERR_NONFINITE if any update since the last such call produced a non-finite value.
+ */
+int fs_marginal_error(fs_solver *s, int norm, double *row_err, double *col_err, void *stream);
+
+/* Copy the current scalings (scaling domain: u, v; log domain: f, g) into caller DEVICE buffers of
+ * [nbatch][n] floats each; either may be NULL.  Synchronises `stream`; reports FS_ERR_NONFINITE
+ * like fs_marginal_error (the copy is still made). */
+int fs_scalings(fs_solver *s, float *u_dev_out, float *v_dev_out, void *stream);
+
+/* Overwrite the current scalings (resume from a checkpoint).  DEVICE [nbatch][n]; either may be
+ * NULL (left as is).  Asynchronous on `stream`. */
+int fs_set_scalings(fs_solver *s, const float *u_dev, const float *v_dev, void *stream);
+
+/* Reset to the initial state of Algorithm 1 (u = v = 1, resp. f = g = 0), iteration counter and
+ * error trace to zero.  Asynchronous on `stream`. */
+int fs_reset(fs_solver *s, void *stream);
+
+/*
+ * fs_transport_cost -- <P,C> = sum_il P_il C_il for the current state (first term of Eq. 1).
+ *   C_dev, ldc   DEVICE n x n fp32 cost.  May be NULL when the solver was created from a cost
+ *                matrix (then that matrix is used).
+ *   cost_out     HOST [nbatch].
+ * Synchronises `stream`.
+ */
+int fs_transport_cost(fs_solver *s, const float *C_dev, int64_t ldc, double *cost_out, void *stream);
+
+/* Error trace: with check_every = m > 0, fs_iterate records err_a (1-norm and 2-norm, problem 0)
+ * of the state after every m-th iteration.  The value for a state is produced by the NEXT row
+ * pass, where u .* (K v) is available at no cost; when fs_iterate ends exactly on a check point one
+ * extra non-updating row pass is run for it.  0 switches the trace off.  Clears the trace. */
+int fs_set_error_trace(fs_solver *s, int32_t check_every);
+
+/* Read the trace: up to `cap` entries are written to the HOST arrays (either may be NULL);
+ * *count receives the number recorded so far; iteration numbers are m, 2m, 3m, ...
+ * Synchronises `stream`. */
+int fs_error_trace(fs_solver *s, double *l1_out, double *l2_out, int32_t cap, int32_t *count, void *stream);
+
+/* Per-block row error of the last evaluated state: HOST [c] doubles, the 1-norm share of each
+ * row block I_j (the "few scalars" a client would contribute).  Valid after fs_marginal_error. */
+int fs_block_errors(fs_solver *s, double *block_l1_out);
+
+int fs_set_option(fs_solver *s, int option, int64_t value);
+
+/* Number of iterations enqueued since creation / fs_reset. */
+int64_t fs_iterations_done(const fs_solver *s);
+
+/* Number of kernel launches this handle has enqueued so far (graph replays count their nodes). */
+int64_t fs_launch_count(const fs_solver *s);
+
+int fs_destroy(fs_solver *s);
+
+/*
+ * fs_solve_host -- the whole path from HOST buffers: allocates device memory, copies the matrix and
+ * the marginals to the device, runs `iters` iterations, copies the scalings back and frees everything.
+ * All pointers are HOST pointers; M_host is n x n with leading dimension ld; a, b, u_out, v_out are
+ * [nbatch][n]; row_err_l1_out is [nbatch] or NULL (1-norm row marginal error of the final state).
+ * Synchronous.
+ */
+int fs_solve_host(int64_t n, int32_t c, const int64_t *row_offsets, const float *M_host, int64_t ld,
+                  int matrix_kind, double eps, const float *a_host, const float *b_host, int32_t nbatch,
+                  int domain, int32_t iters, float *u_out, float *v_out, double *row_err_l1_out);
+
+const char *fs_strerror(int code);
+
+/* Text of the last CUDA error seen by this thread's calls ("" if none). */
+const char *fs_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FS_B200_H */

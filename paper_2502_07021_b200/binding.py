@@ -1,0 +1,221 @@
+"""ctypes binding over the C ABI of libfs_b200.so -- argument marshalling only.
+
+Every function here has the name and the argument order of its C counterpart in
+``include/fs.h``; device buffers are passed as torch CUDA tensors (or raw integer addresses),
+streams as ``torch.cuda.Stream`` / integer / None.  All arithmetic runs in the library's CUDA
+kernels; there is no fallback: if the shared library has not been built, ``lib()`` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+FS_DOMAIN_SCALING, FS_DOMAIN_LOG = 0, 1
+FS_MATRIX_KERNEL, FS_MATRIX_COST = 0, 1
+FS_OK = 0
+FS_ERR_NULL, FS_ERR_BAD_N, FS_ERR_BAD_OFFSETS, FS_ERR_BAD_EPS = -1, -2, -3, -4
+FS_ERR_NONPOSITIVE_MARGINAL, FS_ERR_MASS_MISMATCH, FS_ERR_DOMAIN = -5, -6, -7
+FS_ERR_CUDA, FS_ERR_NONFINITE, FS_ERR_UNSUPPORTED = -8, -9, -10
+FS_OPT_USE_GRAPH, FS_OPT_BATCH_ENGINE, FS_OPT_ROW_SHAPE, FS_OPT_COL_SHAPE = 1, 2, 3, 4
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libfs_b200.so")
+
+_vp = ctypes.c_void_p
+_i64 = ctypes.c_int64
+_i32 = ctypes.c_int32
+_int = ctypes.c_int
+_dbl = ctypes.c_double
+_SIGNATURES = {
+    "fs_create": (_int, [ctypes.POINTER(_vp), _i64, _i32, _vp, _vp, _i64, _int, _dbl, _vp, _vp, _i32, _int, _vp]),
+    "fs_iterate": (_int, [_vp, _i32, _vp]),
+    "fs_row_pass": (_int, [_vp, _vp]),
+    "fs_col_pass": (_int, [_vp, _vp]),
+    "fs_marginal_error": (_int, [_vp, _int, _vp, _vp, _vp]),
+    "fs_scalings": (_int, [_vp, _vp, _vp, _vp]),
+    "fs_set_scalings": (_int, [_vp, _vp, _vp, _vp]),
+    "fs_reset": (_int, [_vp, _vp]),
+    "fs_transport_cost": (_int, [_vp, _vp, _i64, _vp, _vp]),
+    "fs_set_error_trace": (_int, [_vp, _i32]),
+    "fs_error_trace": (_int, [_vp, _vp, _vp, _i32, ctypes.POINTER(_i32), _vp]),
+    "fs_block_errors": (_int, [_vp, _vp]),
+    "fs_set_option": (_int, [_vp, _int, _i64]),
+    "fs_iterations_done": (_i64, [_vp]),
+    "fs_launch_count": (_i64, [_vp]),
+    "fs_destroy": (_int, [_vp]),
+    "fs_solve_host": (_int, [_i64, _i32, _vp, _vp, _i64, _int, _dbl, _vp, _vp, _i32, _int, _i32, _vp, _vp, _vp]),
+    "fs_strerror": (ctypes.c_char_p, [_int]),
+    "fs_last_cuda_error": (ctypes.c_char_p, []),
+}
+
+_lib = None
+
+
+class FsError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        detail = ""
+        if code == FS_ERR_CUDA:
+            detail = " [" + lib().fs_last_cuda_error().decode() + "]"
+        super().__init__(f"{where}: {lib().fs_strerror(code).decode()} ({code}){detail}")
+
+
+def lib() -> ctypes.CDLL:
+    """Load libfs_b200.so (built by ``python -m paper_2502_07021_b200.build``); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2502_07021_b200.build` "
+                               "(there is no CPU fallback)")
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = handle
+    return _lib
+
+
+def exported_symbols():
+    return sorted(_SIGNATURES)
+
+
+def _dev(t):
+    """Device address of a torch CUDA tensor (contiguity in the last dimension is the caller's
+    contract), an integer address, or None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    return t.data_ptr()
+
+
+def _stream(s):
+    if s is None:
+        return None
+    if isinstance(s, int):
+        return s
+    return s.cuda_stream
+
+
+def _check(code: int, where: str, allow=()):
+    if code != FS_OK and code not in allow:
+        raise FsError(code, where)
+    return code
+
+
+def _host(arr, dtype):
+    a = np.ascontiguousarray(arr, dtype=dtype)
+    return a, a.ctypes.data_as(_vp)
+
+
+def fs_create(n, c, row_offsets, M_dev, ld, matrix_kind, eps, a_dev, b_dev, nbatch, domain, stream=None):
+    off, offp = _host(row_offsets, np.int64)
+    if off.shape != (c + 1,):
+        raise FsError(FS_ERR_BAD_OFFSETS, "fs_create")
+    out = _vp()
+    _check(lib().fs_create(ctypes.byref(out), n, c, offp, _dev(M_dev), ld, matrix_kind, float(eps), _dev(a_dev),
+                           _dev(b_dev), nbatch, domain, _stream(stream)), "fs_create")
+    return out
+
+
+def fs_iterate(s, k, stream=None):
+    _check(lib().fs_iterate(s, k, _stream(stream)), "fs_iterate")
+
+
+def fs_row_pass(s, stream=None):
+    _check(lib().fs_row_pass(s, _stream(stream)), "fs_row_pass")
+
+
+def fs_col_pass(s, stream=None):
+    _check(lib().fs_col_pass(s, _stream(stream)), "fs_col_pass")
+
+
+def fs_marginal_error(s, norm, nbatch=1, stream=None, allow_nonfinite=False):
+    """Returns (row_err[nbatch], col_err[nbatch]) as float64 numpy arrays."""
+    row = np.zeros(nbatch)
+    col = np.zeros(nbatch)
+    _check(lib().fs_marginal_error(s, norm, row.ctypes.data_as(_vp), col.ctypes.data_as(_vp), _stream(stream)),
+           "fs_marginal_error", allow=(FS_ERR_NONFINITE,) if allow_nonfinite else ())
+    return row, col
+
+
+def fs_scalings(s, u_dev_out, v_dev_out, stream=None):
+    return _check(lib().fs_scalings(s, _dev(u_dev_out), _dev(v_dev_out), _stream(stream)), "fs_scalings")
+
+
+def fs_set_scalings(s, u_dev, v_dev, stream=None):
+    _check(lib().fs_set_scalings(s, _dev(u_dev), _dev(v_dev), _stream(stream)), "fs_set_scalings")
+
+
+def fs_reset(s, stream=None):
+    _check(lib().fs_reset(s, _stream(stream)), "fs_reset")
+
+
+def fs_transport_cost(s, C_dev, ldc, nbatch=1, stream=None):
+    out = np.zeros(nbatch)
+    _check(lib().fs_transport_cost(s, _dev(C_dev), ldc, out.ctypes.data_as(_vp), _stream(stream)), "fs_transport_cost")
+    return out
+
+
+def fs_set_error_trace(s, check_every):
+    _check(lib().fs_set_error_trace(s, check_every), "fs_set_error_trace")
+
+
+def fs_error_trace(s, cap=65536, stream=None):
+    """Returns (l1[count], l2[count])."""
+    l1 = np.zeros(cap)
+    l2 = np.zeros(cap)
+    cnt = _i32(0)
+    _check(lib().fs_error_trace(s, l1.ctypes.data_as(_vp), l2.ctypes.data_as(_vp), cap, ctypes.byref(cnt),
+                                _stream(stream)), "fs_error_trace")
+    m = min(cnt.value, cap)
+    return l1[:m], l2[:m]
+
+
+def fs_block_errors(s, c):
+    out = np.zeros(c)
+    _check(lib().fs_block_errors(s, out.ctypes.data_as(_vp)), "fs_block_errors")
+    return out
+
+
+def fs_set_option(s, option, value):
+    _check(lib().fs_set_option(s, option, value), "fs_set_option")
+
+
+def fs_iterations_done(s):
+    return int(lib().fs_iterations_done(s))
+
+
+def fs_launch_count(s):
+    return int(lib().fs_launch_count(s))
+
+
+def fs_destroy(s):
+    _check(lib().fs_destroy(s), "fs_destroy")
+
+
+def fs_solve_host(n, c, row_offsets, M_host, ld, matrix_kind, eps, a_host, b_host, nbatch, domain, iters,
+                  u_out, v_out, want_error=True):
+    """All buffers are host numpy arrays or pinned torch CPU tensors (float32).  u_out, v_out are
+    written in place; returns the 1-norm row marginal error per problem (or None)."""
+    off, offp = _host(row_offsets, np.int64)
+
+    def hp(x):
+        if x is None:
+            return None
+        if hasattr(x, "data_ptr"):
+            if x.is_cuda:
+                raise ValueError("fs_solve_host takes host buffers")
+            return x.data_ptr()
+        if x.dtype != np.float32 or not x.flags["C_CONTIGUOUS"] and x.ndim == 1:
+            raise ValueError("host buffers must be float32")
+        return x.ctypes.data
+    err = np.zeros(nbatch) if want_error else None
+    _check(lib().fs_solve_host(n, c, offp, hp(M_host), ld, matrix_kind, float(eps), hp(a_host), hp(b_host), nbatch,
+                               domain, iters, hp(u_out), hp(v_out), err.ctypes.data_as(_vp) if want_error else None),
+           "fs_solve_host")
+    return err

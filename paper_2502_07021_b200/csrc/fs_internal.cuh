@@ -1,0 +1,133 @@
+// Internal declarations shared by the translation units of libfs_b200.so.
+// Kernels live in passes.cu (single-problem scaling and log passes), batched.cu (shared-K
+// passes) and setup.cu (one-off and O(n) helpers); fs_api.cu owns the handle and the C ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <map>
+#include <tuple>
+#include <vector>
+
+#include "../../include/fs.h"
+
+// A contiguous range of rows [begin, end) that lies inside one row block I_j.
+struct FsRowTile {
+    int32_t begin;
+    int32_t end;
+};
+
+// Launch shape of the single-problem passes, chosen once per handle from n.
+struct FsPassPlan {
+    int row_L;        // threads that cooperate on a row group (32, 64, 128 or 256)
+    int row_R;        // rows per group
+    int col_TX;       // threads across a column strip (each owns 4 columns)
+    int col_TY;       // row lanes of a CTA in the column pass
+    int col_tile_rows; // maximum height of a row tile
+    bool vec;         // 128-bit loads usable (base and ld 16-byte aligned)
+};
+
+struct FsDeviceStatus {
+    int nonfinite;   // set by any kernel that produced a non-finite or non-positive scaling
+    int trace_count; // number of trace entries appended so far
+};
+
+struct fs_solver {
+    int64_t n = 0, ld = 0;
+    int32_t c = 0, nbatch = 1;
+    int domain = 0, matrix_kind = 0;
+    double eps = 0;
+    std::vector<int64_t> offsets;
+
+    const float *M = nullptr;  // caller's matrix (borrowed)
+    float *K_owned = nullptr;  // K materialised from C (scaling domain, cost input)
+    const float *mat = nullptr; // what the passes stream: K (scaling) or C (log)
+    int64_t mat_ld = 0;
+
+    float *a = nullptr, *b = nullptr;       // [nbatch][n]
+    float *loga = nullptr, *logb = nullptr; // log domain: natural logs of a, b
+    float *x = nullptr, *y = nullptr;       // scaling: u, v   log: f, g      [nbatch][n]
+    float *xs = nullptr, *ys = nullptr;     // log: f*log2(e)/eps, g*log2(e)/eps
+    float *rowdiff = nullptr, *coldiff = nullptr; // P1 - a, P^T1 - b of the last evaluated state
+    float *partials = nullptr;              // column-pass stage-1 partials
+    size_t partials_bytes = 0;
+    int64_t n_pad = 0;                      // n rounded up to a multiple of 4
+
+    FsRowTile *tiles_dev = nullptr;
+    std::vector<FsRowTile> tiles;
+    int64_t *offsets_dev = nullptr;
+    double *block_err = nullptr;            // [c][2] per-block sum |d|, sum d^2 (device)
+    double *err_out = nullptr;              // [nbatch][4] row L1, row sumsq, col L1, col sumsq (device)
+    double *trace = nullptr;                // [cap][2]
+    int32_t trace_cap = 0;
+    int32_t check_every = 0;
+    FsDeviceStatus *status = nullptr;       // device
+    std::vector<double> block_err_host;
+
+    FsPassPlan plan{};
+    int64_t iter_done = 0;
+    int64_t launches = 0;
+    bool use_graph = true;
+    int batch_engine = 0;
+
+    // batched tensor-core path
+    void *tc = nullptr;
+
+    cudaStream_t capture_stream = nullptr;
+    struct GraphEntry {
+        cudaGraphExec_t exec;
+        int64_t launches;
+    };
+    // key: (iterations, iter_done % check_every, check_every, skip first trace, final evaluation)
+    std::map<std::tuple<int, int, int, int, int>, GraphEntry> graphs;
+    int64_t last_traced_iter = 0;
+    double *cost_scratch = nullptr; // [nbatch][n] row sums + [nbatch] totals, allocated on first use
+};
+
+// ---- passes.cu ---------------------------------------------------------------------------
+// Row pass, scaling domain: q_i = sum_l K_il v_l; rowdiff_i = u_i q_i - a_i; if update u_i = a_i/q_i.
+void fsk_row_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, const float *v, const float *a,
+                  float *u, float *rowdiff, int update, FsDeviceStatus *status, cudaStream_t st);
+// Column pass, scaling domain, two deterministic stages.
+void fsk_col_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
+                  int ntiles, const float *u, const float *b, float *v, float *partials, float *coldiff,
+                  int update, FsDeviceStatus *status, cudaStream_t st);
+// Log-domain row pass: L_i = LSE_l((g_l - C_il)/eps) streamed once with a running (max, sum).
+// ys = g * log2(e)/eps on input; writes f and xs = f * log2(e)/eps when update.
+void fsk_log_row_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n, double eps, const float *ys,
+                      const float *a, const float *loga, float *f, float *xs, float *rowdiff, int update,
+                      FsDeviceStatus *status, cudaStream_t st);
+void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n, int64_t n_pad, double eps,
+                      const FsRowTile *tiles, int ntiles, const float *xs, const float *b, const float *logb,
+                      float *g, float *ys, float *partials, float *coldiff, int update,
+                      FsDeviceStatus *status, cudaStream_t st);
+int fsk_pass_launches_row();
+int fsk_pass_launches_col();
+
+// ---- batched.cu --------------------------------------------------------------------------
+// out[p][i] = marg[p][i] / sum_l Mat(i,l) in[p][l], Mat(i,l) = K[i][l] (transposed = 0) or K[l][i].
+// diff[p][i] = out_old[p][i] * sum - marg[p][i].
+void fsk_batched_pass_fma(const float *K, int64_t ld, int64_t n, int nbatch, int transposed, const float *in,
+                          const float *marg, float *out, float *diff, int update, FsDeviceStatus *status,
+                          cudaStream_t st);
+
+// ---- setup.cu ----------------------------------------------------------------------------
+void fsk_materialize_kernel(const float *C, int64_t ldc, int64_t n, float neg_inv_eps, float *K, int64_t ldk,
+                            cudaStream_t st);
+// out[p][0] = min, out[p][1] = sum (double) of x[p][0..n)
+void fsk_min_sum(const float *x, int64_t n, int nbatch, double *out, cudaStream_t st);
+void fsk_fill(float *x, int64_t count, float value, cudaStream_t st);
+void fsk_log(const float *x, int64_t count, float *out, cudaStream_t st);
+// out = (float)((double)x * s)
+void fsk_scale(const float *x, int64_t count, double s, float *out, cudaStream_t st);
+// err[p][0] = sum |d|, err[p][1] = sum d^2 over d = diff[p][0..n); one block per problem, fixed order.
+void fsk_diff_norms(const float *diff, int64_t n, int nbatch, double *err /* [nbatch][2] */, cudaStream_t st);
+// per row block: blk[j][0] = sum |d_i|, blk[j][1] = sum d_i^2 for i in block j (problem 0)
+void fsk_block_norms(const float *diff, const int64_t *offsets_dev, int c, double *blk, cudaStream_t st);
+// append (sum over blocks) to the trace; single thread, fixed order
+void fsk_trace_append(const double *blk, int c, double *trace, int cap, FsDeviceStatus *status, cudaStream_t st);
+// cost[p] = sum_il P_il C_il;  scaling: P = x_i K_il y_l;  log: P = exp2(xs_i + ys_l - C_il * s2)
+void fsk_transport_cost(int domain, const float *mat, int64_t ld, const float *C, int64_t ldc, int64_t n, int nbatch,
+                        const float *x, const float *y, float s2, double *rowsum_scratch, double *cost_dev,
+                        cudaStream_t st);

@@ -1,0 +1,211 @@
+// One-off set-up kernels and the O(n) reductions around the passes: materialising the Gibbs
+// kernel K = exp(-C/eps) (Section 1), input validation scans (assumption A2: a, b > 0 with equal
+// mass), norms of the marginal residuals (Section 5.3, err_a = ||P1 - a||), per-row-block error
+// shares, the error trace, and the transport cost <P,C> (first term of Eq. 1).
+// All reductions use a fixed order (no atomics), so every reported number is reproducible.
+#include <math.h>
+
+#include "fs_internal.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__global__ void __launch_bounds__(kThreads)
+materialize_kernel(const float *__restrict__ C, int64_t ldc, int n, float neg_inv_eps, float *__restrict__ K,
+                   int64_t ldk) {
+    const int row = blockIdx.y;
+    for (int c = blockIdx.x * kThreads + threadIdx.x; c < n; c += gridDim.x * kThreads)
+        K[(int64_t)row * ldk + c] = expf(C[(int64_t)row * ldc + c] * neg_inv_eps);
+}
+
+// Block-wide sum of doubles in a fixed order: every thread's value goes to shared memory and
+// thread 0 of each warp, then thread 0, add them by ascending index.
+__device__ double block_sum_fixed(double x, double *sh /* kThreads */) {
+    sh[threadIdx.x] = x;
+    __syncthreads();
+    for (int w = kThreads / 2; w > 0; w >>= 1) {
+        if ((int)threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
+        __syncthreads();
+    }
+    const double r = sh[0];
+    __syncthreads();
+    return r;
+}
+__device__ double block_min_fixed(double x, double *sh) {
+    sh[threadIdx.x] = x;
+    __syncthreads();
+    for (int w = kThreads / 2; w > 0; w >>= 1) {
+        if ((int)threadIdx.x < w) sh[threadIdx.x] = fmin(sh[threadIdx.x], sh[threadIdx.x + w]);
+        __syncthreads();
+    }
+    const double r = sh[0];
+    __syncthreads();
+    return r;
+}
+
+__global__ void __launch_bounds__(kThreads) min_sum_kernel(const float *__restrict__ x, int64_t n, double *out) {
+    __shared__ double sh[kThreads];
+    const float *xp = x + (int64_t)blockIdx.x * n;
+    double s = 0.0, m = INFINITY;
+    for (int64_t i = threadIdx.x; i < n; i += kThreads) {
+        const double v = (double)xp[i];
+        s += v;
+        m = (v == v) ? fmin(m, v) : -INFINITY; // NaN counts as "not positive"
+    }
+    const double mm = block_min_fixed(m, sh);
+    const double ss = block_sum_fixed(s, sh);
+    if (threadIdx.x == 0) {
+        out[2 * blockIdx.x] = mm;
+        out[2 * blockIdx.x + 1] = ss;
+    }
+}
+
+__global__ void fill_kernel(float *x, int64_t count, float value) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+        x[i] = value;
+}
+__global__ void log_kernel(const float *x, int64_t count, float *out) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+        out[i] = (float)log((double)x[i]);
+}
+__global__ void scale_kernel(const float *x, int64_t count, double s, float *out) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+        out[i] = (float)((double)x[i] * s);
+}
+
+__global__ void __launch_bounds__(kThreads) diff_norms_kernel(const float *__restrict__ diff, int64_t n, double *err) {
+    __shared__ double sh[kThreads];
+    const float *d = diff + (int64_t)blockIdx.x * n;
+    double l1 = 0.0, l2 = 0.0;
+    for (int64_t i = threadIdx.x; i < n; i += kThreads) {
+        const double v = (double)d[i];
+        l1 += fabs(v);
+        l2 += v * v;
+    }
+    const double a = block_sum_fixed(l1, sh);
+    const double b = block_sum_fixed(l2, sh);
+    if (threadIdx.x == 0) {
+        err[2 * blockIdx.x] = a;
+        err[2 * blockIdx.x + 1] = b;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+block_norms_kernel(const float *__restrict__ diff, const int64_t *__restrict__ offsets, double *blk) {
+    __shared__ double sh[kThreads];
+    const int64_t lo = offsets[blockIdx.x], hi = offsets[blockIdx.x + 1];
+    double l1 = 0.0, l2 = 0.0;
+    for (int64_t i = lo + threadIdx.x; i < hi; i += kThreads) {
+        const double v = (double)diff[i];
+        l1 += fabs(v);
+        l2 += v * v;
+    }
+    const double a = block_sum_fixed(l1, sh);
+    const double b = block_sum_fixed(l2, sh);
+    if (threadIdx.x == 0) {
+        blk[2 * blockIdx.x] = a;
+        blk[2 * blockIdx.x + 1] = b;
+    }
+}
+
+__global__ void trace_append_kernel(const double *blk, int c, double *trace, int cap, FsDeviceStatus *status) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    double l1 = 0.0, l2 = 0.0;
+    for (int j = 0; j < c; ++j) {
+        l1 += blk[2 * j];
+        l2 += blk[2 * j + 1];
+    }
+    const int k = status->trace_count;
+    if (k < cap) {
+        trace[2 * k] = l1;
+        trace[2 * k + 1] = sqrt(l2);
+    }
+    status->trace_count = k + 1;
+}
+
+// One warp per (row, problem): rowsum[p][i] = sum_l P_il C_il.
+__global__ void __launch_bounds__(kThreads)
+cost_rows_kernel(int domain, const float *__restrict__ mat, int64_t ld, const float *__restrict__ C, int64_t ldc, int n,
+                 const float *__restrict__ x, const float *__restrict__ y, float s2, double *__restrict__ rowsum) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i = blockIdx.x * (kThreads / 32) + warp;
+    const int p = blockIdx.y;
+    if (i >= n) return;
+    const float *xp = x + (int64_t)p * n, *yp = y + (int64_t)p * n;
+    const float xi = xp[i];
+    double acc = 0.0;
+    for (int l0 = lane; l0 < n; l0 += 32 * 4) {
+        float part = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int l = l0 + 32 * j;
+            if (l < n) {
+                const float cil = C[(int64_t)i * ldc + l];
+                float pil;
+                if (domain == FS_DOMAIN_SCALING) pil = xi * mat[(int64_t)i * ld + l] * yp[l];
+                else pil = exp2f(fmaf(-s2, cil, xi + yp[l]));
+                part = fmaf(pil, cil, part);
+            }
+        }
+        acc += (double)part;
+    }
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (lane == 0) rowsum[(int64_t)p * n + i] = acc;
+}
+
+__global__ void __launch_bounds__(kThreads) sum_rows_kernel(const double *__restrict__ rowsum, int64_t n, double *out) {
+    __shared__ double sh[kThreads];
+    const double *r = rowsum + (int64_t)blockIdx.x * n;
+    double s = 0.0;
+    for (int64_t i = threadIdx.x; i < n; i += kThreads) s += r[i];
+    const double t = block_sum_fixed(s, sh);
+    if (threadIdx.x == 0) out[blockIdx.x] = t;
+}
+
+unsigned grid_for(int64_t count) {
+    int64_t g = (count + kThreads - 1) / kThreads;
+    return (unsigned)(g < 1 ? 1 : (g > 148 * 16 ? 148 * 16 : g));
+}
+
+} // namespace
+
+void fsk_materialize_kernel(const float *C, int64_t ldc, int64_t n, float neg_inv_eps, float *K, int64_t ldk,
+                            cudaStream_t st) {
+    int64_t gx = (n + kThreads - 1) / kThreads;
+    if (gx > 64) gx = 64;
+    // grid.y is limited to 65535 rows per launch
+    for (int64_t r0 = 0; r0 < n; r0 += 65535) {
+        const int64_t rows = n - r0 < 65535 ? n - r0 : 65535;
+        dim3 grid((unsigned)gx, (unsigned)rows);
+        materialize_kernel<<<grid, kThreads, 0, st>>>(C + r0 * ldc, ldc, (int)n, neg_inv_eps, K + r0 * ldk, ldk);
+    }
+}
+void fsk_min_sum(const float *x, int64_t n, int nbatch, double *out, cudaStream_t st) {
+    min_sum_kernel<<<nbatch, kThreads, 0, st>>>(x, n, out);
+}
+void fsk_fill(float *x, int64_t count, float value, cudaStream_t st) {
+    fill_kernel<<<grid_for(count), kThreads, 0, st>>>(x, count, value);
+}
+void fsk_log(const float *x, int64_t count, float *out, cudaStream_t st) {
+    log_kernel<<<grid_for(count), kThreads, 0, st>>>(x, count, out);
+}
+void fsk_scale(const float *x, int64_t count, double s, float *out, cudaStream_t st) {
+    scale_kernel<<<grid_for(count), kThreads, 0, st>>>(x, count, s, out);
+}
+void fsk_diff_norms(const float *diff, int64_t n, int nbatch, double *err, cudaStream_t st) {
+    diff_norms_kernel<<<nbatch, kThreads, 0, st>>>(diff, n, err);
+}
+void fsk_block_norms(const float *diff, const int64_t *offsets_dev, int c, double *blk, cudaStream_t st) {
+    block_norms_kernel<<<c, kThreads, 0, st>>>(diff, offsets_dev, blk);
+}
+void fsk_trace_append(const double *blk, int c, double *trace, int cap, FsDeviceStatus *status, cudaStream_t st) {
+    trace_append_kernel<<<1, 32, 0, st>>>(blk, c, trace, cap, status);
+}
+void fsk_transport_cost(int domain, const float *mat, int64_t ld, const float *C, int64_t ldc, int64_t n, int nbatch,
+                        const float *x, const float *y, float s2, double *rowsum_scratch, double *cost_dev,
+                        cudaStream_t st) {
+    dim3 grid((unsigned)((n + 7) / 8), (unsigned)nbatch);
+    cost_rows_kernel<<<grid, kThreads, 0, st>>>(domain, mat, ld, C, ldc, (int)n, x, y, s2, rowsum_scratch);
+    sum_rows_kernel<<<nbatch, kThreads, 0, st>>>(rowsum_scratch, n, cost_dev);
+}
