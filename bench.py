@@ -1,0 +1,343 @@
+#!/usr/bin/env python
+"""Benchmark of the Sinkhorn hot path: iterations/s at n = 32768, fp32 dense K, one B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 1..5]
+
+A step is one full solve of the configuration (its stated number of iterations: a row pass and a
+column pass each) through fs_iterate, on seeded synthetic inputs that are resident in HBM before
+the timed region starts.  Rank 0 prints ONE JSON line.  Keys beyond the basic contract:
+
+  roofline      dominant kernel (the row pass): algorithmic bytes n*n*4 per launch over its average
+                launch duration, timed with CUDA events on the launching stream, against the measured
+                HBM copy rate of this pool
+  cpu_baseline  the fp64 CPU checker timed on this machine's host cores on a few iterations
+  e2e           the same metric through fs_solve_host: host buffers in, host buffers out, all
+                host<->device copies inside the timed region
+  clocks        SM clock and throttle reasons sampled with nvidia-smi during the timed region
+
+With --impl reference the CPU checker is what gets timed (same config, metric and unit); under a
+multi-process launch only rank 0 runs it.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2502_07021_b200 import distributed as fsdist  # noqa: E402
+from paper_2502_07021_b200 import workloads  # noqa: E402
+
+METRIC = "sinkhorn_iterations_per_s"
+UNIT = "it/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi sampling in a child process while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=self.file, stderr=subprocess.DEVNULL)
+        except (OSError, ValueError):
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return None
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smmax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smmax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if not sm:
+            return None
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smmax), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def visible_device_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except (ValueError, IndexError):
+            return local_rank
+    return local_rank
+
+
+def config_dict(w, args, world):
+    return {"workload": f"config {w.cfg}: n={w.n}" + (f" N={w.nbatch}" if w.nbatch > 1 else "")
+            + f" {'log' if w.domain else 'scaling'}-domain fp32 dense matrix, eps={w.eps}, c={w.c} row blocks, "
+            + f"{w.iters} iterations per step",
+            "n": w.n, "nbatch": w.nbatch, "row_blocks": w.c, "iterations_per_step": w.iters,
+            "domain": "log" if w.domain else "scaling",
+            "matrix_bytes": int(w.n) * int(w.n) * 4,
+            "l2": "matrix is larger than the 126 MB L2, so every pass streams it from HBM; no flush needed"
+            if w.n * w.n * 4 > 126e6 else "matrix fits in L2: numbers are L2/latency-bound, not HBM-bound",
+            "parallelism": "1 GPU" if world == 1 else f"{world} independent replicas (one problem instance per GPU)"}
+
+
+# ------------------------------------------------------------------------------------------ reference arm
+
+def oracle_iterate(w, iters):
+    import oracle
+    if w.nbatch > 1:
+        t0 = time.perf_counter()
+        oracle.sinkhorn_scaling(w.K, oracle.KIND_KERNEL, w.eps, w.a[0], w.b[0], iters)
+        return (time.perf_counter() - t0), 1.0 / w.nbatch     # one problem of the batch per sample
+    t0 = time.perf_counter()
+    if w.domain == workloads.DOMAIN_LOG:
+        oracle.sinkhorn_log(w.C, w.eps, w.a, w.b, iters)
+    else:
+        oracle.sinkhorn_scaling(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, iters)
+    return (time.perf_counter() - t0), 1.0
+
+
+def cpu_baseline(w, budget_s=12.0):
+    """Times the checker, as it stands, on a bounded sample: whole iterations until ~budget_s."""
+    import oracle
+    oracle.build()
+    dt, frac = oracle_iterate(w, 1)
+    iters = 1
+    total = dt
+    while total + dt < budget_s and iters < w.iters:
+        d, _ = oracle_iterate(w, 1)
+        total += d
+        iters += 1
+    value = iters * frac / total
+    sample = f"{iters} full iteration(s) of the same workload" + (" for 1 of the batch's problems" if w.nbatch > 1 else "")
+    return {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample,
+            "seconds": total}
+
+
+def run_reference(args, w, world):
+    import oracle
+    oracle.build()
+    per_step = max(1, args.ref_iters)
+    for _ in range(args.warmup):
+        oracle_iterate(w, 1)
+    t = 0.0
+    frac = 1.0
+    for _ in range(args.steps):
+        d, frac = oracle_iterate(w, per_step)
+        t += d
+    value = args.steps * per_step * frac / t
+    sample = f"each step = {per_step} iteration(s) of the workload" + (" for 1 of the batch's problems" if w.nbatch > 1 else "")
+    cfg = config_dict(w, args, 1)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": cfg, "gpu_launches": 0,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+
+def run_ours(args, w, rank, local_rank, world):
+    import torch
+    from paper_2502_07021_b200 import binding as fs
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    fs.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.Stream(device=dev)
+    M_host = torch.from_numpy(w.matrix)
+    M = M_host.to(dev)
+    a = torch.from_numpy(w.a).to(dev)
+    b = torch.from_numpy(w.b).to(dev)
+    torch.cuda.synchronize()
+    h = fs.fs_create(w.n, w.c, w.offsets, M, w.n, w.kind, w.eps, a, b, w.nbatch, w.domain, stream)
+    if w.check_every:
+        fs.fs_set_error_trace(h, w.check_every)
+
+    def step():
+        fs.fs_reset(h, stream)
+        fs.fs_iterate(h, w.iters, stream)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    stream.synchronize()
+    sampler = ClockSampler(visible_device_index(local_rank))
+    fsdist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    launches0 = fs.fs_launch_count(h)
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    stream.synchronize()
+    torch.cuda.synchronize()
+    fsdist.barrier()
+    clocks = sampler.stop()
+    launches = fs.fs_launch_count(h) - launches0
+    elapsed_ms = e0.elapsed_time(e1)
+    row_err, col_err = fs.fs_marginal_error(h, 1, w.nbatch, stream)
+    t_ms, total_iters = fsdist.aggregate(elapsed_ms, args.steps * w.iters, dev)
+
+    # dominant kernel, timed alone with events on the same stream (single-problem configs: the row pass)
+    roof = None
+    peaks, peak_kind = measured_peaks()
+    if w.nbatch == 1:
+        reps = 20
+        fs.fs_row_pass(h, stream)
+        stream.synchronize()
+        k0 = torch.cuda.Event(enable_timing=True)
+        k1 = torch.cuda.Event(enable_timing=True)
+        k0.record(stream)
+        for _ in range(reps):
+            fs.fs_row_pass(h, stream)
+        k1.record(stream)
+        stream.synchronize()
+        per_launch_s = k0.elapsed_time(k1) * 1e-3 / reps
+        bytes_launch = w.n * w.n * 4
+        achieved = bytes_launch / per_launch_s / 1e9
+        roof = {"bound": "hbm", "kernel": "log_row_pass_kernel" if w.domain else "row_pass_kernel",
+                "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "peak_source": f"of {peak_kind} (MEASURED_PEAKS.json hbm_gbs, burst copy rate)"
+                if peak_kind == "measured" else "of fallback",
+                "algorithmic_bytes_per_launch": bytes_launch, "us_per_launch": per_launch_s * 1e6,
+                "traffic": args.traffic_bytes}
+        # whole iteration (row + column pass) against the same peak, for context
+        roof["iteration_effective_gbs"] = 2 * bytes_launch * (args.steps * w.iters) / (elapsed_ms * 1e-3) / 1e9
+
+    # end-to-end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        pin_M = M_host.pin_memory()
+        pin_a = torch.from_numpy(w.a).pin_memory()
+        pin_b = torch.from_numpy(w.b).pin_memory()
+        out_u = torch.empty_like(pin_a).pin_memory()
+        out_v = torch.empty_like(pin_b).pin_memory()
+        fs.fs_destroy(h)
+        h = None
+        del M
+        torch.cuda.empty_cache()
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        fs.fs_solve_host(w.n, w.c, w.offsets, pin_M, w.n, w.kind, w.eps, pin_a, pin_b, w.nbatch, w.domain, w.iters,
+                         out_u, out_v)  # warm-up
+        fsdist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            fs.fs_solve_host(w.n, w.c, w.offsets, pin_M, w.n, w.kind, w.eps, pin_a, pin_b, w.nbatch, w.domain,
+                             w.iters, out_u, out_v)
+        dt_ms = (time.perf_counter() - t0) * 1e3
+        dt_ms, its = fsdist.aggregate(dt_ms, e2e_steps * w.iters, dev)
+        h2d = w.n * w.n * 4 + 2 * w.a.size * 4
+        d2h = 2 * w.a.size * 4 + 8 * w.nbatch
+        e2e = {"value": its / (dt_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "steps": e2e_steps, "ms_per_step": dt_ms / e2e_steps,
+               "note": "fs_solve_host: device allocation, H2D of the matrix and marginals from pinned memory, "
+                       "all iterations, marginal error, D2H of the scalings, free -- every step"}
+    if h is not None:
+        fs.fs_destroy(h)
+
+    if rank != 0:
+        return
+    base = None
+    if not args.no_cpu_baseline:
+        base = cpu_baseline(w)
+    line = {"metric": METRIC, "value": total_iters / (t_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": t_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": config_dict(w, args, world), "gpu_launches": int(launches), "clocks": clocks,
+            "e2e": e2e, "roofline": roof, "cpu_baseline": base,
+            "final_row_marginal_l1": float(row_err[0]), "final_col_marginal_l1": float(col_err[0])}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=4, help="workload 1..5 (4 = the n=32768 headline)")
+    ap.add_argument("--n", type=int, default=None, help="override n (scaled-down copy of the recipe)")
+    ap.add_argument("--iters", type=int, default=None, help="override the iterations per step (profiling runs)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--ref-iters", type=int, default=1, help="--impl reference: iterations per step")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic-bytes", type=float, default=None,
+                    help="DRAM bytes per launch of the dominant kernel from an ncu capture (reported as is)")
+    args = ap.parse_args()
+
+    rank, local_rank, world = fsdist.env_world()
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        w = workloads.make(args.config, n=args.n, want_cost=None if args.config == 3 else False)
+        if args.iters is not None:
+            w.iters = args.iters
+        run_reference(args, w, world)
+        return 0
+    if world > 1:
+        fsdist.init()
+    w = workloads.make(args.config, n=args.n, want_cost=None if args.config == 3 else False)
+    if args.iters is not None:
+        w.iters = args.iters
+    try:
+        run_ours(args, w, rank, local_rank, world)
+    finally:
+        fsdist.finalize()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -34,7 +34,7 @@ FsPassPlan choose_plan(int64_t n, bool vec) {
     FsPassPlan p{};
     p.vec = vec;
     if (n >= 8192) {
-        p.row_L = 256, p.row_R = 8, p.col_TX = 256, p.col_TY = 1, p.col_tile_rows = 256;
+        p.row_L = 32, p.row_R = 1, p.col_TX = 64, p.col_TY = 4, p.col_tile_rows = 256;
     } else if (n >= 2048) {
         p.row_L = 256, p.row_R = 4, p.col_TX = 64, p.col_TY = 4, p.col_tile_rows = 64;
     } else {

@@ -186,10 +186,14 @@ def check_converged(w, iters, C_for_cost, problems=(0,)):
         ap, bp = (w.a[p], w.b[p]) if batched else (w.a, w.b)
         e = oracle.marginal_errors(w.matrix, w.kind, w.eps, w.domain, xp, yp, ap, bp)
         assert e["row_l1"] <= TOL_L1 and e["col_l1"] <= TOL_L1, (p, e)
-        # the library's own numbers describe the same state
-        assert abs(row_gpu[p] - e["row_l1"]) <= 1e-6
-        assert abs(col_gpu[p] - e["col_l1"]) <= 1e-6
-        assert abs(row2_gpu[p] - e["row_l2"]) <= 1e-6
+        # the library's own numbers describe the same state.  They are computed with the same fp32
+        # sums that produced the scalings, so they can miss the part of the residual that is the
+        # rounding error of those sums: about sqrt(n) * 2^-24 * mass, i.e. ~1e-6 for the batched
+        # path (one chain of n products per output) and far less for the tree-shaped single sums.
+        agree = 3e-6 if batched else 1e-6
+        assert abs(row_gpu[p] - e["row_l1"]) <= agree
+        assert abs(col_gpu[p] - e["col_l1"]) <= agree
+        assert abs(row2_gpu[p] - e["row_l2"]) <= agree
         if C_for_cost is not None:
             ref = oracle.objectives(w.matrix, w.kind, w.eps, w.domain, xp, yp, C_for_cost)["cost"]
             assert abs(cost_gpu[p] - ref) <= TOL_COST * abs(ref)
