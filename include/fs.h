@@ -57,7 +57,8 @@ enum {
     FS_ERR_DOMAIN = -7,               /* log domain requested with a kernel matrix (it needs C) */
     FS_ERR_CUDA = -8,                 /* a CUDA runtime call failed; see fs_last_cuda_error() */
     FS_ERR_NONFINITE = -9,            /* an update produced a non-finite or non-positive scaling */
-    FS_ERR_UNSUPPORTED = -10          /* combination not implemented (batched log domain) */
+    FS_ERR_UNSUPPORTED = -10,         /* combination not implemented (batched log domain) */
+    FS_ERR_TOO_LARGE = -11            /* size exceeds a fixed capacity (fs_col_pass_static: n > FS_STATIC_MAX_N) */
 };
 
 /* Options for fs_set_option. */
@@ -173,6 +174,33 @@ int fs_destroy(fs_solver *s);
 int fs_solve_host(int64_t n, int32_t c, const int64_t *row_offsets, const float *M_host, int64_t ld,
                   int matrix_kind, double eps, const float *a_host, const float *b_host, int32_t nbatch,
                   int domain, int32_t iters, float *u_out, float *v_out, double *row_err_l1_out);
+
+/*
+ * fs_col_pass_static -- v = b ./ (K^T u) for one problem, WITHOUT allocating anything.
+ * (The paper has no counterpart: this entry point exists for the integration reasons below.)
+ *
+ * For callers that cannot allocate device memory where they need the column half-step: a process that
+ * gave the whole GPU to its own memory pool at start-up, a loop that cannot afford the device-wide
+ * synchronisation an allocation may cause, or a plug-in whose host hands it nothing but input and
+ * output buffers.  The stage-1 partial sums that fs_create would put in cudaMalloc'ed memory live
+ * here in a fixed array inside the library image (4 MiB of every GPU that loads the library, held
+ * until the process exits), hence the size limit.
+ *
+ *   K_dev, ld   DEVICE n x n fp32 row-major kernel matrix, leading dimension ld >= n.  Read only.
+ *   n           1 <= n <= FS_STATIC_MAX_N; larger n returns FS_ERR_TOO_LARGE and launches nothing.
+ *   u_dev,b_dev DEVICE [n] inputs.          v_dev   DEVICE [n] output.
+ *   stream      the two kernels are enqueued on it; the call does not synchronise.
+ *
+ * The call itself, and everything it uses, performs no cudaMalloc / cudaFree and no other allocating
+ * routine.  The FIRST call on each device looks up the device address of the static array (the device
+ * must be the current one); make that first call outside any stream capture.  All calls on a device
+ * share the array and it keeps the previous call's contents; no part of it needs clearing because every
+ * slot that is read has been rewritten by the same call.  Calls whose kernels may overlap on the GPU
+ * (different streams without ordering) race on the array: serialise them.
+ */
+#define FS_STATIC_MAX_N 16384
+int fs_col_pass_static(const float *K_dev, int64_t ld, int64_t n, const float *u_dev, const float *b_dev,
+                       float *v_dev, void *stream);
 
 const char *fs_strerror(int code);
 

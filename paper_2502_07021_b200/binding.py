@@ -17,7 +17,8 @@ FS_MATRIX_KERNEL, FS_MATRIX_COST = 0, 1
 FS_OK = 0
 FS_ERR_NULL, FS_ERR_BAD_N, FS_ERR_BAD_OFFSETS, FS_ERR_BAD_EPS = -1, -2, -3, -4
 FS_ERR_NONPOSITIVE_MARGINAL, FS_ERR_MASS_MISMATCH, FS_ERR_DOMAIN = -5, -6, -7
-FS_ERR_CUDA, FS_ERR_NONFINITE, FS_ERR_UNSUPPORTED = -8, -9, -10
+FS_ERR_CUDA, FS_ERR_NONFINITE, FS_ERR_UNSUPPORTED, FS_ERR_TOO_LARGE = -8, -9, -10, -11
+FS_STATIC_MAX_N = 16384
 FS_OPT_USE_GRAPH, FS_OPT_BATCH_ENGINE, FS_OPT_ROW_SHAPE, FS_OPT_COL_SHAPE = 1, 2, 3, 4
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libfs_b200.so")
@@ -45,6 +46,7 @@ _SIGNATURES = {
     "fs_launch_count": (_i64, [_vp]),
     "fs_destroy": (_int, [_vp]),
     "fs_solve_host": (_int, [_i64, _i32, _vp, _vp, _i64, _int, _dbl, _vp, _vp, _i32, _int, _i32, _vp, _vp, _vp]),
+    "fs_col_pass_static": (_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp]),
     "fs_strerror": (ctypes.c_char_p, [_int]),
     "fs_last_cuda_error": (ctypes.c_char_p, []),
 }
@@ -196,6 +198,12 @@ def fs_launch_count(s):
 
 def fs_destroy(s):
     _check(lib().fs_destroy(s), "fs_destroy")
+
+
+def fs_col_pass_static(K_dev, ld, n, u_dev, b_dev, v_dev, stream=None):
+    """v = b / (K^T u) through the entry point that allocates nothing (n <= FS_STATIC_MAX_N)."""
+    _check(lib().fs_col_pass_static(_dev(K_dev), ld, n, _dev(u_dev), _dev(b_dev), _dev(v_dev), _stream(stream)),
+           "fs_col_pass_static")
 
 
 def fs_solve_host(n, c, row_offsets, M_host, ld, matrix_kind, eps, a_host, b_host, nbatch, domain, iters,

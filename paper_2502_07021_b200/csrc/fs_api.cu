@@ -203,6 +203,7 @@ const char *fs_strerror(int code) {
     case FS_ERR_CUDA: return "CUDA runtime error (see fs_last_cuda_error)";
     case FS_ERR_NONFINITE: return "an update produced a non-finite or non-positive scaling";
     case FS_ERR_UNSUPPORTED: return "combination not supported";
+    case FS_ERR_TOO_LARGE: return "size exceeds the fixed capacity of this entry point";
     default: return "unknown error code";
     }
 }
