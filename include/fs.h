@@ -58,13 +58,15 @@ enum {
     FS_ERR_CUDA = -8,                 /* a CUDA runtime call failed; see fs_last_cuda_error() */
     FS_ERR_NONFINITE = -9,            /* an update produced a non-finite or non-positive scaling */
     FS_ERR_UNSUPPORTED = -10,         /* combination not implemented (batched log domain) */
-    FS_ERR_TOO_LARGE = -11            /* size exceeds a fixed capacity (fs_col_pass_static: n > FS_STATIC_MAX_N) */
+    FS_ERR_TOO_LARGE = -11,           /* size exceeds a fixed capacity (fs_col_pass_static: n > FS_STATIC_MAX_N) */
+    FS_ERR_TIMEOUT = -12              /* a bounded wait inside a kernel ran out; the handle's results are invalid */
 };
 
 /* Options for fs_set_option. */
 enum {
     FS_OPT_USE_GRAPH = 1,   /* 1 (default): fs_iterate replays a captured CUDA graph; 0: plain launches */
-    FS_OPT_BATCH_ENGINE = 2, /* batched passes: 0 = auto, 1 = fp32 FMA kernels, 2 = tensor-core kernels */
+    FS_OPT_BATCH_ENGINE = 2, /* batched passes: 0 = auto (tensor cores when nbatch >= 32 and n >= 512),
+                                1 = fp32 FMA kernels, 2 = tensor-core kernels (bf16 hi/lo split, fp32 accumulate) */
     /* Tuning knobs for the single-problem passes (defaults are chosen from n at fs_create): */
     FS_OPT_ROW_SHAPE = 3,   /* value = L*1000 + R: L threads sweep R rows at once; (32,1), (256,4), (256,8) */
     FS_OPT_COL_SHAPE = 4    /* value = TX*1000 + H: TX in {32,64,256} threads across a column strip of 4*TX

@@ -1,0 +1,417 @@
+// Shared-K batched passes on the 5th-generation tensor cores (tcgen05 + TMEM + TMA).
+//
+// With N marginal pairs sharing one K (Section 5.1.1) the passes are dense contractions,
+//   row pass     Q[i][p] = sum_l K[i][l] V[p][l],   U = A ./ Q
+//   column pass  R[l][p] = sum_i K[i][l] U[p][i],   V = B ./ R,
+// at N = 128 about 64 flop per matrix byte: below the tensor-core ridge, so the kernel is shaped
+// to stream K once from HBM and keep the tensor pipe off the critical path.
+//
+// Precision.  fp32 inputs are split into two bf16 terms, x = hi + lo with hi = bf16(x) and
+// lo = bf16(x - hi); the pair carries 16 significand bits (relative error <= 2^-17 per entry).
+// The product keeps three of the four cross terms, hi*hi + hi*lo + lo*hi, accumulated in fp32
+// in tensor memory; the dropped lo*lo term is <= 2^-18 relative.  K is constant over the
+// iterations, so its split is made once at set-up and costs exactly the bytes of the fp32 matrix
+// (2 + 2 bytes per entry); the small operand (the scalings) is re-split by the epilogue that
+// produces it.  Both passes use the same K-major kernel: the column pass reads a transposed
+// split copy of K made at set-up.
+//
+// Kernel: one CTA per (128-row tile of the output, split of the contraction range).  Warp 0
+// issues TMA tile loads (128 x 64 bf16, 128-byte swizzle) into a 3-stage shared-memory ring,
+// warp 1 issues the tcgen05.mma instructions (M = N = 128, K = 16, three per k-step) into a
+// 128-column TMEM accumulator and releases ring slots with tcgen05.commit, warps 2-5 read the
+// accumulator back with tcgen05.ld and store the fp32 partial tile.  A second small kernel adds
+// the partial tiles of the splits in a fixed order and applies the divide, the marginal residual
+// and the bf16 re-split of the new scalings.  Every mbarrier wait is bounded: on expiry the
+// kernel raises a status flag, stops issuing work, drains what it had in flight and exits.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "fs_internal.cuh"
+
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 64, STAGES = 3;
+constexpr int TILE_BYTES = BM * BK * 2;     // one operand tile: 128 rows of 128 bytes
+constexpr int STAGE_BYTES = 4 * TILE_BYTES; // A_hi, A_lo, B_hi, B_lo
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 128;
+constexpr int kTcThreads = 192;
+constexpr int TMEM_COLS = 128;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct TcState {
+    int64_t n = 0, ldb = 0, rows_pad = 0;
+    int nbatch = 0, nb_pad = 0, mtiles = 0, ntiles = 0, kblocks = 0, ksplit = 1;
+    __nv_bfloat16 *K_hi = nullptr, *K_lo = nullptr, *Kt_hi = nullptr, *Kt_lo = nullptr;
+    __nv_bfloat16 *U_hi = nullptr, *U_lo = nullptr, *V_hi = nullptr, *V_lo = nullptr;
+    float *partials = nullptr;
+    CUtensorMap tmK_hi, tmK_lo, tmKt_hi, tmKt_lo, tmU_hi, tmU_lo, tmV_hi, tmV_lo;
+};
+
+// ---- PTX wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok)
+                 : "r"(bar), "r"(parity)
+                 : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it > 128) __nanosleep(64);
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(const CUtensorMap *map, uint32_t dst, uint32_t bar, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
+    uint32_t r[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr)
+                 : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+}
+
+// Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes with the 128-byte
+// swizzle: 8-row groups 1024 bytes apart (stride byte offset), descriptor version 1.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+    d |= (uint64_t)1 << 16;          // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32; // stride byte offset
+    d |= (uint64_t)1 << 46;          // version
+    d |= (uint64_t)2 << 61;          // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: D = fp32, A = B = bf16, both K-major, N = 128, M = 128.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+// ---- GEMM kernel -------------------------------------------------------------------------
+// blockIdx.x = output row tile, blockIdx.y = split of the contraction range, blockIdx.z = tile of problems.
+__global__ void __launch_bounds__(kTcThreads, 1)
+batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_constant__ CUtensorMap tmA_lo,
+                  const __grid_constant__ CUtensorMap tmB_hi, const __grid_constant__ CUtensorMap tmB_lo,
+                  float *__restrict__ partials, int kblocks, int ksplit, FsDeviceStatus *status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bars = base + STAGES * STAGE_BYTES; // full[STAGES], empty[STAGES], accum
+    const uint32_t tmem_slot = bars + 8 * (2 * STAGES + 1);
+    uint32_t *tmem_slot_ptr = reinterpret_cast<uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int mtile = blockIdx.x, ks = blockIdx.y, ntile = blockIdx.z;
+    const int kb0 = (int)((int64_t)kblocks * ks / ksplit), kb1 = (int)((int64_t)kblocks * (ks + 1) / ksplit);
+    const int nkb = kb1 - kb0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bars + 8 * s, 1);
+            mbar_init(bars + 8 * (STAGES + s), 1);
+        }
+        mbar_init(bars + 8 * 2 * STAGES, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot_ptr;
+    bool ok = true;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int it = 0; it < nkb; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                if (!mbar_wait(bars + 8 * (STAGES + s), ph ^ 1u)) { ok = false; break; }
+                const uint32_t full = bars + 8 * s;
+                const uint32_t dst = base + s * STAGE_BYTES;
+                mbar_expect_tx(full, STAGE_BYTES);
+                const int x = (kb0 + it) * BK;
+                tma_load_2d(&tmA_hi, dst, full, x, mtile * BM);
+                tma_load_2d(&tmA_lo, dst + TILE_BYTES, full, x, mtile * BM);
+                tma_load_2d(&tmB_hi, dst + 2 * TILE_BYTES, full, x, ntile * BN);
+                tma_load_2d(&tmB_lo, dst + 3 * TILE_BYTES, full, x, ntile * BN);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int it = 0;
+            for (; it < nkb; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                if (!mbar_wait(bars + 8 * s, ph)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t st = base + s * STAGE_BYTES;
+                const uint64_t a_hi = make_desc(st), a_lo = make_desc(st + TILE_BYTES);
+                const uint64_t b_hi = make_desc(st + 2 * TILE_BYTES), b_lo = make_desc(st + 3 * TILE_BYTES);
+#pragma unroll
+                for (int kk = 0; kk < BK / 16; ++kk) {
+                    const uint64_t adv = (uint64_t)(kk * 32 >> 4); // 16 bf16 = 32 bytes along K
+                    tc_mma_bf16(tmem, a_lo + adv, b_hi + adv, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+                    tc_mma_bf16(tmem, a_hi + adv, b_lo + adv, kIdesc, 1u);
+                    tc_mma_bf16(tmem, a_hi + adv, b_hi + adv, kIdesc, 1u);
+                }
+                tc_commit(bars + 8 * (STAGES + s)); // frees the ring slot when these MMAs have read it
+            }
+            if (ok) {
+                tc_commit(bars + 8 * 2 * STAGES);   // accumulator complete
+            } else {
+                // drain: loads already issued into later slots must land before the CTA exits
+                for (int j = it; j < nkb && j < it + STAGES; ++j)
+                    (void)mbar_wait(bars + 8 * (j % STAGES), (uint32_t)(j / STAGES) & 1u);
+            }
+        }
+    } else {
+        // epilogue warps 2..5: TMEM lane quarter = warp % 4
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        if (nkb > 0) ok = mbar_wait(bars + 8 * 2 * STAGES, 0);
+        ok = __all_sync(0xffffffffu, ok);
+        tc_fence_after();
+        const int unit = ((ntile * gridDim.x + mtile) * ksplit + ks);
+        float *out = partials + (size_t)unit * (BM * BN) + row;
+        if (ok) {
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                float v[32];
+                if (nkb > 0) {
+                    tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), v);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < 32; ++j) out[(size_t)(c * 32 + j) * BM] = v[j];
+            }
+        }
+    }
+    if (!ok) status->timeout = 1;
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- epilogue over the partial tiles -----------------------------------------------------
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
+    hi = __float2bfloat16_rn(x);
+    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+__global__ void __launch_bounds__(256)
+batched_tc_finish_kernel(const float *__restrict__ partials, int ksplit, int n, int nbatch, int64_t ldb,
+                         const float *__restrict__ marg, float *__restrict__ out, float *__restrict__ diff,
+                         __nv_bfloat16 *__restrict__ op_hi, __nv_bfloat16 *__restrict__ op_lo, int update,
+                         FsDeviceStatus *status) {
+    const int mtile = blockIdx.x, ntile = blockIdx.y;
+    const float *base = partials + (size_t)((ntile * gridDim.x + mtile) * ksplit) * (BM * BN);
+    for (int e = threadIdx.x; e < BM * BN; e += 256) {
+        const int p = e / BM, i = e % BM;
+        const int gi = mtile * BM + i, gp = ntile * BN + p;
+        if (gi >= n || gp >= nbatch) continue;
+        float q = 0.f;
+        for (int k = 0; k < ksplit; ++k) q += base[(size_t)k * (BM * BN) + e];
+        const int64_t idx = (int64_t)gp * n + gi;
+        const float mg = marg[idx], old = out[idx];
+        diff[idx] = fmaf(old, q, -mg);
+        if (update) {
+            const float nv = mg / q;
+            out[idx] = nv;
+            __nv_bfloat16 hi, lo;
+            split_bf16(nv, hi, lo);
+            op_hi[(int64_t)gp * ldb + gi] = hi;
+            op_lo[(int64_t)gp * ldb + gi] = lo;
+            if (!(nv > 0.f) || isinf(nv)) status->nonfinite = 1;
+        }
+    }
+}
+
+// ---- set-up kernels ----------------------------------------------------------------------
+// hi/lo split of the n x n fp32 matrix, written both as stored and transposed (32 x 32 tiles
+// through shared memory so that both writes are coalesced).
+__global__ void __launch_bounds__(256)
+split_matrix_kernel(const float *__restrict__ K, int64_t ld, int n, int64_t ldb, __nv_bfloat16 *__restrict__ hi,
+                    __nv_bfloat16 *__restrict__ lo, __nv_bfloat16 *__restrict__ thi, __nv_bfloat16 *__restrict__ tlo) {
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x % 32, ty = threadIdx.x / 32; // 32 x 8
+    const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    for (int j = ty; j < 32; j += 8) {
+        const int r = r0 + j, c = c0 + tx;
+        float v = 0.f;
+        if (r < n && c < n) {
+            v = K[(int64_t)r * ld + c];
+            __nv_bfloat16 h, l;
+            split_bf16(v, h, l);
+            hi[(int64_t)r * ldb + c] = h;
+            lo[(int64_t)r * ldb + c] = l;
+        }
+        tile[j][tx] = v;
+    }
+    __syncthreads();
+    for (int j = ty; j < 32; j += 8) {
+        const int r = c0 + j, c = r0 + tx; // transposed coordinates
+        if (r < n && c < n) {
+            __nv_bfloat16 h, l;
+            split_bf16(tile[tx][j], h, l);
+            thi[(int64_t)r * ldb + c] = h;
+            tlo[(int64_t)r * ldb + c] = l;
+        }
+    }
+}
+
+__global__ void split_vectors_kernel(const float *__restrict__ x, int n, int nbatch, int64_t ldb,
+                                     __nv_bfloat16 *__restrict__ hi, __nv_bfloat16 *__restrict__ lo) {
+    const int p = blockIdx.y;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        __nv_bfloat16 h, l;
+        split_bf16(x[(int64_t)p * n + i], h, l);
+        hi[(int64_t)p * ldb + i] = h;
+        lo[(int64_t)p * ldb + i] = l;
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// rows x cols bf16 matrix, row pitch ldb elements; box = 64 columns x 128 rows, 128-byte swizzle
+bool make_map(CUtensorMap *map, const __nv_bfloat16 *ptr, int64_t rows, int64_t cols, int64_t ldb) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ldb * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16 *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+void tc_free(TcState *t) {
+    if (!t) return;
+    cudaFree(t->K_hi), cudaFree(t->K_lo), cudaFree(t->Kt_hi), cudaFree(t->Kt_lo);
+    cudaFree(t->U_hi), cudaFree(t->U_lo), cudaFree(t->V_hi), cudaFree(t->V_lo);
+    cudaFree(t->partials);
+    delete t;
+}
+
+} // namespace
+
+void fsk_tc_destroy(void *tc) { tc_free(static_cast<TcState *>(tc)); }
+
+// Builds the split operands, tensor maps and partial-tile buffer.  Returns nullptr on failure
+// (the caller then stays on the FMA engine).
+void *fsk_tc_create(const float *K, int64_t ld, int64_t n, int nbatch, cudaStream_t st) {
+    if (!encode_fn()) return nullptr;
+    TcState *t = new TcState();
+    t->n = n, t->nbatch = nbatch;
+    t->ldb = (n + BK - 1) / BK * BK;
+    t->rows_pad = (n + BM - 1) / BM * BM;
+    t->nb_pad = (nbatch + BN - 1) / BN * BN;
+    t->mtiles = (int)(t->rows_pad / BM), t->ntiles = t->nb_pad / BN, t->kblocks = (int)(t->ldb / BK);
+    int ks = 148 / (t->mtiles * t->ntiles);
+    if (ks < 1) ks = 1;
+    if (ks > t->kblocks) ks = t->kblocks;
+    if (ks > 16) ks = 16;
+    t->ksplit = ks;
+    const size_t mat_bytes = (size_t)t->rows_pad * t->ldb * 2, vec_bytes = (size_t)t->nb_pad * t->ldb * 2;
+    const size_t part_bytes = (size_t)t->mtiles * t->ntiles * t->ksplit * BM * BN * sizeof(float);
+    bool ok = true;
+    __nv_bfloat16 **mats[4] = {&t->K_hi, &t->K_lo, &t->Kt_hi, &t->Kt_lo};
+    __nv_bfloat16 **vecs[4] = {&t->U_hi, &t->U_lo, &t->V_hi, &t->V_lo};
+    for (auto m : mats) ok = ok && cudaMalloc(m, mat_bytes) == cudaSuccess && cudaMemsetAsync(*m, 0, mat_bytes, st) == cudaSuccess;
+    for (auto v : vecs) ok = ok && cudaMalloc(v, vec_bytes) == cudaSuccess && cudaMemsetAsync(*v, 0, vec_bytes, st) == cudaSuccess;
+    ok = ok && cudaMalloc(&t->partials, part_bytes) == cudaSuccess;
+    if (ok) {
+        dim3 grid((unsigned)((n + 31) / 32), (unsigned)((n + 31) / 32));
+        split_matrix_kernel<<<grid, 256, 0, st>>>(K, ld, (int)n, t->ldb, t->K_hi, t->K_lo, t->Kt_hi, t->Kt_lo);
+        ok = cudaGetLastError() == cudaSuccess;
+    }
+    ok = ok && make_map(&t->tmK_hi, t->K_hi, t->rows_pad, t->ldb, t->ldb) && make_map(&t->tmK_lo, t->K_lo, t->rows_pad, t->ldb, t->ldb) &&
+         make_map(&t->tmKt_hi, t->Kt_hi, t->rows_pad, t->ldb, t->ldb) && make_map(&t->tmKt_lo, t->Kt_lo, t->rows_pad, t->ldb, t->ldb) &&
+         make_map(&t->tmU_hi, t->U_hi, t->nb_pad, t->ldb, t->ldb) && make_map(&t->tmU_lo, t->U_lo, t->nb_pad, t->ldb, t->ldb) &&
+         make_map(&t->tmV_hi, t->V_hi, t->nb_pad, t->ldb, t->ldb) && make_map(&t->tmV_lo, t->V_lo, t->nb_pad, t->ldb, t->ldb);
+    ok = ok && cudaFuncSetAttribute(batched_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        tc_free(t);
+        return nullptr;
+    }
+    return t;
+}
+
+// Re-split the current scalings into the bf16 operand buffers (after a reset or fs_set_scalings).
+void fsk_tc_refresh(void *tc, const float *u, const float *v, cudaStream_t st) {
+    TcState *t = static_cast<TcState *>(tc);
+    dim3 grid((unsigned)((t->n + 255) / 256 > 64 ? 64 : (t->n + 255) / 256), (unsigned)t->nbatch);
+    if (u) split_vectors_kernel<<<grid, 256, 0, st>>>(u, (int)t->n, t->nbatch, t->ldb, t->U_hi, t->U_lo);
+    if (v) split_vectors_kernel<<<grid, 256, 0, st>>>(v, (int)t->n, t->nbatch, t->ldb, t->V_hi, t->V_lo);
+}
+
+// One batched pass on the tensor-core engine; two launches.
+void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float *diff, int update,
+                 FsDeviceStatus *status, cudaStream_t st) {
+    TcState *t = static_cast<TcState *>(tc);
+    dim3 grid((unsigned)t->mtiles, (unsigned)t->ksplit, (unsigned)t->ntiles);
+    if (!transposed)
+        batched_tc_kernel<<<grid, kTcThreads, SMEM_BYTES, st>>>(t->tmK_hi, t->tmK_lo, t->tmV_hi, t->tmV_lo, t->partials,
+                                                              t->kblocks, t->ksplit, status);
+    else
+        batched_tc_kernel<<<grid, kTcThreads, SMEM_BYTES, st>>>(t->tmKt_hi, t->tmKt_lo, t->tmU_hi, t->tmU_lo, t->partials,
+                                                              t->kblocks, t->ksplit, status);
+    dim3 fgrid((unsigned)t->mtiles, (unsigned)t->ntiles);
+    batched_tc_finish_kernel<<<fgrid, 256, 0, st>>>(t->partials, t->ksplit, (int)t->n, t->nbatch, t->ldb, marg, out, diff,
+                                                   transposed ? t->V_hi : t->U_hi, transposed ? t->V_lo : t->U_lo, update,
+                                                   status);
+}

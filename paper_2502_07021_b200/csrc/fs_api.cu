@@ -29,6 +29,8 @@ int cuda_fail(cudaError_t e, const char *what) {
 constexpr double kLog2e = 1.4426950408889634;
 constexpr int kGraphChunk = 64;
 constexpr int kTraceCap = 1 << 16;
+constexpr int kTcMinBatch = 32;
+constexpr int kTcMinN = 512;
 
 FsPassPlan choose_plan(int64_t n, bool vec) {
     FsPassPlan p{};
@@ -85,6 +87,7 @@ void destroy_solver(fs_solver *s) {
     free_dev(s->trace);
     free_dev(s->status);
     free_dev(s->cost_scratch);
+    if (s->tc) fsk_tc_destroy(s->tc);
     delete s;
 }
 
@@ -104,8 +107,13 @@ int upload_tiles(fs_solver *s) {
 
 // ---- enqueue helpers ---------------------------------------------------------------------
 
+bool use_tc(const fs_solver *s) { return s->tc != nullptr && s->batch_engine != 1; }
+
 void enqueue_row(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
-    if (s->nbatch > 1) {
+    if (s->nbatch > 1 && use_tc(s)) {
+        fsk_tc_pass(s->tc, 0, s->a, s->x, s->rowdiff, update, s->status, st);
+        launches += 2;
+    } else if (s->nbatch > 1) {
         fsk_batched_pass_fma(s->mat, s->mat_ld, s->n, s->nbatch, 0, s->y, s->a, s->x, s->rowdiff, update, s->status, st);
         launches += 1;
     } else if (s->domain == FS_DOMAIN_SCALING) {
@@ -119,7 +127,10 @@ void enqueue_row(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
 }
 
 void enqueue_col(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
-    if (s->nbatch > 1) {
+    if (s->nbatch > 1 && use_tc(s)) {
+        fsk_tc_pass(s->tc, 1, s->b, s->y, s->coldiff, update, s->status, st);
+        launches += 2;
+    } else if (s->nbatch > 1) {
         fsk_batched_pass_fma(s->mat, s->mat_ld, s->n, s->nbatch, 1, s->x, s->b, s->y, s->coldiff, update, s->status, st);
         launches += 1;
     } else if (s->domain == FS_DOMAIN_SCALING) {
@@ -162,6 +173,11 @@ int check_status(fs_solver *s, cudaStream_t st) {
     FsDeviceStatus h{};
     FS_CU(cudaMemcpyAsync(&h, s->status, sizeof(h), cudaMemcpyDeviceToHost, st));
     FS_CU(cudaStreamSynchronize(st));
+    if (h.timeout) {
+        FS_CU(cudaMemsetAsync(&s->status->timeout, 0, sizeof(int), st));
+        FS_CU(cudaStreamSynchronize(st));
+        return FS_ERR_TIMEOUT;
+    }
     if (h.nonfinite) {
         FS_CU(cudaMemsetAsync(&s->status->nonfinite, 0, sizeof(int), st));
         FS_CU(cudaStreamSynchronize(st));
@@ -179,6 +195,7 @@ int set_initial_state(fs_solver *s, cudaStream_t st) {
         fsk_fill(s->xs, cnt, 0.f, st);
         fsk_fill(s->ys, cnt, 0.f, st);
     }
+    if (s->tc) fsk_tc_refresh(s->tc, s->x, s->y, st);
     FS_CU(cudaMemsetAsync(s->status, 0, sizeof(FsDeviceStatus), st));
     FS_CU(cudaGetLastError());
     s->iter_done = 0;
@@ -204,6 +221,7 @@ const char *fs_strerror(int code) {
     case FS_ERR_NONFINITE: return "an update produced a non-finite or non-positive scaling";
     case FS_ERR_UNSUPPORTED: return "combination not supported";
     case FS_ERR_TOO_LARGE: return "size exceeds the fixed capacity of this entry point";
+    case FS_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     default: return "unknown error code";
     }
 }
@@ -300,6 +318,8 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
     s->plan = choose_plan(n, vec);
     int rc = upload_tiles(s);
     if (rc != FS_OK) return rc;
+    // batched problems: tensor-core engine when the batch is wide enough to fill its 128-problem tiles
+    if (nbatch >= kTcMinBatch && n >= kTcMinN) s->tc = fsk_tc_create(s->mat, s->mat_ld, n, nbatch, st);
     rc = set_initial_state(s, st);
     if (rc != FS_OK) return rc;
     FS_CU(cudaStreamSynchronize(st));
@@ -324,7 +344,16 @@ int fs_set_option(fs_solver *s, int option, int64_t value) {
         return FS_OK;
     case FS_OPT_BATCH_ENGINE:
         if (value < 0 || value > 2) return FS_ERR_BAD_N;
-        if (value == 2) return FS_ERR_UNSUPPORTED;
+        if (s->nbatch < 2) return value == 2 ? FS_ERR_UNSUPPORTED : FS_OK;
+        cudaDeviceSynchronize();
+        if (value == 2 && !s->tc) {
+            s->tc = fsk_tc_create(s->mat, s->mat_ld, s->n, s->nbatch, nullptr);
+            if (!s->tc) return FS_ERR_UNSUPPORTED;
+        }
+        if (value != 1 && s->tc) {
+            fsk_tc_refresh(s->tc, s->x, s->y, nullptr);
+            cudaDeviceSynchronize();
+        }
         s->batch_engine = (int)value;
         destroy_graphs(s);
         return FS_OK;
@@ -469,6 +498,10 @@ int fs_set_scalings(fs_solver *s, const float *u_dev, const float *v_dev, void *
     const size_t bytes = sizeof(float) * (size_t)cnt;
     if (u_dev) FS_CU(cudaMemcpyAsync(s->x, u_dev, bytes, cudaMemcpyDeviceToDevice, st));
     if (v_dev) FS_CU(cudaMemcpyAsync(s->y, v_dev, bytes, cudaMemcpyDeviceToDevice, st));
+    if (s->tc) {
+        fsk_tc_refresh(s->tc, u_dev ? s->x : nullptr, v_dev ? s->y : nullptr, st);
+        FS_CU(cudaGetLastError());
+    }
     if (s->domain == FS_DOMAIN_LOG) {
         if (u_dev) fsk_scale(s->x, cnt, kLog2e / s->eps, s->xs, st);
         if (v_dev) fsk_scale(s->y, cnt, kLog2e / s->eps, s->ys, st);

@@ -31,6 +31,7 @@ struct FsPassPlan {
 struct FsDeviceStatus {
     int nonfinite;   // set by any kernel that produced a non-finite or non-positive scaling
     int trace_count; // number of trace entries appended so far
+    int timeout;     // a bounded device-side wait ran out (tensor-core engine)
 };
 
 struct fs_solver {
@@ -111,6 +112,14 @@ int fsk_pass_launches_col();
 void fsk_batched_pass_fma(const float *K, int64_t ld, int64_t n, int nbatch, int transposed, const float *in,
                           const float *marg, float *out, float *diff, int update, FsDeviceStatus *status,
                           cudaStream_t st);
+
+// ---- batched_tc.cu -----------------------------------------------------------------------
+// Tensor-core engine for the batched passes (bf16 hi/lo split operands, fp32 accumulation).
+void *fsk_tc_create(const float *K, int64_t ld, int64_t n, int nbatch, cudaStream_t st); // nullptr on failure
+void fsk_tc_destroy(void *tc);
+void fsk_tc_refresh(void *tc, const float *u, const float *v, cudaStream_t st);
+void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float *diff, int update,
+                 FsDeviceStatus *status, cudaStream_t st);
 
 // ---- setup.cu ----------------------------------------------------------------------------
 void fsk_materialize_kernel(const float *C, int64_t ldc, int64_t n, float neg_inv_eps, float *K, int64_t ldk,

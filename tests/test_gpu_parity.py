@@ -150,6 +150,27 @@ def test_config5_scaled_down_ten_iterations(n, nb):
     batched_sample(w, U, V, 10, sorted({0, 1, nb // 2, nb - 1}))
 
 
+@pytest.mark.parametrize("n,nb", [(512, 32), (1000, 40), (2048, 128)])
+def test_batched_engines_agree(n, nb):
+    """The fp32 FMA engine and the tensor-core engine (bf16 hi/lo split, fp32 accumulation) run the
+    same problem; both must meet the tolerance against the oracle and agree with each other."""
+    w = workloads.make(5, n=n, nbatch=nb)
+    res = {}
+    for engine in (1, 2):
+        with GpuSolver(w.K, KK, w.eps, w.a, w.b, w.offsets, SC) as g:
+            fs.fs_set_option(g.h, fs.FS_OPT_BATCH_ENGINE, engine)
+            g.iterate(10)
+            res[engine] = g.scalings()
+    for engine in (1, 2):
+        batched_sample(w, res[engine][0], res[engine][1], 10, sorted({0, nb // 2, nb - 1}))
+    assert rel_err(res[2][0], res[1][0]) < 5e-5 and rel_err(res[2][1], res[1][1]) < 5e-5
+
+
+def test_batched_tensor_core_engine_converges():
+    w = workloads.make(5, n=1024, nbatch=64)
+    check_converged(w, w.iters, w.C, problems=(0, 33, 63))
+
+
 @pytest.mark.slow
 def test_config3_full_size_ten_iterations():
     check_ten_iterations(workloads.make(3))
