@@ -29,6 +29,7 @@ int cuda_fail(cudaError_t e, const char *what) {
 constexpr double kLog2e = 1.4426950408889634;
 constexpr int kGraphChunk = 64;
 constexpr int kTraceCap = 1 << 16;
+constexpr int64_t kFusedAutoMinN = 12288;
 constexpr int kTcMinBatch = 32;
 constexpr int kTcMinN = 512;
 
@@ -81,6 +82,8 @@ void destroy_solver(fs_solver *s) {
     free_dev(s->coldiff);
     free_dev(s->partials);
     free_dev(s->tiles_dev);
+    free_dev(s->fused_tiles_dev);
+    free_dev(s->fused_partials);
     free_dev(s->offsets_dev);
     free_dev(s->block_err);
     free_dev(s->err_out);
@@ -144,6 +147,23 @@ void enqueue_col(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
     }
 }
 
+// The single-read fused iteration replaces row pass + column stage 1 when it applies.
+bool use_fused(const fs_solver *s) {
+    if (!s->fused.enabled || s->fused_mode == 0) return false;
+    return s->fused_mode == 2 || s->n >= kFusedAutoMinN;
+}
+
+void enqueue_fused_rows(fs_solver *s, cudaStream_t st, int64_t &launches) {
+    fsk_fused_iteration(s->fused, s->mat, s->mat_ld, s->n, s->fused_tiles_dev, s->fused_ntiles, s->y, s->a, s->x,
+                        s->rowdiff, s->fused_partials, s->status, st);
+    launches += 1;
+}
+
+void enqueue_fused_finish(fs_solver *s, cudaStream_t st, int64_t &launches) {
+    fsk_col_finish(s->n, s->n, s->fused.nclusters, s->fused_partials, s->b, s->y, s->coldiff, 1, s->status, st);
+    launches += 1;
+}
+
 void enqueue_trace(fs_solver *s, cudaStream_t st, int64_t &launches) {
     fsk_block_norms(s->rowdiff, s->offsets_dev, s->c, s->block_err, st);
     fsk_trace_append(s->block_err, s->c, s->trace, s->trace_cap, s->status, st);
@@ -157,11 +177,14 @@ void enqueue_trace(fs_solver *s, cudaStream_t st, int64_t &launches) {
 void enqueue_range(fs_solver *s, int phase, int len, bool trace_first, bool final_eval, cudaStream_t st,
                    int64_t &launches) {
     const int ce = s->check_every;
+    const bool fused = use_fused(s);
     for (int it = 0; it < len; ++it) {
-        enqueue_row(s, 1, st, launches);
+        if (fused) enqueue_fused_rows(s, st, launches);
+        else enqueue_row(s, 1, st, launches);
         const bool check = it == 0 ? trace_first : (ce > 0 && (phase + it) % ce == 0);
         if (check) enqueue_trace(s, st, launches);
-        enqueue_col(s, 1, st, launches);
+        if (fused) enqueue_fused_finish(s, st, launches);
+        else enqueue_col(s, 1, st, launches);
     }
     if (final_eval) {
         enqueue_row(s, 0, st, launches);
@@ -318,6 +341,17 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
     s->plan = choose_plan(n, vec);
     int rc = upload_tiles(s);
     if (rc != FS_OK) return rc;
+    if (domain == FS_DOMAIN_SCALING && nbatch == 1) {
+        s->fused = fsk_fused_plan(n, vec);
+        if (s->fused.enabled) {
+            const std::vector<FsRowTile> ft = build_tiles(s->offsets, s->fused.tile_rows);
+            s->fused_ntiles = (int)ft.size();
+            FS_CU(cudaMalloc(&s->fused_tiles_dev, sizeof(FsRowTile) * ft.size()));
+            FS_CU(cudaMemcpy(s->fused_tiles_dev, ft.data(), sizeof(FsRowTile) * ft.size(), cudaMemcpyHostToDevice));
+            FS_CU(cudaMalloc(&s->fused_partials, sizeof(float) * (size_t)s->fused.nclusters * (size_t)n));
+            FS_CU(cudaMemsetAsync(s->fused_partials, 0, sizeof(float) * (size_t)s->fused.nclusters * (size_t)n, st));
+        }
+    }
     // batched problems: tensor-core engine when the batch is wide enough to fill its 128-problem tiles
     if (nbatch >= kTcMinBatch && n >= kTcMinN) s->tc = fsk_tc_create(s->mat, s->mat_ld, n, nbatch, st);
     rc = set_initial_state(s, st);
@@ -355,6 +389,12 @@ int fs_set_option(fs_solver *s, int option, int64_t value) {
             cudaDeviceSynchronize();
         }
         s->batch_engine = (int)value;
+        destroy_graphs(s);
+        return FS_OK;
+    case FS_OPT_FUSED:
+        if (value < 0 || value > 2) return FS_ERR_BAD_N;
+        if (value == 2 && !s->fused.enabled) return FS_ERR_UNSUPPORTED;
+        s->fused_mode = (int)value;
         destroy_graphs(s);
         return FS_OK;
     case FS_OPT_ROW_SHAPE: {

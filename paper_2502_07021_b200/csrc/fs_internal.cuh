@@ -28,6 +28,16 @@ struct FsPassPlan {
     bool vec;         // 128-bit loads usable (base and ld 16-byte aligned)
 };
 
+// Configuration of the single-read fused iteration (fused.cu); enabled = false when it does not apply.
+struct FsFusedPlan {
+    bool enabled;
+    int S;         // CTAs per cluster (column segments per row)
+    int F;         // 128-bit column groups per thread: a CTA covers F*1024 columns
+    int nstages;   // shared-memory ring depth (row segments in flight per CTA)
+    int nclusters; // clusters resident at once = number of column-partial rows
+    int tile_rows; // height of the row tiles dealt to the clusters
+};
+
 struct FsDeviceStatus {
     int nonfinite;   // set by any kernel that produced a non-finite or non-positive scaling
     int trace_count; // number of trace entries appended so far
@@ -67,6 +77,11 @@ struct fs_solver {
     std::vector<double> block_err_host;
 
     FsPassPlan plan{};
+    FsFusedPlan fused{};
+    int fused_mode = 1;                     // 0 = never, 1 = automatic, 2 = whenever it applies
+    FsRowTile *fused_tiles_dev = nullptr;
+    int fused_ntiles = 0;
+    float *fused_partials = nullptr;
     int64_t iter_done = 0;
     int64_t launches = 0;
     bool use_graph = true;
@@ -103,8 +118,17 @@ void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n
                       const FsRowTile *tiles, int ntiles, const float *xs, const float *b, const float *logb,
                       float *g, float *ys, float *partials, float *coldiff, int update,
                       FsDeviceStatus *status, cudaStream_t st);
+// Stage 2 of the column pass alone: r_l = sum over `ntiles` partial rows of pitch n_pad, residual, divide.
+void fsk_col_finish(int64_t n, int64_t n_pad, int ntiles, const float *partials, const float *b, float *v,
+                    float *coldiff, int update, FsDeviceStatus *status, cudaStream_t st);
 int fsk_pass_launches_row();
 int fsk_pass_launches_col();
+
+// ---- fused.cu ----------------------------------------------------------------------------
+FsFusedPlan fsk_fused_plan(int64_t n, bool vec);
+cudaError_t fsk_fused_iteration(const FsFusedPlan &p, const float *K, int64_t ld, int64_t n, const FsRowTile *tiles,
+                                int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials,
+                                FsDeviceStatus *status, cudaStream_t st);
 
 // ---- batched.cu --------------------------------------------------------------------------
 // out[p][i] = marg[p][i] / sum_l Mat(i,l) in[p][l], Mat(i,l) = K[i][l] (transposed = 0) or K[l][i].

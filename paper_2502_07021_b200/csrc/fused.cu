@@ -1,0 +1,363 @@
+// Single-read fused iteration, scaling domain, one problem.
+//
+// One Sinkhorn iteration (Algorithm 1, loop body) needs every entry of K twice: once for
+// q = K v and, after u = a ./ q is known, once more for r = K^T u.  A row of K only needs its own
+// q_i before it can be reused, so a CTA pair that holds a whole row on chip can do both with ONE
+// read of K from HBM: the iterates are unchanged (the column sums still complete only after all
+// rows), the DRAM traffic per iteration drops from 2 n^2 to n^2 elements.
+//
+// Layout of the work.  A cluster of S CTAs owns a set of row tiles (tiles never cross a row-block
+// boundary and are dealt round-robin to the clusters).  CTA k of the cluster owns the column
+// segment [k W, (k+1) W) of every row, W = F * 1024.  Inside a CTA
+//   - one producer thread streams row segments into a ring of shared-memory stages with bulk
+//     async copies (cp.async.bulk, completion on an mbarrier) - no registers, deep queue;
+//   - 8 "dot" warps keep their slice of v in registers, multiply a landed segment with it and
+//     send one partial sum per warp to every CTA of the cluster through distributed shared
+//     memory with st.async, whose completion is counted on the receiving CTA's mbarrier (no
+//     fence, no round trip on the sender's side);
+//   - 8 "accumulate" warps keep the column partial sums r in registers; when all S*8 partials of
+//     a row have arrived they add them in a fixed order, form u_i = a_i / q_i and accumulate
+//     K_il * u_i from the same shared-memory stage, then hand the stage back to the producer.
+// The two groups work on different rows at the same time, so the exchange latency is hidden.
+// At the end each CTA writes its column partials; the ordinary stage-2 kernel adds them over
+// the clusters in a fixed order and applies v = b ./ r.  No atomics: results are reproducible.
+//
+// Every wait is bounded; when one runs out the kernel raises the status flag, stops, drains its
+// own copies and leaves through the final cluster barrier.
+#include "fs_internal.cuh"
+
+namespace {
+
+constexpr int kGroup = 256;                 // threads per compute group
+constexpr int kFusedThreads = 2 * kGroup + 32;
+constexpr int kWarpsPerGroup = kGroup / 32;
+constexpr int kMaxS = 4;
+constexpr int kXchgStride = 32;             // floats per exchange slot: S*8 per-warp partial sums
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it > 64) __nanosleep(40);
+    }
+    return false;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (it > 64) __nanosleep(40);
+    }
+    return false;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+// Asynchronous store of one float into (possibly another CTA's) shared memory; its completion is
+// counted as 4 transaction bytes on the mbarrier that lives in the same CTA as the destination.
+__device__ __forceinline__ void st_async_f32(uint32_t addr, float v, uint32_t bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];"
+                 ::"r"(addr), "f"(v), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ float4 lds4(uint32_t addr) {
+    float4 r;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(addr));
+    return r;
+}
+
+// F = 128-bit column groups per thread: a CTA covers W = F*1024 columns of each row.
+template <int F>
+__global__ void __launch_bounds__(kFusedThreads, 1)
+fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, int nclusters, int nstages,
+                       const FsRowTile *__restrict__ tiles, int ntiles, const float *__restrict__ v,
+                       const float *__restrict__ a, float *__restrict__ u, float *__restrict__ rowdiff,
+                       float *__restrict__ partials, FsDeviceStatus *status) {
+    extern __shared__ uint8_t smem_raw[];
+    constexpr int W = F * 1024;
+    const uint32_t stage_bytes = W * 4;
+    const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
+    const uint32_t xchg = base + (uint32_t)nstages * stage_bytes;           // [2*nstages][kXchgStride] floats
+    const uint32_t bars = xchg + (uint32_t)(2 * nstages) * kXchgStride * 4; // full[ns], empty[ns], qbar[2 ns]
+    const uint32_t rank = cluster_ctarank();
+    const int cluster = blockIdx.x / S;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int col0 = (int)rank * W;
+    const int seg = max(0, min(W, n - col0)); // columns of this CTA's segment (multiple of 4)
+    const int seg4 = seg >> 2;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < nstages; ++s) {
+            mbar_init(bars + 8 * s, 1);
+            mbar_init(bars + 8 * (nstages + s), kWarpsPerGroup);
+        }
+        for (int s = 0; s < 2 * nstages; ++s) mbar_init(bars + 8 * (2 * nstages + s), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    cluster_sync_all(); // every CTA's barriers exist before anyone arrives on them remotely
+
+    bool ok = true;
+    if (warp == 2 * kWarpsPerGroup) {
+        // ---------------- producer ----------------
+        if (lane == 0) {
+            int k = 0;
+            for (int t = cluster; t < ntiles && ok; t += nclusters) {
+                const FsRowTile tile = tiles[t];
+                for (int row = tile.begin; row < tile.end; ++row, ++k) {
+                    const int s = k % nstages;
+                    const uint32_t ph = (uint32_t)(k / nstages) & 1u;
+                    if (!mbar_wait(bars + 8 * (nstages + s), ph ^ 1u)) { ok = false; break; }
+                    const uint32_t full = bars + 8 * s;
+                    // this row's exchange slot: S*8 floats will arrive as asynchronous stores
+                    mbar_expect_tx(bars + 8 * (2 * nstages + k % (2 * nstages)), (uint32_t)(S * kWarpsPerGroup) * 4u);
+                    if (seg > 0) {
+                        mbar_expect_tx(full, (uint32_t)seg * 4u);
+                        const float *src = K + (int64_t)row * ld + col0;
+                        const uint32_t dst = base + (uint32_t)s * stage_bytes;
+                        for (int off = 0; off < seg; off += 4096) { // 16 KB pieces
+                            const int cnt = min(4096, seg - off);
+                            bulk_load(dst + (uint32_t)off * 4u, src + off, (uint32_t)cnt * 4u, full);
+                        }
+                    } else {
+                        mbar_arrive(full);
+                    }
+                }
+            }
+            if (!ok) {
+                // drain: copies already issued must land before this CTA's shared memory goes away
+                for (int j = max(0, k - nstages); j < k; ++j)
+                    (void)mbar_wait(bars + 8 * (j % nstages), (uint32_t)(j / nstages) & 1u);
+            }
+        }
+    } else if (warp < kWarpsPerGroup) {
+        // ---------------- dot group ----------------
+        const int t = threadIdx.x; // 0..255
+        float4 v4[F];
+#pragma unroll
+        for (int j = 0; j < F; ++j) {
+            const int c4 = j * kGroup + t;
+            v4[j] = c4 < seg4 ? __ldg(reinterpret_cast<const float4 *>(v + col0) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        int k = 0;
+        for (int tl = cluster; tl < ntiles && ok; tl += nclusters) {
+            const FsRowTile tile = tiles[tl];
+            for (int row = tile.begin; row < tile.end; ++row, ++k) {
+                const int s = k % nstages;
+                const int slot = k % (2 * nstages);
+                if (!mbar_wait(bars + 8 * s, (uint32_t)(k / nstages) & 1u)) { ok = false; break; }
+                const uint32_t st = base + (uint32_t)s * stage_bytes + (uint32_t)t * 16u;
+                float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+                for (int j = 0; j < F; ++j) {
+                    if (j * kGroup + t < seg4) {
+                        const float4 kv = lds4(st + (uint32_t)j * (kGroup * 16u));
+                        acc0 = fmaf(kv.x, v4[j].x, acc0);
+                        acc1 = fmaf(kv.y, v4[j].y, acc1);
+                        acc0 = fmaf(kv.z, v4[j].z, acc0);
+                        acc1 = fmaf(kv.w, v4[j].w, acc1);
+                    }
+                }
+                float acc = acc0 + acc1;
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+                if (lane < S) { // lane r delivers this warp's partial to CTA r of the cluster
+                    const uint32_t cell = xchg + (uint32_t)(slot * kXchgStride + (int)rank * kWarpsPerGroup + warp) * 4u;
+                    const uint32_t qb = bars + 8 * (2 * nstages + slot);
+                    st_async_f32(map_to_cta(cell, (uint32_t)lane), acc, map_to_cta(qb, (uint32_t)lane));
+                }
+            }
+        }
+    } else {
+        // ---------------- accumulate group ----------------
+        const int t = threadIdx.x - kGroup; // 0..255
+        const int gw = warp - kWarpsPerGroup;
+        float4 r4[F];
+#pragma unroll
+        for (int j = 0; j < F; ++j) r4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        int k = 0;
+        for (int tl = cluster; tl < ntiles && ok; tl += nclusters) {
+            const FsRowTile tile = tiles[tl];
+            // the tile's marginal entries and old scalings (at most 32 rows): one load per tile, lane i keeps row i
+            float a_lane = 1.f, uo_lane = 0.f;
+            if (tile.begin + lane < tile.end) {
+                a_lane = a[tile.begin + lane];
+                uo_lane = u[tile.begin + lane];
+            }
+            for (int row = tile.begin; row < tile.end; ++row, ++k) {
+                const int s = k % nstages;
+                const int slot = k % (2 * nstages);
+                if (!mbar_wait(bars + 8 * s, (uint32_t)(k / nstages) & 1u)) { ok = false; break; }
+                if (!mbar_wait_cluster(bars + 8 * (2 * nstages + slot), (uint32_t)(k / (2 * nstages)) & 1u)) { ok = false; break; }
+                const uint32_t my = xchg + (uint32_t)(slot * kXchgStride) * 4u;
+                float q = 0.f;
+#pragma unroll
+                for (int i = 0; i < kMaxS * kWarpsPerGroup / 4; ++i) {
+                    if (i < S * kWarpsPerGroup / 4) {
+                        const float4 c = lds4(my + (uint32_t)i * 16u);
+                        q += (c.x + c.y) + (c.z + c.w);
+                    }
+                }
+                const float ai = __shfl_sync(0xffffffffu, a_lane, row - tile.begin);
+                const float uo = __shfl_sync(0xffffffffu, uo_lane, row - tile.begin);
+                const float ui = ai / q;
+                if (t == 0 && rank == 0) {
+                    rowdiff[row] = fmaf(uo, q, -ai);
+                    u[row] = ui;
+                    if (!(ui > 0.f) || isinf(ui)) status->nonfinite = 1;
+                }
+                const uint32_t st = base + (uint32_t)s * stage_bytes + (uint32_t)t * 16u;
+#pragma unroll
+                for (int j = 0; j < F; ++j) {
+                    if (j * kGroup + t < seg4) {
+                        const float4 kv = lds4(st + (uint32_t)j * (kGroup * 16u));
+                        r4[j].x = fmaf(kv.x, ui, r4[j].x);
+                        r4[j].y = fmaf(kv.y, ui, r4[j].y);
+                        r4[j].z = fmaf(kv.z, ui, r4[j].z);
+                        r4[j].w = fmaf(kv.w, ui, r4[j].w);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bars + 8 * (nstages + s)); // stage back to the producer
+            }
+        }
+        (void)gw;
+        if (ok) {
+            float4 *out = reinterpret_cast<float4 *>(partials + (int64_t)cluster * n + col0);
+#pragma unroll
+            for (int j = 0; j < F; ++j) {
+                const int c4 = j * kGroup + t;
+                if (c4 < seg4) out[c4] = r4[j];
+            }
+        }
+    }
+    if (!ok) status->timeout = 1;
+    __syncwarp();
+    cluster_sync_all(); // nobody leaves while a peer may still write into its shared memory
+}
+
+size_t fused_smem_bytes(int F, int nstages) {
+    return (size_t)nstages * F * 4096 + (size_t)2 * nstages * kXchgStride * 4 + (size_t)8 * 4 * nstages + 256;
+}
+
+template <int F>
+cudaError_t launch_fused(int S, int nclusters, int nstages, cudaStream_t st, const float *K, int64_t ld, int n,
+                         const FsRowTile *tiles, int ntiles, const float *v, const float *a, float *u, float *rowdiff,
+                         float *partials, FsDeviceStatus *status) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(nclusters * S));
+    cfg.blockDim = dim3(kFusedThreads);
+    cfg.dynamicSmemBytes = fused_smem_bytes(F, nstages);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fused_iteration_kernel<F>, K, ld, n, S, nclusters, nstages, tiles, ntiles, v, a, u,
+                              rowdiff, partials, status);
+}
+
+template <int F>
+int query_clusters(int S, int nstages) {
+    const size_t smem = fused_smem_bytes(F, nstages);
+    if (cudaFuncSetAttribute(fused_iteration_kernel<F>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(148 * S));
+    cfg.blockDim = dim3(kFusedThreads);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int nc = 0;
+    if (cudaOccupancyMaxActiveClusters(&nc, fused_iteration_kernel<F>, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    return nc;
+}
+
+} // namespace
+
+// Chooses the fused configuration for an n x n problem; plan.enabled = false when it does not apply.
+FsFusedPlan fsk_fused_plan(int64_t n, bool vec) {
+    FsFusedPlan p{};
+    if (!vec || (n & 3) != 0 || n < 2048) return p;
+    int S = 2;
+    int64_t f = (n + 2047) / 2048; // 128-bit groups per thread with S = 2
+    if (f > 16) {
+        S = 4;
+        f = (n + 4095) / 4096;
+    }
+    if (f > 16) return p;
+    const int F = f <= 2 ? 2 : f <= 4 ? 4 : f <= 8 ? 8 : 16;
+    int ns = (int)(200 * 1024 / (F * 4096));
+    if (ns > 8) ns = 8;
+    if (ns < 2) return p;
+    int nc = 0;
+    switch (F) {
+    case 2: nc = query_clusters<2>(S, ns); break;
+    case 4: nc = query_clusters<4>(S, ns); break;
+    case 8: nc = query_clusters<8>(S, ns); break;
+    default: nc = query_clusters<16>(S, ns); break;
+    }
+    if (nc < 1) return p;
+    p.enabled = true, p.S = S, p.F = F, p.nstages = ns, p.nclusters = nc, p.tile_rows = 32;
+    return p;
+}
+
+// One fused iteration minus the final divide: writes u, rowdiff and the per-cluster column partials
+// [nclusters][n]; the caller runs the stage-2 kernel over them.
+cudaError_t fsk_fused_iteration(const FsFusedPlan &p, const float *K, int64_t ld, int64_t n, const FsRowTile *tiles,
+                                int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials,
+                                FsDeviceStatus *status, cudaStream_t st) {
+    switch (p.F) {
+    case 2: return launch_fused<2>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, status);
+    case 4: return launch_fused<4>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, status);
+    case 8: return launch_fused<8>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, status);
+    default: return launch_fused<16>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, status);
+    }
+}

@@ -526,5 +526,11 @@ void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n
         (int)n, n_pad, ntiles, s2, eps, partials, b, logb, g, ys, coldiff, update, status);
 }
 
+void fsk_col_finish(int64_t n, int64_t n_pad, int ntiles, const float *partials, const float *b, float *v,
+                    float *coldiff, int update, FsDeviceStatus *status, cudaStream_t st) {
+    col_finish_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>((int)n, n_pad, ntiles, partials, b, v,
+                                                                                   coldiff, update, status);
+}
+
 int fsk_pass_launches_row() { return 1; }
 int fsk_pass_launches_col() { return 2; }

@@ -150,6 +150,49 @@ def test_config5_scaled_down_ten_iterations(n, nb):
     batched_sample(w, U, V, 10, sorted({0, 1, nb // 2, nb - 1}))
 
 
+@pytest.mark.parametrize("n,offsets", [(2048, None), (4100, None), (8192, [0, 5, 37, 4096, 4100, 8192]),
+                                       (8200, None), (16384, None)])
+def test_fused_single_read_iteration(n, offsets):
+    """fs_iterate with the single-read fused kernel against the two-pass path and the oracle:
+    column segments that end inside a CTA (n = 4100, 8200), row tiles cut by block boundaries,
+    and a run long enough for the shared-memory ring and the exchange slots to wrap many times."""
+    w = workloads.make(4, n=n)
+    off = w.offsets if offsets is None else np.asarray(offsets, dtype=np.int64)
+    res = {}
+    for mode in (0, 2):
+        with GpuSolver(w.K, KK, w.eps, w.a, w.b, off, SC) as g:
+            fs.fs_set_option(g.h, fs.FS_OPT_FUSED, mode)
+            before = fs.fs_launch_count(g.h)
+            g.iterate(10)
+            assert fs.fs_launch_count(g.h) - before == (30 if mode == 0 else 20)
+            res[mode] = g.scalings()
+            row, col = g.errors(1)
+            res[mode] += (row[0], col[0])
+    u, v = oracle.sinkhorn_scaling(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, 10)
+    for mode in (0, 2):
+        assert rel_err(res[mode][0], u) <= TOL_UV and rel_err(res[mode][1], v) <= TOL_UV
+    assert rel_err(res[2][0], res[0][0]) < 1e-5 and rel_err(res[2][1], res[0][1]) < 1e-5
+    assert abs(res[2][2] - res[0][2]) < 1e-6
+
+
+def test_fused_is_reproducible_and_traces():
+    w = workloads.make(4, n=4096)
+    runs = []
+    for _ in range(2):
+        with GpuSolver(w.K, KK, w.eps, w.a, w.b, w.offsets, SC) as g:
+            fs.fs_set_option(g.h, fs.FS_OPT_FUSED, 2)
+            fs.fs_set_error_trace(g.h, 4)
+            g.iterate(9)
+            runs.append(g.scalings() + fs.fs_error_trace(g.h, stream=g.stream))
+    assert all(np.array_equal(x, y) for x, y in zip(runs[0], runs[1]))
+    l1 = runs[0][2]
+    assert len(l1) == 2
+    for k, t in enumerate((4, 8)):
+        u, v = oracle.sinkhorn_scaling(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, t)
+        e = oracle.marginal_errors(w.K, oracle.KIND_KERNEL, w.eps, SC, u, v, w.a, w.b)
+        assert l1[k] == pytest.approx(e["row_l1"], rel=1e-3, abs=1e-6)
+
+
 @pytest.mark.parametrize("n,nb", [(512, 32), (1000, 40), (2048, 128)])
 def test_batched_engines_agree(n, nb):
     """The fp32 FMA engine and the tensor-core engine (bf16 hi/lo split, fp32 accumulation) run the
