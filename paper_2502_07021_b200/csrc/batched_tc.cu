@@ -19,7 +19,12 @@
 // issues TMA tile loads (128 x 64 bf16, 128-byte swizzle) into a 3-stage shared-memory ring,
 // warp 1 issues the tcgen05.mma instructions (M = N = 128, K = 16, three per k-step) into a
 // 128-column TMEM accumulator and releases ring slots with tcgen05.commit, warps 2-5 read the
-// accumulator back with tcgen05.ld and store the fp32 partial tile.  A second small kernel adds
+// accumulator back with tcgen05.ld and store the fp32 partial tile.  The tensor core adds into its
+// fp32 accumulator without round-to-nearest, a bias that grows with the number of accumulated
+// MMAs (a uniform ~2e-5 relative deficit was measured after the 6144 MMAs of a full n = 8192
+// contraction in one accumulator); so the contraction is cut into chunks of 8 k-blocks (96 MMAs)
+// that alternate between two TMEM accumulators, and the epilogue warps add each finished chunk
+// into fp32 registers with round-to-nearest while the next chunk is being computed.  A second small kernel adds
 // the partial tiles of the splits in a fixed order and applies the divide, the marginal residual
 // and the bf16 re-split of the new scalings.  Every mbarrier wait is bounded: on expiry the
 // kernel raises a status flag, stops issuing work, drains what it had in flight and exits.
@@ -34,8 +39,10 @@ constexpr int BM = 128, BN = 128, BK = 64, STAGES = 3;
 constexpr int TILE_BYTES = BM * BK * 2;     // one operand tile: 128 rows of 128 bytes
 constexpr int STAGE_BYTES = 4 * TILE_BYTES; // A_hi, A_lo, B_hi, B_lo
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 128;
+constexpr int NUM_BARS = 2 * STAGES + 4;    // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]
 constexpr int kTcThreads = 192;
-constexpr int TMEM_COLS = 128;
+constexpr int TMEM_COLS = 256;              // two 128-column fp32 accumulators
+constexpr int CHUNK_KB = 8;                 // k-blocks accumulated in TMEM before the chunk is drained
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 struct TcState {
@@ -128,8 +135,9 @@ batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_const
                   float *__restrict__ partials, int kblocks, int ksplit, FsDeviceStatus *status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bars = base + STAGES * STAGE_BYTES; // full[STAGES], empty[STAGES], accum
-    const uint32_t tmem_slot = bars + 8 * (2 * STAGES + 1);
+    const uint32_t bars = base + STAGES * STAGE_BYTES;
+    const uint32_t acc_full = bars + 8 * (2 * STAGES), acc_empty = bars + 8 * (2 * STAGES + 2);
+    const uint32_t tmem_slot = bars + 8 * NUM_BARS;
     uint32_t *tmem_slot_ptr = reinterpret_cast<uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int mtile = blockIdx.x, ks = blockIdx.y, ntile = blockIdx.z;
@@ -141,7 +149,10 @@ batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_const
             mbar_init(bars + 8 * s, 1);
             mbar_init(bars + 8 * (STAGES + s), 1);
         }
-        mbar_init(bars + 8 * 2 * STAGES, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(acc_full + 8 * b, 1);
+            mbar_init(acc_empty + 8 * b, 4); // one arrival per epilogue warp
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -176,50 +187,64 @@ batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_const
             for (; it < nkb; ++it) {
                 const int s = it % STAGES;
                 const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                const int chunk = it / CHUNK_KB, buf = chunk & 1;
+                if (it % CHUNK_KB == 0) { // this accumulator must have been drained (first use: passes at once)
+                    if (!mbar_wait(acc_empty + 8 * buf, ((uint32_t)(chunk >> 1) & 1u) ^ 1u)) { ok = false; break; }
+                    tc_fence_after();
+                }
                 if (!mbar_wait(bars + 8 * s, ph)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t st = base + s * STAGE_BYTES;
+                const uint32_t acc = tmem + (uint32_t)(buf * BN);
                 const uint64_t a_hi = make_desc(st), a_lo = make_desc(st + TILE_BYTES);
                 const uint64_t b_hi = make_desc(st + 2 * TILE_BYTES), b_lo = make_desc(st + 3 * TILE_BYTES);
 #pragma unroll
                 for (int kk = 0; kk < BK / 16; ++kk) {
                     const uint64_t adv = (uint64_t)(kk * 32 >> 4); // 16 bf16 = 32 bytes along K
-                    tc_mma_bf16(tmem, a_lo + adv, b_hi + adv, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
-                    tc_mma_bf16(tmem, a_hi + adv, b_lo + adv, kIdesc, 1u);
-                    tc_mma_bf16(tmem, a_hi + adv, b_hi + adv, kIdesc, 1u);
+                    tc_mma_bf16(acc, a_lo + adv, b_hi + adv, kIdesc, (it % CHUNK_KB != 0 || kk > 0) ? 1u : 0u);
+                    tc_mma_bf16(acc, a_hi + adv, b_lo + adv, kIdesc, 1u);
+                    tc_mma_bf16(acc, a_hi + adv, b_hi + adv, kIdesc, 1u);
                 }
                 tc_commit(bars + 8 * (STAGES + s)); // frees the ring slot when these MMAs have read it
+                if (it % CHUNK_KB == CHUNK_KB - 1 || it == nkb - 1) tc_commit(acc_full + 8 * buf); // chunk complete
             }
-            if (ok) {
-                tc_commit(bars + 8 * 2 * STAGES);   // accumulator complete
-            } else {
+            if (!ok) {
                 // drain: loads already issued into later slots must land before the CTA exits
                 for (int j = it; j < nkb && j < it + STAGES; ++j)
                     (void)mbar_wait(bars + 8 * (j % STAGES), (uint32_t)(j / STAGES) & 1u);
             }
         }
     } else {
-        // epilogue warps 2..5: TMEM lane quarter = warp % 4
+        // epilogue warps 2..5: TMEM lane quarter = warp % 4; running sums of the chunks in registers
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
-        if (nkb > 0) ok = mbar_wait(bars + 8 * 2 * STAGES, 0);
-        ok = __all_sync(0xffffffffu, ok);
-        tc_fence_after();
-        const int unit = ((ntile * gridDim.x + mtile) * ksplit + ks);
-        float *out = partials + (size_t)unit * (BM * BN) + row;
-        if (ok) {
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+        float sum[BN];
+#pragma unroll
+        for (int j = 0; j < BN; ++j) sum[j] = 0.f;
+        const int nchunks = (nkb + CHUNK_KB - 1) / CHUNK_KB;
+        for (int c = 0; c < nchunks && ok; ++c) {
+            const int buf = c & 1;
+            ok = mbar_wait(acc_full + 8 * buf, (uint32_t)(c >> 1) & 1u);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+#pragma unroll
+            for (int cc = 0; cc < BN / 32; ++cc) {
                 float v[32];
-                if (nkb > 0) {
-                    tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), v);
-                } else {
+                tmem_ld32(taddr + (uint32_t)(cc * 32), v);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = 0.f;
-                }
-#pragma unroll
-                for (int j = 0; j < 32; ++j) out[(size_t)(c * 32 + j) * BM] = v[j];
+                for (int j = 0; j < 32; ++j) sum[cc * 32 + j] += v[j];
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_empty + 8 * buf) : "memory");
+        }
+        if (ok) {
+            const int unit = ((ntile * gridDim.x + mtile) * ksplit + ks);
+            float *out = partials + (size_t)unit * (BM * BN) + row;
+#pragma unroll
+            for (int j = 0; j < BN; ++j) out[(size_t)j * BM] = sum[j];
         }
     }
     if (!ok) status->timeout = 1;
@@ -236,29 +261,38 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bflo
     lo = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
+// blockIdx.x = (ntile * mtiles + mtile) * 16 + slice: 1024 outputs per CTA, 4 consecutive rows per thread.
 __global__ void __launch_bounds__(256)
-batched_tc_finish_kernel(const float *__restrict__ partials, int ksplit, int n, int nbatch, int64_t ldb,
+batched_tc_finish_kernel(const float *__restrict__ partials, int ksplit, int n, int nbatch, int64_t ldb, int mtiles,
                          const float *__restrict__ marg, float *__restrict__ out, float *__restrict__ diff,
                          __nv_bfloat16 *__restrict__ op_hi, __nv_bfloat16 *__restrict__ op_lo, int update,
                          FsDeviceStatus *status) {
-    const int mtile = blockIdx.x, ntile = blockIdx.y;
-    const float *base = partials + (size_t)((ntile * gridDim.x + mtile) * ksplit) * (BM * BN);
-    for (int e = threadIdx.x; e < BM * BN; e += 256) {
-        const int p = e / BM, i = e % BM;
-        const int gi = mtile * BM + i, gp = ntile * BN + p;
-        if (gi >= n || gp >= nbatch) continue;
-        float q = 0.f;
-        for (int k = 0; k < ksplit; ++k) q += base[(size_t)k * (BM * BN) + e];
-        const int64_t idx = (int64_t)gp * n + gi;
+    const int tile = blockIdx.x >> 4, slice = blockIdx.x & 15;
+    const int mtile = tile % mtiles, ntile = tile / mtiles;
+    const int e = (slice * 256 + threadIdx.x) * 4; // element index inside the 128 x 128 tile, [p][i] order
+    const int p = e / BM, i = e % BM;
+    const int gi = mtile * BM + i, gp = ntile * BN + p;
+    if (gi >= n || gp >= nbatch) return;
+    const float *base = partials + (size_t)tile * ksplit * (BM * BN) + e;
+    float4 q = *reinterpret_cast<const float4 *>(base);
+    for (int k = 1; k < ksplit; ++k) {
+        const float4 t = *reinterpret_cast<const float4 *>(base + (size_t)k * (BM * BN));
+        q.x += t.x, q.y += t.y, q.z += t.z, q.w += t.w;
+    }
+    const float qs[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if (gi + j >= n) break;
+        const int64_t idx = (int64_t)gp * n + gi + j;
         const float mg = marg[idx], old = out[idx];
-        diff[idx] = fmaf(old, q, -mg);
+        diff[idx] = fmaf(old, qs[j], -mg);
         if (update) {
-            const float nv = mg / q;
+            const float nv = mg / qs[j];
             out[idx] = nv;
             __nv_bfloat16 hi, lo;
             split_bf16(nv, hi, lo);
-            op_hi[(int64_t)gp * ldb + gi] = hi;
-            op_lo[(int64_t)gp * ldb + gi] = lo;
+            op_hi[(int64_t)gp * ldb + gi + j] = hi;
+            op_lo[(int64_t)gp * ldb + gi + j] = lo;
             if (!(nv > 0.f) || isinf(nv)) status->nonfinite = 1;
         }
     }
@@ -410,8 +444,7 @@ void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float 
     else
         batched_tc_kernel<<<grid, kTcThreads, SMEM_BYTES, st>>>(t->tmKt_hi, t->tmKt_lo, t->tmU_hi, t->tmU_lo, t->partials,
                                                               t->kblocks, t->ksplit, status);
-    dim3 fgrid((unsigned)t->mtiles, (unsigned)t->ntiles);
-    batched_tc_finish_kernel<<<fgrid, 256, 0, st>>>(t->partials, t->ksplit, (int)t->n, t->nbatch, t->ldb, marg, out, diff,
+    batched_tc_finish_kernel<<<(unsigned)(t->mtiles * t->ntiles * 16), 256, 0, st>>>(t->partials, t->ksplit, (int)t->n, t->nbatch, t->ldb, t->mtiles, marg, out, diff,
                                                    transposed ? t->V_hi : t->U_hi, transposed ? t->V_lo : t->U_lo, update,
                                                    status);
 }
