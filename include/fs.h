@@ -68,7 +68,8 @@ enum {
     FS_OPT_BATCH_ENGINE = 2, /* batched passes: 0 = auto (tensor cores when nbatch >= 32 and n >= 512),
                                 1 = fp32 FMA kernels, 2 = tensor-core kernels (bf16 hi/lo split, fp32 accumulate) */
     /* Tuning knobs for the single-problem passes (defaults are chosen from n at fs_create): */
-    FS_OPT_ROW_SHAPE = 3,   /* value = L*1000 + R: L threads sweep R rows at once; (32,1), (256,4), (256,8) */
+    FS_OPT_ROW_SHAPE = 3,   /* value = L*1000 + R: L threads sweep R rows at once; (32,1), (32,2), (64,1),
+                               (64,2), (128,2), (256,4), (256,8) */
     FS_OPT_COL_SHAPE = 4,   /* value = TX*1000 + H: TX in {32,64,256} threads across a column strip of 4*TX
                                columns, row tiles of at most H <= 256 rows */
     FS_OPT_FUSED = 5        /* single-read fused iteration in fs_iterate (scaling domain, one problem, 16-byte

@@ -33,11 +33,12 @@ constexpr int64_t kFusedAutoMinN = 12288;
 constexpr int kTcMinBatch = 32;
 constexpr int kTcMinN = 512;
 
-FsPassPlan choose_plan(int64_t n, bool vec) {
+FsPassPlan choose_plan(int64_t n, bool vec, int domain) {
     FsPassPlan p{};
     p.vec = vec;
     if (n >= 8192) {
         p.row_L = 32, p.row_R = 1, p.col_TX = 64, p.col_TY = 4, p.col_tile_rows = 256;
+        if (domain == FS_DOMAIN_LOG) p.row_L = 128, p.row_R = 2; // measured: 169 us against 176 us at n = 16384
     } else if (n >= 2048) {
         p.row_L = 256, p.row_R = 4, p.col_TX = 64, p.col_TY = 4, p.col_tile_rows = 64;
     } else {
@@ -338,7 +339,7 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
         s->mat = M_dev, s->mat_ld = ld;
     }
     const bool vec = (reinterpret_cast<uintptr_t>(s->mat) & 15) == 0 && (s->mat_ld & 3) == 0;
-    s->plan = choose_plan(n, vec);
+    s->plan = choose_plan(n, vec, domain);
     int rc = upload_tiles(s);
     if (rc != FS_OK) return rc;
     if (domain == FS_DOMAIN_SCALING && nbatch == 1) {
@@ -399,7 +400,9 @@ int fs_set_option(fs_solver *s, int option, int64_t value) {
         return FS_OK;
     case FS_OPT_ROW_SHAPE: {
         const int L = (int)(value / 1000), R = (int)(value % 1000);
-        if (!((L == 32 && R == 1) || (L == 256 && (R == 4 || R == 8)))) return FS_ERR_BAD_N;
+        if (!((L == 32 && (R == 1 || R == 2)) || (L == 64 && (R == 1 || R == 2)) || (L == 128 && R == 2) ||
+              (L == 256 && (R == 4 || R == 8))))
+            return FS_ERR_BAD_N;
         s->plan.row_L = L, s->plan.row_R = R;
         destroy_graphs(s);
         return FS_OK;

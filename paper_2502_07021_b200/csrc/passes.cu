@@ -159,7 +159,7 @@ log_row_pass_kernel(const float *__restrict__ C, int64_t ld, int n, float s2, do
                     FsDeviceStatus *status) {
     constexpr int G = kThreads / L;
     constexpr int W = L / 32;
-    constexpr int U = (R >= 4) ? 2 : 4;
+    constexpr int U = (R >= 4) ? 2 : (R >= 2 ? 4 : 8); // column chunks in flight per thread
     __shared__ float red_m[kThreads / 32][R], red_s[kThreads / 32][R];
 
     const int grp = threadIdx.x / L, lane = threadIdx.x % L;
@@ -463,20 +463,23 @@ log_col_finish_kernel(int n, int64_t n_pad, int ntiles, float s2, double eps, co
 // ------------------------------------------------------------------------------------------
 // Host-side dispatch.
 
+#define FS_ROW_CASE(KERNEL, L_, R_, ...)                                                          \
+    if (p.row_L == L_ && p.row_R == R_) {                                                         \
+        if (p.vec) KERNEL<L_, R_, true><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                  \
+        else KERNEL<L_, R_, false><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                       \
+    } else
+
 #define FS_ROW_DISPATCH(KERNEL, ...)                                                              \
     do {                                                                                          \
         const int G_ = kThreads / p.row_L;                                                        \
         const unsigned grid_ = (unsigned)((n + (int64_t)G_ * p.row_R - 1) / ((int64_t)G_ * p.row_R)); \
-        if (p.row_L == 32 && p.row_R == 1) {                                                      \
-            if (p.vec) KERNEL<32, 1, true><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);               \
-            else KERNEL<32, 1, false><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                    \
-        } else if (p.row_L == 256 && p.row_R == 4) {                                              \
-            if (p.vec) KERNEL<256, 4, true><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);              \
-            else KERNEL<256, 4, false><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                   \
-        } else {                                                                                  \
-            if (p.vec) KERNEL<256, 8, true><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);              \
-            else KERNEL<256, 8, false><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                   \
-        }                                                                                         \
+        FS_ROW_CASE(KERNEL, 32, 1, __VA_ARGS__)                                                   \
+        FS_ROW_CASE(KERNEL, 32, 2, __VA_ARGS__)                                                   \
+        FS_ROW_CASE(KERNEL, 64, 1, __VA_ARGS__)                                                   \
+        FS_ROW_CASE(KERNEL, 64, 2, __VA_ARGS__)                                                   \
+        FS_ROW_CASE(KERNEL, 128, 2, __VA_ARGS__)                                                  \
+        FS_ROW_CASE(KERNEL, 256, 4, __VA_ARGS__)                                                  \
+        FS_ROW_CASE(KERNEL, 256, 8, __VA_ARGS__) {}                                               \
     } while (0)
 
 #define FS_COL_DISPATCH(KERNEL, ...)                                                              \
