@@ -72,8 +72,9 @@ enum {
                                (64,2), (128,2), (256,4), (256,8) */
     FS_OPT_COL_SHAPE = 4,   /* value = TX*1000 + H: TX in {32,64,256} threads across a column strip of 4*TX
                                columns, row tiles of at most H <= 256 rows */
-    FS_OPT_FUSED = 5        /* single-read fused iteration in fs_iterate (scaling domain, one problem, 16-byte
-                               aligned matrix, n a multiple of 4): 0 = never, 1 = automatic (default: n >= 12288),
+    FS_OPT_FUSED = 5        /* single-read fused iteration in fs_iterate (scaling or log domain, one problem, 16-byte
+                               aligned matrix, n a multiple of 4): 0 = never, 1 = automatic (default: scaling domain with
+                               n >= 12288; the log-domain variant is slower than the two passes and is opt-in),
                                2 = whenever it applies (FS_ERR_UNSUPPORTED if it does not) */
 };
 

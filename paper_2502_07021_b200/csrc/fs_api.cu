@@ -151,17 +151,29 @@ void enqueue_col(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
 // The single-read fused iteration replaces row pass + column stage 1 when it applies.
 bool use_fused(const fs_solver *s) {
     if (!s->fused.enabled || s->fused_mode == 0) return false;
-    return s->fused_mode == 2 || s->n >= kFusedAutoMinN;
+    if (s->fused_mode == 2) return true;
+    // automatic: only where it is measured faster.  The log-domain fused kernel is bound by instruction
+    // issue and the ex2 unit rather than by HBM (440 us against 327 us for the two passes at n = 16384),
+    // so it is opt-in.
+    return s->domain == FS_DOMAIN_SCALING && s->n >= kFusedAutoMinN;
 }
 
 void enqueue_fused_rows(fs_solver *s, cudaStream_t st, int64_t &launches) {
-    fsk_fused_iteration(s->fused, s->mat, s->mat_ld, s->n, s->fused_tiles_dev, s->fused_ntiles, s->y, s->a, s->x,
-                        s->rowdiff, s->fused_partials, s->status, st);
+    if (s->domain == FS_DOMAIN_LOG)
+        fsk_fused_log_iteration(s->fused, s->mat, s->mat_ld, s->n, s->eps, s->fused_tiles_dev, s->fused_ntiles, s->ys, s->a,
+                                s->loga, s->x, s->xs, s->rowdiff, s->fused_partials, s->status, st);
+    else
+        fsk_fused_iteration(s->fused, s->mat, s->mat_ld, s->n, s->fused_tiles_dev, s->fused_ntiles, s->y, s->a, s->x,
+                            s->rowdiff, s->fused_partials, s->status, st);
     launches += 1;
 }
 
 void enqueue_fused_finish(fs_solver *s, cudaStream_t st, int64_t &launches) {
-    fsk_col_finish(s->n, s->n, s->fused.nclusters, s->fused_partials, s->b, s->y, s->coldiff, 1, s->status, st);
+    if (s->domain == FS_DOMAIN_LOG)
+        fsk_log_col_finish(s->n, s->n, s->fused.nclusters, s->eps, s->fused_partials, s->b, s->logb, s->y, s->ys,
+                           s->coldiff, 1, s->status, st);
+    else
+        fsk_col_finish(s->n, s->n, s->fused.nclusters, s->fused_partials, s->b, s->y, s->coldiff, 1, s->status, st);
     launches += 1;
 }
 
@@ -342,15 +354,17 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
     s->plan = choose_plan(n, vec, domain);
     int rc = upload_tiles(s);
     if (rc != FS_OK) return rc;
-    if (domain == FS_DOMAIN_SCALING && nbatch == 1) {
-        s->fused = fsk_fused_plan(n, vec);
+    if (nbatch == 1) {
+        s->fused = domain == FS_DOMAIN_LOG ? fsk_fused_log_plan(n, vec) : fsk_fused_plan(n, vec);
         if (s->fused.enabled) {
+            const size_t planes = domain == FS_DOMAIN_LOG ? 2 : 1;
             const std::vector<FsRowTile> ft = build_tiles(s->offsets, s->fused.tile_rows);
             s->fused_ntiles = (int)ft.size();
             FS_CU(cudaMalloc(&s->fused_tiles_dev, sizeof(FsRowTile) * ft.size()));
             FS_CU(cudaMemcpy(s->fused_tiles_dev, ft.data(), sizeof(FsRowTile) * ft.size(), cudaMemcpyHostToDevice));
-            FS_CU(cudaMalloc(&s->fused_partials, sizeof(float) * (size_t)s->fused.nclusters * (size_t)n));
-            FS_CU(cudaMemsetAsync(s->fused_partials, 0, sizeof(float) * (size_t)s->fused.nclusters * (size_t)n, st));
+            const size_t pbytes = sizeof(float) * planes * (size_t)s->fused.nclusters * (size_t)n;
+            FS_CU(cudaMalloc(&s->fused_partials, pbytes));
+            FS_CU(cudaMemsetAsync(s->fused_partials, 0, pbytes, st));
         }
     }
     // batched problems: tensor-core engine when the batch is wide enough to fill its 128-problem tiles

@@ -121,6 +121,9 @@ void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n
 // Stage 2 of the column pass alone: r_l = sum over `ntiles` partial rows of pitch n_pad, residual, divide.
 void fsk_col_finish(int64_t n, int64_t n_pad, int ntiles, const float *partials, const float *b, float *v,
                     float *coldiff, int update, FsDeviceStatus *status, cudaStream_t st);
+void fsk_log_col_finish(int64_t n, int64_t n_pad, int ntiles, double eps, const float *partials, const float *b,
+                        const float *logb, float *g, float *ys, float *coldiff, int update, FsDeviceStatus *status,
+                        cudaStream_t st);
 int fsk_pass_launches_row();
 int fsk_pass_launches_col();
 
@@ -129,6 +132,13 @@ FsFusedPlan fsk_fused_plan(int64_t n, bool vec);
 cudaError_t fsk_fused_iteration(const FsFusedPlan &p, const float *K, int64_t ld, int64_t n, const FsRowTile *tiles,
                                 int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials,
                                 FsDeviceStatus *status, cudaStream_t st);
+
+// ---- fused_log.cu ------------------------------------------------------------------------
+FsFusedPlan fsk_fused_log_plan(int64_t n, bool vec);
+cudaError_t fsk_fused_log_iteration(const FsFusedPlan &p, const float *C, int64_t ld, int64_t n, double eps,
+                                    const FsRowTile *tiles, int ntiles, const float *ys, const float *a,
+                                    const float *loga, float *f, float *xs, float *rowdiff, float *partials,
+                                    FsDeviceStatus *status, cudaStream_t st);
 
 // ---- batched.cu --------------------------------------------------------------------------
 // out[p][i] = marg[p][i] / sum_l Mat(i,l) in[p][l], Mat(i,l) = K[i][l] (transposed = 0) or K[l][i].

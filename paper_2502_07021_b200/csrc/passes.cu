@@ -535,5 +535,13 @@ void fsk_col_finish(int64_t n, int64_t n_pad, int ntiles, const float *partials,
                                                                                    coldiff, update, status);
 }
 
+void fsk_log_col_finish(int64_t n, int64_t n_pad, int ntiles, double eps, const float *partials, const float *b,
+                        const float *logb, float *g, float *ys, float *coldiff, int update, FsDeviceStatus *status,
+                        cudaStream_t st) {
+    const float s2 = (float)(1.4426950408889634 / eps);
+    log_col_finish_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>(
+        (int)n, n_pad, ntiles, s2, eps, partials, b, logb, g, ys, coldiff, update, status);
+}
+
 int fsk_pass_launches_row() { return 1; }
 int fsk_pass_launches_col() { return 2; }

@@ -175,6 +175,48 @@ def test_fused_single_read_iteration(n, offsets):
     assert abs(res[2][2] - res[0][2]) < 1e-6
 
 
+@pytest.mark.parametrize("n,offsets", [(2048, None), (4100, None), (8192, [0, 5, 37, 4096, 4100, 8192]), (8200, None)])
+def test_fused_single_read_iteration_log_domain(n, offsets):
+    """The log-domain fused kernel (row LSE, then per-column running (max, sum) pairs from the same
+    on-chip row) against the two-pass log path and the oracle."""
+    w = workloads.make(3, n=n)
+    off = w.offsets if offsets is None else np.asarray(offsets, dtype=np.int64)
+    res = {}
+    for mode in (0, 2):
+        with GpuSolver(w.C, KC, w.eps, w.a, w.b, off, LG) as g:
+            fs.fs_set_option(g.h, fs.FS_OPT_FUSED, mode)
+            before = fs.fs_launch_count(g.h)
+            g.iterate(10)
+            assert fs.fs_launch_count(g.h) - before == (30 if mode == 0 else 20)
+            res[mode] = g.scalings()
+            row, col = g.errors(1)
+            res[mode] += (row[0], col[0])
+    f, gg = oracle.sinkhorn_log(w.C, w.eps, w.a, w.b, 10)
+    for mode in (0, 2):
+        assert np.max(np.abs(res[mode][0] - f)) / w.eps <= TOL_UV
+        assert np.max(np.abs(res[mode][1] - gg)) / w.eps <= TOL_UV
+    assert np.max(np.abs(res[2][0] - res[0][0])) / w.eps < 3e-5
+    assert abs(res[2][2] - res[0][2]) < 2e-5 * max(1.0, res[0][2])
+
+
+def test_fused_log_is_reproducible_and_traces():
+    w = workloads.make(3, n=2048)
+    runs = []
+    for _ in range(2):
+        with GpuSolver(w.C, KC, w.eps, w.a, w.b, w.offsets, LG) as g:
+            fs.fs_set_option(g.h, fs.FS_OPT_FUSED, 2)
+            fs.fs_set_error_trace(g.h, 4)
+            g.iterate(9)
+            runs.append(g.scalings() + fs.fs_error_trace(g.h, stream=g.stream))
+    assert all(np.array_equal(x, y) for x, y in zip(runs[0], runs[1]))
+    l1 = runs[0][2]
+    assert len(l1) == 2
+    for k, t in enumerate((4, 8)):
+        f, gg = oracle.sinkhorn_log(w.C, w.eps, w.a, w.b, t)
+        e = oracle.marginal_errors(w.C, oracle.KIND_COST, w.eps, LG, f, gg, w.a, w.b)
+        assert l1[k] == pytest.approx(e["row_l1"], rel=2e-3, abs=1e-6)
+
+
 def test_fused_is_reproducible_and_traces():
     w = workloads.make(4, n=4096)
     runs = []
