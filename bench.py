@@ -14,6 +14,7 @@ the timed region starts.  Rank 0 prints ONE JSON line.  Keys beyond the basic co
   e2e           the same metric through fs_solve_host: host buffers in, host buffers out, all
                 host<->device copies inside the timed region
   clocks        SM clock and throttle reasons sampled with nvidia-smi during the timed region
+  other_configs it/s of configurations 1, 2, 3 and 5 from short runs of the same kind (N = 1 only)
 
 With --impl reference the CPU checker is what gets timed (same config, metric and unit); under a
 multi-process launch only rank 0 runs it.
@@ -192,6 +193,43 @@ def run_reference(args, w, world):
 
 # ------------------------------------------------------------------------------------------ GPU arm
 
+def time_config(fs, torch, dev, stream, w, steps=3):
+    """it/s of one configuration through fs_iterate (device-resident inputs, CUDA events)."""
+    M = torch.from_numpy(w.matrix).to(dev)
+    a = torch.from_numpy(w.a).to(dev)
+    b = torch.from_numpy(w.b).to(dev)
+    torch.cuda.synchronize()
+    h = fs.fs_create(w.n, w.c, w.offsets, M, w.n, w.kind, w.eps, a, b, w.nbatch, w.domain, stream)
+    try:
+        if w.check_every:
+            fs.fs_set_error_trace(h, w.check_every)
+
+        def step():
+            fs.fs_reset(h, stream)
+            fs.fs_iterate(h, w.iters, stream)
+
+        for _ in range(3):
+            step()
+        stream.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            step()
+        e1.record(stream)
+        stream.synchronize()
+        ms = e0.elapsed_time(e1)
+        row, col = fs.fs_marginal_error(h, 1, w.nbatch, stream)
+    finally:
+        fs.fs_destroy(h)
+    its = steps * w.iters
+    return {"workload": f"n={w.n}" + (f" N={w.nbatch}" if w.nbatch > 1 else "") + (" log" if w.domain else " scaling"),
+            "value": its / (ms * 1e-3), "unit": UNIT, "us_per_iteration": ms * 1e3 / its, "steps": steps,
+            "iterations_per_step": w.iters,
+            "effective_gbs_2n2": 2 * w.n * w.n * 4 * its / (ms * 1e-3) / 1e9,
+            "final_row_marginal_l1_max": float(row.max()), "final_col_marginal_l1_max": float(col.max())}
+
+
 def run_ours(args, w, rank, local_rank, world):
     import torch
     from paper_2502_07021_b200 import binding as fs
@@ -283,6 +321,16 @@ def run_ours(args, w, rank, local_rank, world):
             # BASELINE's accounting (every iteration streams 2 n^2 elements) applied to the timed region
             "iteration_effective_gbs_2n2": 2 * n2 * (args.steps * w.iters) / (elapsed_ms * 1e-3) / 1e9}
 
+    # the other four configurations, briefly (single GPU runs only): same step definition, fewer steps
+    others = None
+    if world == 1 and not args.headline_only and args.config == 4 and args.n is None and args.iters is None:
+        others = {}
+        for cfg in (1, 2, 3, 5):
+            try:
+                others[f"config{cfg}"] = time_config(fs, torch, dev, stream, workloads.make(cfg, want_cost=None if cfg == 3 else False))
+            except Exception as exc:  # a failure here must not lose the headline line
+                others[f"config{cfg}"] = {"error": repr(exc)}
+
     # end-to-end through the host-buffer entry point
     e2e = None
     if not args.no_e2e:
@@ -323,7 +371,7 @@ def run_ours(args, w, rank, local_rank, world):
             "warmup": max(3, args.warmup), "ms_per_step": t_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": config_dict(w, args, world), "gpu_launches": int(launches), "clocks": clocks,
-            "e2e": e2e, "roofline": roof, "cpu_baseline": base,
+            "e2e": e2e, "roofline": roof, "cpu_baseline": base, "other_configs": others,
             "final_row_marginal_l1": float(row_err[0]), "final_col_marginal_l1": float(col_err[0])}
     print(json.dumps(line), flush=True)
 
@@ -340,6 +388,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-iters", type=int, default=1, help="--impl reference: iterations per step")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--headline-only", action="store_true", help="skip the short runs of configurations 1, 2, 3, 5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture (reported as is)")
