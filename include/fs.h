@@ -146,6 +146,15 @@ int fs_reset(fs_solver *s, void *stream);
  */
 int fs_transport_cost(fs_solver *s, const float *C_dev, int64_t ldc, double *cost_out, void *stream);
 
+/*
+ * fs_set_damping -- relaxed (damped) scaling updates of Section 3.3,
+ *      u <- (1 - eta) u + eta a ./ (K v),     v <- (1 - eta) v + eta b ./ (K^T u),
+ * for every later pass of this handle.  0 < eta <= 1; eta = 1 (the default) is plain Sinkhorn and is
+ * bit-identical to never calling this.  Scaling domain only (the log-domain analogue would be the
+ * geometric damping the paper leaves to future work): FS_ERR_UNSUPPORTED there unless eta = 1.
+ */
+int fs_set_damping(fs_solver *s, double eta);
+
 /* Error trace: with check_every = m > 0, fs_iterate records err_a (1-norm and 2-norm, problem 0)
  * of the state after every m-th iteration.  The value for a state is produced by the NEXT row
  * pass, where u .* (K v) is available at no cost; when fs_iterate ends exactly on a check point one

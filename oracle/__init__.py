@@ -61,6 +61,7 @@ def _load():
                 "or_row_pass": [_i64, _f32p, _i64, _int, _dbl, _f32p, _f64p, _f64p, _f64p],
                 "or_col_pass": [_i64, _f32p, _i64, _int, _dbl, _f32p, _f64p, _f64p, _f64p],
                 "or_sinkhorn_scaling": [_i64, _f32p, _i64, _int, _dbl, _f32p, _f32p, _i64, _f64p, _f64p],
+                "or_sinkhorn_damped": [_i64, _f32p, _i64, _int, _dbl, _f32p, _f32p, _dbl, _i64, _f64p, _f64p],
                 "or_sinkhorn_protocol": [_i64, _i32, _i64p, _f32p, _i64, _int, _dbl, _f32p, _f32p, _i64,
                                          _f64p, _f64p, ctypes.POINTER(_i32)],
                 "or_sinkhorn_rowpartition": [_i64, _i32, _i64p, _f32p, _i64, _int, _dbl, _f32p, _f32p,
@@ -161,6 +162,17 @@ def sinkhorn_scaling(M, kind, eps, a, b, iters, u0=None, v0=None):
     v = _f64(np.ones(n) if v0 is None else v0, n)
     _load().or_sinkhorn_scaling(n, _p32(M), ld, kind, float(eps), _p32(a), _p32(b), int(iters),
                                 _p64(u), _p64(v))
+    return u, v
+
+
+def sinkhorn_damped(M, kind, eps, a, b, eta, iters, u0=None, v0=None):
+    """Relaxed iteration u <- (1-eta) u + eta a/(Kv), v <- (1-eta) v + eta b/(K^T u) from u0, v0 (default ones)."""
+    M, n, ld = _mat(M)
+    a, b = _f32(a, n), _f32(b, n)
+    u = _f64(np.ones(n) if u0 is None else u0, n)
+    v = _f64(np.ones(n) if v0 is None else v0, n)
+    _load().or_sinkhorn_damped(n, _p32(M), ld, kind, float(eps), _p32(a), _p32(b), float(eta), int(iters),
+                               _p64(u), _p64(v))
     return u, v
 
 

@@ -21,6 +21,7 @@
  *   - the c-client All-to-All protocol with row blocks I_j, local matvecs
  *     q_I = K_{I,:} v and r_I = (K_{:,I})^T u, Allgather of slices
  *                                           (Algorithm 1, Section 3.1, Assumption 1)
+ *   - the relaxed update u <- (1-eta) u + eta a ./ (K v) and its v counterpart         (Section 3.3)
  *   - the strict row-partition form r = sum_j K_{I_j,:}^T u_{I_j}
  *                                           (2D block baseline of the appendix)
  *   - stabilised log-domain updates with f = eps log u, g = eps log v
@@ -126,6 +127,21 @@ void or_sinkhorn_scaling(int64_t n, const float *M, int64_t ld, int kind, double
         or_row_pass(n, M, ld, kind, eps, a, v, u, NULL);
         or_col_pass(n, M, ld, kind, eps, b, u, v, NULL);
     }
+}
+
+/* Relaxed (damped) scaling iteration, the centralized view given with the asynchronous variant
+ * (Section 3.3):  u <- (1 - eta) u + eta a ./ (K v),  v <- (1 - eta) v + eta b ./ (K^T u), the v update
+ * using the new u.  eta = 1 is or_sinkhorn_scaling. */
+void or_sinkhorn_damped(int64_t n, const float *M, int64_t ld, int kind, double eps, const float *a,
+                        const float *b, double eta, int64_t iters, double *u, double *v) {
+    double *t = (double *)malloc(sizeof(double) * (size_t)n);
+    for (int64_t it = 0; it < iters; ++it) {
+        or_row_pass(n, M, ld, kind, eps, a, v, t, NULL);
+        for (int64_t i = 0; i < n; ++i) u[i] = (1.0 - eta) * u[i] + eta * t[i];
+        or_col_pass(n, M, ld, kind, eps, b, u, t, NULL);
+        for (int64_t l = 0; l < n; ++l) v[l] = (1.0 - eta) * v[l] + eta * t[l];
+    }
+    free(t);
 }
 
 /* Algorithm 1 taken literally with c logical clients.  Client j keeps its OWN copy of the

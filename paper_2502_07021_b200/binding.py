@@ -38,6 +38,7 @@ _SIGNATURES = {
     "fs_set_scalings": (_int, [_vp, _vp, _vp, _vp]),
     "fs_reset": (_int, [_vp, _vp]),
     "fs_transport_cost": (_int, [_vp, _vp, _i64, _vp, _vp]),
+    "fs_set_damping": (_int, [_vp, _dbl]),
     "fs_set_error_trace": (_int, [_vp, _i32]),
     "fs_error_trace": (_int, [_vp, _vp, _vp, _i32, ctypes.POINTER(_i32), _vp]),
     "fs_block_errors": (_int, [_vp, _vp]),
@@ -161,6 +162,10 @@ def fs_transport_cost(s, C_dev, ldc, nbatch=1, stream=None):
     out = np.zeros(nbatch)
     _check(lib().fs_transport_cost(s, _dev(C_dev), ldc, out.ctypes.data_as(_vp), _stream(stream)), "fs_transport_cost")
     return out
+
+
+def fs_set_damping(s, eta):
+    _check(lib().fs_set_damping(s, float(eta)), "fs_set_damping")
 
 
 def fs_set_error_trace(s, check_every):

@@ -30,7 +30,7 @@ template <bool TRANS>
 __global__ void __launch_bounds__(kThreads)
 batched_fma_kernel(const float *__restrict__ K, int64_t ld, int n, int nbatch, const float *__restrict__ in,
                    const float *__restrict__ marg, float *__restrict__ out, float *__restrict__ diff, int update,
-                   int vecK, int vecV, FsDeviceStatus *status) {
+                   float eta, int vecK, int vecV, FsDeviceStatus *status) {
     __shared__ __align__(16) float As[BK][BM + 4];
     __shared__ __align__(16) float Bs[BK][BN + 4];
     const int tid = threadIdx.x;
@@ -104,7 +104,7 @@ batched_fma_kernel(const float *__restrict__ K, int64_t ld, int n, int nbatch, c
             const float s = acc[r][q], mg = marg[idx], old = out[idx];
             diff[idx] = fmaf(old, s, -mg);
             if (update) {
-                const float nv = mg / s;
+                const float nv = eta == 1.f ? mg / s : fmaf(eta, mg / s, (1.f - eta) * old);
                 out[idx] = nv;
                 if (!(nv > 0.f) || isinf(nv)) status->nonfinite = 1;
             }
@@ -115,15 +115,15 @@ batched_fma_kernel(const float *__restrict__ K, int64_t ld, int n, int nbatch, c
 } // namespace
 
 void fsk_batched_pass_fma(const float *K, int64_t ld, int64_t n, int nbatch, int transposed, const float *in,
-                          const float *marg, float *out, float *diff, int update, FsDeviceStatus *status,
+                          const float *marg, float *out, float *diff, int update, float eta, FsDeviceStatus *status,
                           cudaStream_t st) {
     dim3 grid((unsigned)((n + BM - 1) / BM), (unsigned)((nbatch + BN - 1) / BN));
     const int vecK = ((reinterpret_cast<uintptr_t>(K) & 15) == 0 && (ld & 3) == 0) ? 1 : 0;
     const int vecV = ((reinterpret_cast<uintptr_t>(in) & 15) == 0 && (n & 3) == 0) ? 1 : 0;
     if (transposed)
-        batched_fma_kernel<true><<<grid, kThreads, 0, st>>>(K, ld, (int)n, nbatch, in, marg, out, diff, update, vecK,
-                                                           vecV, status);
+        batched_fma_kernel<true><<<grid, kThreads, 0, st>>>(K, ld, (int)n, nbatch, in, marg, out, diff, update, eta,
+                                                           vecK, vecV, status);
     else
-        batched_fma_kernel<false><<<grid, kThreads, 0, st>>>(K, ld, (int)n, nbatch, in, marg, out, diff, update, vecK,
-                                                            vecV, status);
+        batched_fma_kernel<false><<<grid, kThreads, 0, st>>>(K, ld, (int)n, nbatch, in, marg, out, diff, update, eta,
+                                                            vecK, vecV, status);
 }

@@ -265,7 +265,7 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bflo
 __global__ void __launch_bounds__(256)
 batched_tc_finish_kernel(const float *__restrict__ partials, int ksplit, int n, int nbatch, int64_t ldb, int mtiles,
                          const float *__restrict__ marg, float *__restrict__ out, float *__restrict__ diff,
-                         __nv_bfloat16 *__restrict__ op_hi, __nv_bfloat16 *__restrict__ op_lo, int update,
+                         __nv_bfloat16 *__restrict__ op_hi, __nv_bfloat16 *__restrict__ op_lo, int update, float eta,
                          FsDeviceStatus *status) {
     const int tile = blockIdx.x >> 4, slice = blockIdx.x & 15;
     const int mtile = tile % mtiles, ntile = tile / mtiles;
@@ -287,7 +287,7 @@ batched_tc_finish_kernel(const float *__restrict__ partials, int ksplit, int n, 
         const float mg = marg[idx], old = out[idx];
         diff[idx] = fmaf(old, qs[j], -mg);
         if (update) {
-            const float nv = mg / qs[j];
+            const float nv = eta == 1.f ? mg / qs[j] : fmaf(eta, mg / qs[j], (1.f - eta) * old);
             out[idx] = nv;
             __nv_bfloat16 hi, lo;
             split_bf16(nv, hi, lo);
@@ -434,7 +434,7 @@ void fsk_tc_refresh(void *tc, const float *u, const float *v, cudaStream_t st) {
 }
 
 // One batched pass on the tensor-core engine; two launches.
-void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float *diff, int update,
+void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float *diff, int update, float eta,
                  FsDeviceStatus *status, cudaStream_t st) {
     TcState *t = static_cast<TcState *>(tc);
     dim3 grid((unsigned)t->mtiles, (unsigned)t->ksplit, (unsigned)t->ntiles);
@@ -445,6 +445,6 @@ void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float 
         batched_tc_kernel<<<grid, kTcThreads, SMEM_BYTES, st>>>(t->tmKt_hi, t->tmKt_lo, t->tmU_hi, t->tmU_lo, t->partials,
                                                               t->kblocks, t->ksplit, status);
     batched_tc_finish_kernel<<<(unsigned)(t->mtiles * t->ntiles * 16), 256, 0, st>>>(t->partials, t->ksplit, (int)t->n, t->nbatch, t->ldb, t->mtiles, marg, out, diff,
-                                                   transposed ? t->V_hi : t->U_hi, transposed ? t->V_lo : t->U_lo, update,
+                                                   transposed ? t->V_hi : t->U_hi, transposed ? t->V_lo : t->U_lo, update, eta,
                                                    status);
 }

@@ -115,13 +115,14 @@ bool use_tc(const fs_solver *s) { return s->tc != nullptr && s->batch_engine != 
 
 void enqueue_row(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
     if (s->nbatch > 1 && use_tc(s)) {
-        fsk_tc_pass(s->tc, 0, s->a, s->x, s->rowdiff, update, s->status, st);
+        fsk_tc_pass(s->tc, 0, s->a, s->x, s->rowdiff, update, s->eta, s->status, st);
         launches += 2;
     } else if (s->nbatch > 1) {
-        fsk_batched_pass_fma(s->mat, s->mat_ld, s->n, s->nbatch, 0, s->y, s->a, s->x, s->rowdiff, update, s->status, st);
+        fsk_batched_pass_fma(s->mat, s->mat_ld, s->n, s->nbatch, 0, s->y, s->a, s->x, s->rowdiff, update, s->eta, s->status,
+                             st);
         launches += 1;
     } else if (s->domain == FS_DOMAIN_SCALING) {
-        fsk_row_pass(s->plan, s->mat, s->mat_ld, s->n, s->y, s->a, s->x, s->rowdiff, update, s->status, st);
+        fsk_row_pass(s->plan, s->mat, s->mat_ld, s->n, s->y, s->a, s->x, s->rowdiff, update, s->eta, s->status, st);
         launches += fsk_pass_launches_row();
     } else {
         fsk_log_row_pass(s->plan, s->mat, s->mat_ld, s->n, s->eps, s->ys, s->a, s->loga, s->x, s->xs, s->rowdiff,
@@ -132,14 +133,15 @@ void enqueue_row(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
 
 void enqueue_col(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
     if (s->nbatch > 1 && use_tc(s)) {
-        fsk_tc_pass(s->tc, 1, s->b, s->y, s->coldiff, update, s->status, st);
+        fsk_tc_pass(s->tc, 1, s->b, s->y, s->coldiff, update, s->eta, s->status, st);
         launches += 2;
     } else if (s->nbatch > 1) {
-        fsk_batched_pass_fma(s->mat, s->mat_ld, s->n, s->nbatch, 1, s->x, s->b, s->y, s->coldiff, update, s->status, st);
+        fsk_batched_pass_fma(s->mat, s->mat_ld, s->n, s->nbatch, 1, s->x, s->b, s->y, s->coldiff, update, s->eta, s->status,
+                             st);
         launches += 1;
     } else if (s->domain == FS_DOMAIN_SCALING) {
         fsk_col_pass(s->plan, s->mat, s->mat_ld, s->n, s->n_pad, s->tiles_dev, (int)s->tiles.size(), s->x, s->b, s->y,
-                     s->partials, s->coldiff, update, s->status, st);
+                     s->partials, s->coldiff, update, s->eta, s->status, st);
         launches += fsk_pass_launches_col();
     } else {
         fsk_log_col_pass(s->plan, s->mat, s->mat_ld, s->n, s->n_pad, s->eps, s->tiles_dev, (int)s->tiles.size(), s->xs,
@@ -164,7 +166,7 @@ void enqueue_fused_rows(fs_solver *s, cudaStream_t st, int64_t &launches) {
                                 s->loga, s->x, s->xs, s->rowdiff, s->fused_partials, s->status, st);
     else
         fsk_fused_iteration(s->fused, s->mat, s->mat_ld, s->n, s->fused_tiles_dev, s->fused_ntiles, s->y, s->a, s->x,
-                            s->rowdiff, s->fused_partials, s->status, st);
+                            s->rowdiff, s->fused_partials, s->eta, s->status, st);
     launches += 1;
 }
 
@@ -173,7 +175,7 @@ void enqueue_fused_finish(fs_solver *s, cudaStream_t st, int64_t &launches) {
         fsk_log_col_finish(s->n, s->n, s->fused.nclusters, s->eps, s->fused_partials, s->b, s->logb, s->y, s->ys,
                            s->coldiff, 1, s->status, st);
     else
-        fsk_col_finish(s->n, s->n, s->fused.nclusters, s->fused_partials, s->b, s->y, s->coldiff, 1, s->status, st);
+        fsk_col_finish(s->n, s->n, s->fused.nclusters, s->fused_partials, s->b, s->y, s->coldiff, 1, s->eta, s->status, st);
     launches += 1;
 }
 
@@ -432,6 +434,16 @@ int fs_set_option(fs_solver *s, int option, int64_t value) {
     default:
         return FS_ERR_BAD_N;
     }
+}
+
+int fs_set_damping(fs_solver *s, double eta) {
+    if (!s) return FS_ERR_NULL;
+    if (!(eta > 0.0) || eta > 1.0) return FS_ERR_BAD_N;
+    if (s->domain == FS_DOMAIN_LOG && eta != 1.0) return FS_ERR_UNSUPPORTED;
+    cudaDeviceSynchronize();
+    s->eta = (float)eta;
+    destroy_graphs(s);
+    return FS_OK;
 }
 
 int fs_set_error_trace(fs_solver *s, int32_t check_every) {

@@ -86,6 +86,7 @@ struct fs_solver {
     int64_t launches = 0;
     bool use_graph = true;
     int batch_engine = 0;
+    float eta = 1.f;                        // relaxation of the scaling updates (1 = plain Sinkhorn)
 
     // batched tensor-core path
     void *tc = nullptr;
@@ -104,11 +105,11 @@ struct fs_solver {
 // ---- passes.cu ---------------------------------------------------------------------------
 // Row pass, scaling domain: q_i = sum_l K_il v_l; rowdiff_i = u_i q_i - a_i; if update u_i = a_i/q_i.
 void fsk_row_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, const float *v, const float *a,
-                  float *u, float *rowdiff, int update, FsDeviceStatus *status, cudaStream_t st);
+                  float *u, float *rowdiff, int update, float eta, FsDeviceStatus *status, cudaStream_t st);
 // Column pass, scaling domain, two deterministic stages.
 void fsk_col_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
                   int ntiles, const float *u, const float *b, float *v, float *partials, float *coldiff,
-                  int update, FsDeviceStatus *status, cudaStream_t st);
+                  int update, float eta, FsDeviceStatus *status, cudaStream_t st);
 // Log-domain row pass: L_i = LSE_l((g_l - C_il)/eps) streamed once with a running (max, sum).
 // ys = g * log2(e)/eps on input; writes f and xs = f * log2(e)/eps when update.
 void fsk_log_row_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n, double eps, const float *ys,
@@ -120,7 +121,7 @@ void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n
                       FsDeviceStatus *status, cudaStream_t st);
 // Stage 2 of the column pass alone: r_l = sum over `ntiles` partial rows of pitch n_pad, residual, divide.
 void fsk_col_finish(int64_t n, int64_t n_pad, int ntiles, const float *partials, const float *b, float *v,
-                    float *coldiff, int update, FsDeviceStatus *status, cudaStream_t st);
+                    float *coldiff, int update, float eta, FsDeviceStatus *status, cudaStream_t st);
 void fsk_log_col_finish(int64_t n, int64_t n_pad, int ntiles, double eps, const float *partials, const float *b,
                         const float *logb, float *g, float *ys, float *coldiff, int update, FsDeviceStatus *status,
                         cudaStream_t st);
@@ -131,7 +132,7 @@ int fsk_pass_launches_col();
 FsFusedPlan fsk_fused_plan(int64_t n, bool vec);
 cudaError_t fsk_fused_iteration(const FsFusedPlan &p, const float *K, int64_t ld, int64_t n, const FsRowTile *tiles,
                                 int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials,
-                                FsDeviceStatus *status, cudaStream_t st);
+                                float eta, FsDeviceStatus *status, cudaStream_t st);
 
 // ---- fused_log.cu ------------------------------------------------------------------------
 FsFusedPlan fsk_fused_log_plan(int64_t n, bool vec);
@@ -144,7 +145,7 @@ cudaError_t fsk_fused_log_iteration(const FsFusedPlan &p, const float *C, int64_
 // out[p][i] = marg[p][i] / sum_l Mat(i,l) in[p][l], Mat(i,l) = K[i][l] (transposed = 0) or K[l][i].
 // diff[p][i] = out_old[p][i] * sum - marg[p][i].
 void fsk_batched_pass_fma(const float *K, int64_t ld, int64_t n, int nbatch, int transposed, const float *in,
-                          const float *marg, float *out, float *diff, int update, FsDeviceStatus *status,
+                          const float *marg, float *out, float *diff, int update, float eta, FsDeviceStatus *status,
                           cudaStream_t st);
 
 // ---- batched_tc.cu -----------------------------------------------------------------------
@@ -152,7 +153,7 @@ void fsk_batched_pass_fma(const float *K, int64_t ld, int64_t n, int nbatch, int
 void *fsk_tc_create(const float *K, int64_t ld, int64_t n, int nbatch, cudaStream_t st); // nullptr on failure
 void fsk_tc_destroy(void *tc);
 void fsk_tc_refresh(void *tc, const float *u, const float *v, cudaStream_t st);
-void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float *diff, int update,
+void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float *diff, int update, float eta,
                  FsDeviceStatus *status, cudaStream_t st);
 
 // ---- setup.cu ----------------------------------------------------------------------------

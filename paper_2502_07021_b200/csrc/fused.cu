@@ -42,7 +42,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, int nclusters, int nstages,
                        const FsRowTile *__restrict__ tiles, int ntiles, const float *__restrict__ v,
                        const float *__restrict__ a, float *__restrict__ u, float *__restrict__ rowdiff,
-                       float *__restrict__ partials, FsDeviceStatus *status) {
+                       float *__restrict__ partials, float eta, FsDeviceStatus *status) {
     extern __shared__ uint8_t smem_raw[];
     constexpr int W = F * 1024;
     const uint32_t stage_bytes = W * 4;
@@ -170,7 +170,7 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
                 }
                 const float ai = __shfl_sync(0xffffffffu, a_lane, row - tile.begin);
                 const float uo = __shfl_sync(0xffffffffu, uo_lane, row - tile.begin);
-                const float ui = ai / q;
+                const float ui = eta == 1.f ? ai / q : fmaf(eta, ai / q, (1.f - eta) * uo);
                 if (t == 0 && rank == 0) {
                     rowdiff[row] = fmaf(uo, q, -ai);
                     u[row] = ui;
@@ -213,7 +213,7 @@ size_t fused_smem_bytes(int F, int nstages) {
 template <int F>
 cudaError_t launch_fused(int S, int nclusters, int nstages, cudaStream_t st, const float *K, int64_t ld, int n,
                          const FsRowTile *tiles, int ntiles, const float *v, const float *a, float *u, float *rowdiff,
-                         float *partials, FsDeviceStatus *status) {
+                         float *partials, float eta, FsDeviceStatus *status) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(nclusters * S));
     cfg.blockDim = dim3(kFusedThreads);
@@ -227,7 +227,7 @@ cudaError_t launch_fused(int S, int nclusters, int nstages, cudaStream_t st, con
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, fused_iteration_kernel<F>, K, ld, n, S, nclusters, nstages, tiles, ntiles, v, a, u,
-                              rowdiff, partials, status);
+                              rowdiff, partials, eta, status);
 }
 
 template <int F>
@@ -289,11 +289,11 @@ FsFusedPlan fsk_fused_plan(int64_t n, bool vec) {
 // [nclusters][n]; the caller runs the stage-2 kernel over them.
 cudaError_t fsk_fused_iteration(const FsFusedPlan &p, const float *K, int64_t ld, int64_t n, const FsRowTile *tiles,
                                 int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials,
-                                FsDeviceStatus *status, cudaStream_t st) {
+                                float eta, FsDeviceStatus *status, cudaStream_t st) {
     switch (p.F) {
-    case 2: return launch_fused<2>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, status);
-    case 4: return launch_fused<4>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, status);
-    case 8: return launch_fused<8>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, status);
-    default: return launch_fused<16>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, status);
+    case 2: return launch_fused<2>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
+    case 4: return launch_fused<4>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
+    case 8: return launch_fused<8>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
+    default: return launch_fused<16>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
     }
 }

@@ -57,6 +57,10 @@ __device__ __forceinline__ void lse_merge(float &m, float &s, float mo, float so
     m = mn;
 }
 __device__ __forceinline__ void flag_bad(FsDeviceStatus *status) { status->nonfinite = 1; }
+// Relaxed update of Section 3.3, x <- (1 - eta) x_old + eta x_new; eta = 1 is the plain update, bit for bit.
+__device__ __forceinline__ float damped(float x_new, float x_old, float eta) {
+    return eta == 1.f ? x_new : fmaf(eta, x_new, (1.f - eta) * x_old);
+}
 
 // ------------------------------------------------------------------------------------------
 // Row pass, scaling domain.
@@ -64,7 +68,7 @@ template <int L, int R, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 row_pass_kernel(const float *__restrict__ K, int64_t ld, int n, const float *__restrict__ v,
                 const float *__restrict__ a, float *__restrict__ u, float *__restrict__ rowdiff, int update,
-                FsDeviceStatus *status) {
+                float eta, FsDeviceStatus *status) {
     constexpr int G = kThreads / L;
     constexpr int W = L / 32;                        // warps per group
     constexpr int U = (R >= 8) ? 2 : (R >= 4 ? 4 : 8); // column chunks in flight; R*U 128-bit loads per thread
@@ -142,7 +146,7 @@ row_pass_kernel(const float *__restrict__ K, int64_t ld, int n, const float *__r
             const float ai = a[row], uo = u[row];
             rowdiff[row] = fmaf(uo, q, -ai);
             if (update) {
-                const float un = ai / q;
+                const float un = damped(ai / q, uo, eta);
                 u[row] = un;
                 if (!(un > 0.f) || isinf(un)) flag_bad(status);
             }
@@ -339,7 +343,7 @@ col_partial_kernel(const float *__restrict__ K, int64_t ld, int n, int64_t n_pad
 // Column pass stage 2: r_l = sum over tiles in tile order; residual; divide.
 __global__ void __launch_bounds__(kThreads)
 col_finish_kernel(int n, int64_t n_pad, int ntiles, const float *__restrict__ partials, const float *__restrict__ b,
-                  float *__restrict__ v, float *__restrict__ coldiff, int update, FsDeviceStatus *status) {
+                  float *__restrict__ v, float *__restrict__ coldiff, int update, float eta, FsDeviceStatus *status) {
     const int l = blockIdx.x * kThreads + threadIdx.x;
     if (l >= n) return;
     float r = 0.f;
@@ -347,7 +351,7 @@ col_finish_kernel(int n, int64_t n_pad, int ntiles, const float *__restrict__ pa
     const float bl = b[l], vo = v[l];
     coldiff[l] = fmaf(vo, r, -bl);
     if (update) {
-        const float vn = bl / r;
+        const float vn = damped(bl / r, vo, eta);
         v[l] = vn;
         if (!(vn > 0.f) || isinf(vn)) flag_bad(status);
     }
@@ -500,16 +504,16 @@ log_col_finish_kernel(int n, int64_t n_pad, int ntiles, float s2, double eps, co
     } while (0)
 
 void fsk_row_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, const float *v, const float *a,
-                  float *u, float *rowdiff, int update, FsDeviceStatus *status, cudaStream_t st) {
-    FS_ROW_DISPATCH(row_pass_kernel, K, ld, (int)n, v, a, u, rowdiff, update, status);
+                  float *u, float *rowdiff, int update, float eta, FsDeviceStatus *status, cudaStream_t st) {
+    FS_ROW_DISPATCH(row_pass_kernel, K, ld, (int)n, v, a, u, rowdiff, update, eta, status);
 }
 
 void fsk_col_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
                   int ntiles, const float *u, const float *b, float *v, float *partials, float *coldiff,
-                  int update, FsDeviceStatus *status, cudaStream_t st) {
+                  int update, float eta, FsDeviceStatus *status, cudaStream_t st) {
     FS_COL_DISPATCH(col_partial_kernel, K, ld, (int)n, n_pad, tiles, nstrips, u, partials);
     col_finish_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>(
-        (int)n, n_pad, ntiles, partials, b, v, coldiff, update, status);
+        (int)n, n_pad, ntiles, partials, b, v, coldiff, update, eta, status);
 }
 
 void fsk_log_row_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n, double eps, const float *ys,
@@ -530,9 +534,9 @@ void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n
 }
 
 void fsk_col_finish(int64_t n, int64_t n_pad, int ntiles, const float *partials, const float *b, float *v,
-                    float *coldiff, int update, FsDeviceStatus *status, cudaStream_t st) {
+                    float *coldiff, int update, float eta, FsDeviceStatus *status, cudaStream_t st) {
     col_finish_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>((int)n, n_pad, ntiles, partials, b, v,
-                                                                                   coldiff, update, status);
+                                                                                   coldiff, update, eta, status);
 }
 
 void fsk_log_col_finish(int64_t n, int64_t n_pad, int ntiles, double eps, const float *partials, const float *b,

@@ -446,6 +446,43 @@ def test_launch_count_and_iteration_counter():
         assert fs.fs_iterations_done(g.h) == 10
 
 
+# ------------------------------------------------------------------ relaxed (damped) updates, Section 3.3
+
+@pytest.mark.parametrize("cfg,n,nb,eta", [(1, 512, 1, 0.5), (2, 2048, 1, 0.25), (4, 16384, 1, 0.5), (5, 1024, 64, 0.5),
+                                          (5, 300, 4, 0.7)])
+def test_damped_updates(cfg, n, nb, eta):
+    """Every engine (two-pass, fused, batched FMA, batched tensor cores) against the oracle's relaxed
+    iteration; eta = 1 must reproduce the plain run bit for bit."""
+    w = workloads.make(cfg, n=n, nbatch=nb)
+    with GpuSolver(w.K, KK, w.eps, w.a, w.b, w.offsets, SC) as g:
+        fs.fs_set_damping(g.h, eta)
+        g.iterate(10)
+        x, y = g.scalings()
+    with GpuSolver(w.K, KK, w.eps, w.a, w.b, w.offsets, SC) as g:
+        fs.fs_set_damping(g.h, 1.0)
+        g.iterate(3)
+        x1, y1 = g.scalings()
+    x0, y0 = run(w, 3)
+    assert np.array_equal(x1, x0) and np.array_equal(y1, y0)
+    for p in ([0] if nb == 1 else sorted({0, nb - 1})):
+        ap, bp = (w.a, w.b) if nb == 1 else (w.a[p], w.b[p])
+        xp, yp = (x, y) if nb == 1 else (x[p], y[p])
+        u, v = oracle.sinkhorn_damped(w.K, oracle.KIND_KERNEL, w.eps, ap, bp, eta, 10)
+        assert rel_err(xp, u) <= TOL_UV and rel_err(yp, v) <= TOL_UV
+
+
+def test_damping_is_rejected_in_the_log_domain():
+    w = workloads.make(3, n=256)
+    with GpuSolver(w.C, KC, w.eps, w.a, w.b, w.offsets, LG) as g:
+        with pytest.raises(fs.FsError) as ei:
+            fs.fs_set_damping(g.h, 0.5)
+        assert ei.value.code == fs.FS_ERR_UNSUPPORTED
+        fs.fs_set_damping(g.h, 1.0)
+        for bad in (0.0, 1.5, float("nan")):
+            with pytest.raises(fs.FsError):
+                fs.fs_set_damping(g.h, bad)
+
+
 # ------------------------------------------------------------------ failures are reported, not trapped
 
 def test_nonfinite_is_flagged():

@@ -119,6 +119,35 @@ def test_rank1_nonsymmetric_catches_transpose():
     np.testing.assert_allclose(v * r, b, rtol=1e-15)
 
 
+# ------------------------------------------------------------------ relaxed (damped) update
+
+def test_damped_update_closed_form_fixed_point_and_eta_one():
+    n, eps, eta = 21, 0.3, 0.4
+    C, x, y = dyadic_additive(n, 77)
+    a, b = dirichlet_pair(n, 78)
+    a64, b64 = a.astype(np.float64), b.astype(np.float64)
+    p, q = np.exp(-x / eps), np.exp(-y / eps)
+    # one relaxed iteration on the rank-one kernel, from u = v = 1
+    u, v = oracle.sinkhorn_damped(C, C_, eps, a, b, eta, 1)
+    u_ref = (1 - eta) + eta * a64 / (p * q.sum())
+    v_ref = (1 - eta) + eta * b64 / (q * (p * u_ref).sum())
+    np.testing.assert_allclose(u, u_ref, rtol=1e-13)
+    np.testing.assert_allclose(v, v_ref, rtol=1e-13)
+    # eta = 1 is the plain iteration, bit for bit
+    Cr = random_cost(n, 79)
+    u1, v1 = oracle.sinkhorn_damped(Cr, C_, eps, a, b, 1.0, 7)
+    u0, v0 = oracle.sinkhorn_scaling(Cr, C_, eps, a, b, 7)
+    assert np.array_equal(u1, u0) and np.array_equal(v1, v0)
+    # the relaxed map has the same fixed point: same plan as plain Sinkhorn
+    ud, vd = oracle.sinkhorn_damped(Cr, C_, eps, a, b, eta, 4000)
+    us, vs = oracle.sinkhorn_scaling(Cr, C_, eps, a, b, 4000)
+    np.testing.assert_allclose(oracle.plan(Cr, C_, eps, SC, ud, vd), oracle.plan(Cr, C_, eps, SC, us, vs), rtol=1e-9)
+    # and it really is a convex combination of the old value and the plain update
+    u_half, _ = oracle.sinkhorn_damped(Cr, C_, eps, a, b, 0.5, 1)
+    u_full, _ = oracle.sinkhorn_scaling(Cr, C_, eps, a, b, 1)
+    np.testing.assert_allclose(u_half, 0.5 + 0.5 * u_full, rtol=1e-15)
+
+
 # ------------------------------------------------------------------ P2 large-eps limit
 
 def test_large_eps_limit():
