@@ -369,6 +369,7 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
             FS_CU(cudaMemsetAsync(s->fused_partials, 0, pbytes, st));
         }
     }
+    if (domain == FS_DOMAIN_SCALING && nbatch == 1) s->resident = fsk_resident_plan(n);
     // batched problems: tensor-core engine when the batch is wide enough to fill its 128-problem tiles
     if (nbatch >= kTcMinBatch && n >= kTcMinN) s->tc = fsk_tc_create(s->mat, s->mat_ld, n, nbatch, st);
     rc = set_initial_state(s, st);
@@ -413,6 +414,10 @@ int fs_set_option(fs_solver *s, int option, int64_t value) {
         if (value == 2 && !s->fused.enabled) return FS_ERR_UNSUPPORTED;
         s->fused_mode = (int)value;
         destroy_graphs(s);
+        return FS_OK;
+    case FS_OPT_RESIDENT:
+        if (value < 0 || value > 1) return FS_ERR_BAD_N;
+        s->resident_mode = (int)value;
         return FS_OK;
     case FS_OPT_ROW_SHAPE: {
         const int L = (int)(value / 1000), R = (int)(value % 1000);
@@ -463,6 +468,14 @@ int fs_iterate(fs_solver *s, int32_t k, void *stream) {
     const int ce = s->check_every;
     int chunk = kGraphChunk;
     if (ce > 0 && ce <= kGraphChunk) chunk = ce * (kGraphChunk / ce);
+    // small problems without an error trace: all k iterations in one launch of the K-resident kernel
+    if (k > 0 && s->resident.enabled && s->resident_mode != 0 && ce == 0) {
+        FS_CU(fsk_resident_iterate(s->resident, s->mat, s->mat_ld, s->n, k, s->a, s->b, s->x, s->y, s->rowdiff, s->coldiff,
+                                   s->eta, s->status, st));
+        s->launches += 1;
+        s->iter_done += k;
+        return FS_OK;
+    }
     int64_t remaining = k;
     while (remaining > 0) {
         const int len = (int)std::min<int64_t>(remaining, chunk);

@@ -38,6 +38,14 @@ struct FsFusedPlan {
     int tile_rows; // height of the row tiles dealt to the clusters
 };
 
+// Configuration of the K-resident persistent kernel (resident.cu) for small n.
+struct FsResidentPlan {
+    bool enabled;
+    int S;             // CTAs in the one cluster that holds K
+    int m;             // rows (and owned columns) per CTA
+    size_t smem_bytes; // dynamic shared memory per CTA
+};
+
 struct FsDeviceStatus {
     int nonfinite;   // set by any kernel that produced a non-finite or non-positive scaling
     int trace_count; // number of trace entries appended so far
@@ -86,6 +94,8 @@ struct fs_solver {
     int64_t launches = 0;
     bool use_graph = true;
     int batch_engine = 0;
+    FsResidentPlan resident{};
+    int resident_mode = 1;                  // 0 = never, 1 = automatic
     float eta = 1.f;                        // relaxation of the scaling updates (1 = plain Sinkhorn)
 
     // batched tensor-core path
@@ -133,6 +143,12 @@ FsFusedPlan fsk_fused_plan(int64_t n, bool vec);
 cudaError_t fsk_fused_iteration(const FsFusedPlan &p, const float *K, int64_t ld, int64_t n, const FsRowTile *tiles,
                                 int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials,
                                 float eta, FsDeviceStatus *status, cudaStream_t st);
+
+// ---- resident.cu -------------------------------------------------------------------------
+FsResidentPlan fsk_resident_plan(int64_t n);
+cudaError_t fsk_resident_iterate(const FsResidentPlan &p, const float *K, int64_t ld, int64_t n, int iters, const float *a,
+                                 const float *b, float *u, float *v, float *rowdiff, float *coldiff, float eta,
+                                 FsDeviceStatus *status, cudaStream_t st);
 
 // ---- fused_log.cu ------------------------------------------------------------------------
 FsFusedPlan fsk_fused_log_plan(int64_t n, bool vec);

@@ -440,10 +440,52 @@ def test_error_trace_matches_oracle():
 def test_launch_count_and_iteration_counter():
     w = workloads.make(1)
     with GpuSolver(w.matrix, w.kind, w.eps, w.a, w.b, w.offsets, w.domain) as g:
+        fs.fs_set_option(g.h, fs.FS_OPT_RESIDENT, 0)
         before = fs.fs_launch_count(g.h)
         g.iterate(10)
         assert fs.fs_launch_count(g.h) - before == 30          # row pass + two column stages per iteration
         assert fs.fs_iterations_done(g.h) == 10
+        fs.fs_set_option(g.h, fs.FS_OPT_RESIDENT, 1)
+        before = fs.fs_launch_count(g.h)
+        g.iterate(10)
+        assert fs.fs_launch_count(g.h) - before == 1           # K-resident kernel: all iterations in one launch
+        assert fs.fs_iterations_done(g.h) == 20
+
+
+@pytest.mark.parametrize("n", [8, 9, 33, 100, 512, 590, 600, 640, 700, 720])
+def test_resident_kernel_small_problems(n):
+    """The K-resident persistent kernel (one cluster of 8 or 16 CTAs holds K in shared memory and runs all
+    iterations in one launch) against the oracle and the two-pass graph path, with unequal blocks."""
+    w = workloads.make(1, n=n)
+    off = some_offsets(n, 7 * n)
+    res = {}
+    for mode in (0, 1):
+        with GpuSolver(w.K, KK, w.eps, w.a, w.b, off, SC) as g:
+            fs.fs_set_option(g.h, fs.FS_OPT_RESIDENT, mode)
+            before = fs.fs_launch_count(g.h)
+            g.iterate(4)
+            g.iterate(6)
+            launches = fs.fs_launch_count(g.h) - before
+            assert launches == (30 if mode == 0 else 2)
+            res[mode] = g.scalings() + tuple(e[0] for e in g.errors(1))
+    u, v = oracle.sinkhorn_scaling(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, 10)
+    for mode in (0, 1):
+        assert rel_err(res[mode][0], u) <= TOL_UV and rel_err(res[mode][1], v) <= TOL_UV
+    assert rel_err(res[1][0], res[0][0]) < 1e-5 and rel_err(res[1][1], res[0][1]) < 1e-5
+    assert abs(res[1][2] - res[0][2]) < 1e-6
+
+
+def test_resident_kernel_converges_and_flags_nonfinite():
+    w = workloads.make(1)
+    check_converged(w, w.iters, w.C)                          # default path for n = 512 is the resident kernel
+    n = 64
+    C, K, a, b = rand_problem(n, 5)
+    K[7, :] = 0.0
+    with GpuSolver(K, KK, 0.3, a, b, [0, n], SC) as g:
+        g.iterate(2)
+        with pytest.raises(fs.FsError) as ei:
+            g.errors(1)
+        assert ei.value.code == fs.FS_ERR_NONFINITE
 
 
 # ------------------------------------------------------------------ relaxed (damped) updates, Section 3.3
