@@ -278,7 +278,7 @@ def run_ours(args, w, rank, local_rank, world):
 
     # dominant kernel: timed with CUDA events on the launching stream, right after the timed region
     peaks, peak_kind = measured_peaks()
-    fused = w.nbatch == 1 and w.domain == workloads.DOMAIN_SCALING and w.n >= 12288 and w.n % 4 == 0
+    fused = w.nbatch == 1 and w.domain == workloads.DOMAIN_SCALING and w.n >= 6144 and w.n % 4 == 0
     reps = 20
 
     def timed(fn):

@@ -29,7 +29,7 @@ int cuda_fail(cudaError_t e, const char *what) {
 constexpr double kLog2e = 1.4426950408889634;
 constexpr int kGraphChunk = 64;
 constexpr int kTraceCap = 1 << 16;
-constexpr int64_t kFusedAutoMinN = 12288;
+constexpr int64_t kFusedAutoMinN = 6144;
 constexpr int kTcMinBatch = 32;
 constexpr int kTcMinN = 512;
 

@@ -33,6 +33,7 @@ struct FsFusedPlan {
     bool enabled;
     int S;         // CTAs per cluster (column segments per row)
     int F;         // 128-bit column groups per thread: a CTA covers F*1024 columns
+    int R;         // rows per shared-memory stage (scaling-domain kernel)
     int nstages;   // shared-memory ring depth (row segments in flight per CTA)
     int nclusters; // clusters resident at once = number of column-partial rows
     int tile_rows; // height of the row tiles dealt to the clusters

@@ -37,7 +37,9 @@ constexpr int kXchgStride = 32;             // floats per exchange slot: S*8 per
 using namespace fsptx;
 
 // F = 128-bit column groups per thread: a CTA covers W = F*1024 columns of each row.
-template <int F>
+// R = rows per shared-memory stage: short rows are processed R at a time so that the per-step costs
+// (barrier waits, warp reductions, the exchange) are shared by R rows.
+template <int F, int R>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, int nclusters, int nstages,
                        const FsRowTile *__restrict__ tiles, int ntiles, const float *__restrict__ v,
@@ -45,10 +47,12 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
                        float *__restrict__ partials, float eta, FsDeviceStatus *status) {
     extern __shared__ uint8_t smem_raw[];
     constexpr int W = F * 1024;
-    const uint32_t stage_bytes = W * 4;
+    constexpr uint32_t row_bytes = W * 4;
+    constexpr uint32_t stage_bytes = R * row_bytes;
+    constexpr int slot_floats = R * kXchgStride;
     const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
-    const uint32_t xchg = base + (uint32_t)nstages * stage_bytes;           // [2*nstages][kXchgStride] floats
-    const uint32_t bars = xchg + (uint32_t)(2 * nstages) * kXchgStride * 4; // full[ns], empty[ns], qbar[2 ns]
+    const uint32_t xchg = base + (uint32_t)nstages * stage_bytes;           // [2*nstages][R][kXchgStride] floats
+    const uint32_t bars = xchg + (uint32_t)(2 * nstages) * slot_floats * 4; // full[ns], empty[ns], qbar[2 ns]
     const uint32_t rank = cluster_ctarank();
     const int cluster = blockIdx.x / S;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -74,20 +78,23 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
             int k = 0;
             for (int t = cluster; t < ntiles && ok; t += nclusters) {
                 const FsRowTile tile = tiles[t];
-                for (int row = tile.begin; row < tile.end; ++row, ++k) {
+                for (int row = tile.begin; row < tile.end; row += R, ++k) {
+                    const int cnt = min(R, tile.end - row);
                     const int s = k % nstages;
                     const uint32_t ph = (uint32_t)(k / nstages) & 1u;
                     if (!mbar_wait(bars + 8 * (nstages + s), ph ^ 1u)) { ok = false; break; }
                     const uint32_t full = bars + 8 * s;
-                    // this row's exchange slot: S*8 floats will arrive as asynchronous stores
-                    mbar_expect_tx(bars + 8 * (2 * nstages + k % (2 * nstages)), (uint32_t)(S * kWarpsPerGroup) * 4u);
+                    // this step's exchange slot: S*8 floats per row will arrive as asynchronous stores
+                    mbar_expect_tx(bars + 8 * (2 * nstages + k % (2 * nstages)), (uint32_t)(S * kWarpsPerGroup * cnt) * 4u);
                     if (seg > 0) {
-                        mbar_expect_tx(full, (uint32_t)seg * 4u);
-                        const float *src = K + (int64_t)row * ld + col0;
-                        const uint32_t dst = base + (uint32_t)s * stage_bytes;
-                        for (int off = 0; off < seg; off += 4096) { // 16 KB pieces
-                            const int cnt = min(4096, seg - off);
-                            bulk_load(dst + (uint32_t)off * 4u, src + off, (uint32_t)cnt * 4u, full);
+                        mbar_expect_tx(full, (uint32_t)(seg * cnt) * 4u);
+                        for (int r = 0; r < cnt; ++r) {
+                            const float *src = K + (int64_t)(row + r) * ld + col0;
+                            const uint32_t dst = base + (uint32_t)s * stage_bytes + (uint32_t)r * row_bytes;
+                            for (int off = 0; off < seg; off += 4096) { // 16 KB pieces
+                                const int c = min(4096, seg - off);
+                                bulk_load(dst + (uint32_t)off * 4u, src + off, (uint32_t)c * 4u, full);
+                            }
                         }
                     } else {
                         mbar_arrive(full);
@@ -112,36 +119,49 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
         int k = 0;
         for (int tl = cluster; tl < ntiles && ok; tl += nclusters) {
             const FsRowTile tile = tiles[tl];
-            for (int row = tile.begin; row < tile.end; ++row, ++k) {
+            for (int row = tile.begin; row < tile.end; row += R, ++k) {
+                const int cnt = min(R, tile.end - row);
                 const int s = k % nstages;
                 const int slot = k % (2 * nstages);
                 if (!mbar_wait(bars + 8 * s, (uint32_t)(k / nstages) & 1u)) { ok = false; break; }
                 const uint32_t st = base + (uint32_t)s * stage_bytes + (uint32_t)t * 16u;
-                float acc0 = 0.f, acc1 = 0.f;
+                float acc[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) acc[r] = 0.f;
 #pragma unroll
                 for (int j = 0; j < F; ++j) {
                     if (j * kGroup + t < seg4) {
-                        const float4 kv = lds4(st + (uint32_t)j * (kGroup * 16u));
-                        acc0 = fmaf(kv.x, v4[j].x, acc0);
-                        acc1 = fmaf(kv.y, v4[j].y, acc1);
-                        acc0 = fmaf(kv.z, v4[j].z, acc0);
-                        acc1 = fmaf(kv.w, v4[j].w, acc1);
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            if (r < cnt) {
+                                const float4 kv = lds4(st + (uint32_t)r * row_bytes + (uint32_t)j * (kGroup * 16u));
+                                acc[r] = fmaf(kv.x, v4[j].x, acc[r]);
+                                acc[r] = fmaf(kv.y, v4[j].y, acc[r]);
+                                acc[r] = fmaf(kv.z, v4[j].z, acc[r]);
+                                acc[r] = fmaf(kv.w, v4[j].w, acc[r]);
+                            }
+                        }
                     }
                 }
-                float acc = acc0 + acc1;
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-                if (lane < S) { // lane r delivers this warp's partial to CTA r of the cluster
-                    const uint32_t cell = xchg + (uint32_t)(slot * kXchgStride + (int)rank * kWarpsPerGroup + warp) * 4u;
+                for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], off);
+                }
+                if (lane < S * cnt) { // lane (r, dst) delivers this warp's partial of row r to CTA dst of the cluster
+                    const int r = lane / S, dst = lane % S;
+                    float val = acc[0];
+#pragma unroll
+                    for (int q = 1; q < R; ++q) val = r == q ? acc[q] : val;
+                    const uint32_t cell = xchg + (uint32_t)(slot * slot_floats + r * kXchgStride + (int)rank * kWarpsPerGroup + warp) * 4u;
                     const uint32_t qb = bars + 8 * (2 * nstages + slot);
-                    st_async_f32(map_to_cta(cell, (uint32_t)lane), acc, map_to_cta(qb, (uint32_t)lane));
+                    st_async_f32(map_to_cta(cell, (uint32_t)dst), val, map_to_cta(qb, (uint32_t)dst));
                 }
             }
         }
     } else {
         // ---------------- accumulate group ----------------
         const int t = threadIdx.x - kGroup; // 0..255
-        const int gw = warp - kWarpsPerGroup;
         float4 r4[F];
 #pragma unroll
         for (int j = 0; j < F; ++j) r4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -154,44 +174,56 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
                 a_lane = a[tile.begin + lane];
                 uo_lane = u[tile.begin + lane];
             }
-            for (int row = tile.begin; row < tile.end; ++row, ++k) {
+            for (int row = tile.begin; row < tile.end; row += R, ++k) {
+                const int cnt = min(R, tile.end - row);
                 const int s = k % nstages;
                 const int slot = k % (2 * nstages);
                 if (!mbar_wait(bars + 8 * s, (uint32_t)(k / nstages) & 1u)) { ok = false; break; }
                 if (!mbar_wait_cluster(bars + 8 * (2 * nstages + slot), (uint32_t)(k / (2 * nstages)) & 1u)) { ok = false; break; }
-                const uint32_t my = xchg + (uint32_t)(slot * kXchgStride) * 4u;
-                float q = 0.f;
+                float ui[R];
 #pragma unroll
-                for (int i = 0; i < kMaxS * kWarpsPerGroup / 4; ++i) {
-                    if (i < S * kWarpsPerGroup / 4) {
-                        const float4 c = lds4(my + (uint32_t)i * 16u);
-                        q += (c.x + c.y) + (c.z + c.w);
+                for (int r = 0; r < R; ++r) {
+                    ui[r] = 0.f;
+                    if (r < cnt) {
+                        const uint32_t my = xchg + (uint32_t)(slot * slot_floats + r * kXchgStride) * 4u;
+                        float q = 0.f;
+#pragma unroll
+                        for (int i = 0; i < kMaxS * kWarpsPerGroup / 4; ++i) {
+                            if (i < S * kWarpsPerGroup / 4) {
+                                const float4 c = lds4(my + (uint32_t)i * 16u);
+                                q += (c.x + c.y) + (c.z + c.w);
+                            }
+                        }
+                        const float ai = __shfl_sync(0xffffffffu, a_lane, row + r - tile.begin);
+                        const float uo = __shfl_sync(0xffffffffu, uo_lane, row + r - tile.begin);
+                        ui[r] = eta == 1.f ? ai / q : fmaf(eta, ai / q, (1.f - eta) * uo);
+                        if (t == 0 && rank == 0) {
+                            rowdiff[row + r] = fmaf(uo, q, -ai);
+                            u[row + r] = ui[r];
+                            if (!(ui[r] > 0.f) || isinf(ui[r])) status->nonfinite = 1;
+                        }
                     }
-                }
-                const float ai = __shfl_sync(0xffffffffu, a_lane, row - tile.begin);
-                const float uo = __shfl_sync(0xffffffffu, uo_lane, row - tile.begin);
-                const float ui = eta == 1.f ? ai / q : fmaf(eta, ai / q, (1.f - eta) * uo);
-                if (t == 0 && rank == 0) {
-                    rowdiff[row] = fmaf(uo, q, -ai);
-                    u[row] = ui;
-                    if (!(ui > 0.f) || isinf(ui)) status->nonfinite = 1;
                 }
                 const uint32_t st = base + (uint32_t)s * stage_bytes + (uint32_t)t * 16u;
 #pragma unroll
                 for (int j = 0; j < F; ++j) {
                     if (j * kGroup + t < seg4) {
-                        const float4 kv = lds4(st + (uint32_t)j * (kGroup * 16u));
-                        r4[j].x = fmaf(kv.x, ui, r4[j].x);
-                        r4[j].y = fmaf(kv.y, ui, r4[j].y);
-                        r4[j].z = fmaf(kv.z, ui, r4[j].z);
-                        r4[j].w = fmaf(kv.w, ui, r4[j].w);
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            if (r < cnt) {
+                                const float4 kv = lds4(st + (uint32_t)r * row_bytes + (uint32_t)j * (kGroup * 16u));
+                                r4[j].x = fmaf(kv.x, ui[r], r4[j].x);
+                                r4[j].y = fmaf(kv.y, ui[r], r4[j].y);
+                                r4[j].z = fmaf(kv.z, ui[r], r4[j].z);
+                                r4[j].w = fmaf(kv.w, ui[r], r4[j].w);
+                            }
+                        }
                     }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bars + 8 * (nstages + s)); // stage back to the producer
             }
         }
-        (void)gw;
         if (ok) {
             float4 *out = reinterpret_cast<float4 *>(partials + (int64_t)cluster * n + col0);
 #pragma unroll
@@ -206,50 +238,48 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
     cluster_sync_all(); // nobody leaves while a peer may still write into its shared memory
 }
 
-size_t fused_smem_bytes(int F, int nstages) {
-    return (size_t)nstages * F * 4096 + (size_t)2 * nstages * kXchgStride * 4 + (size_t)8 * 4 * nstages + 256;
+size_t fused_smem_bytes(int F, int R, int nstages) {
+    return (size_t)nstages * R * F * 4096 + (size_t)2 * nstages * R * kXchgStride * 4 + (size_t)8 * 4 * nstages + 256;
 }
 
-template <int F>
-cudaError_t launch_fused(int S, int nclusters, int nstages, cudaStream_t st, const float *K, int64_t ld, int n,
-                         const FsRowTile *tiles, int ntiles, const float *v, const float *a, float *u, float *rowdiff,
-                         float *partials, float eta, FsDeviceStatus *status) {
-    cudaLaunchConfig_t cfg = {};
+void fill_cluster_launch(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int S, int nclusters, size_t smem,
+                         cudaStream_t st) {
+    cfg = cudaLaunchConfig_t{};
     cfg.gridDim = dim3((unsigned)(nclusters * S));
     cfg.blockDim = dim3(kFusedThreads);
-    cfg.dynamicSmemBytes = fused_smem_bytes(F, nstages);
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)S;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fused_iteration_kernel<F>, K, ld, n, S, nclusters, nstages, tiles, ntiles, v, a, u,
-                              rowdiff, partials, eta, status);
 }
 
-template <int F>
+template <int F, int R>
+cudaError_t launch_fused(const FsFusedPlan &p, cudaStream_t st, const float *K, int64_t ld, int n, const FsRowTile *tiles,
+                         int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials, float eta,
+                         FsDeviceStatus *status) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    fill_cluster_launch(cfg, attr, p.S, p.nclusters, fused_smem_bytes(F, R, p.nstages), st);
+    return cudaLaunchKernelEx(&cfg, fused_iteration_kernel<F, R>, K, ld, n, p.S, p.nclusters, p.nstages, tiles, ntiles, v, a,
+                              u, rowdiff, partials, eta, status);
+}
+
+template <int F, int R>
 int query_clusters(int S, int nstages) {
-    const size_t smem = fused_smem_bytes(F, nstages);
-    if (cudaFuncSetAttribute(fused_iteration_kernel<F>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    const size_t smem = fused_smem_bytes(F, R, nstages);
+    if (cudaFuncSetAttribute(fused_iteration_kernel<F, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(148 * S));
-    cfg.blockDim = dim3(kFusedThreads);
-    cfg.dynamicSmemBytes = smem;
+    cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)S;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    fill_cluster_launch(cfg, attr, S, 148, smem, nullptr);
     int nc = 0;
-    if (cudaOccupancyMaxActiveClusters(&nc, fused_iteration_kernel<F>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&nc, fused_iteration_kernel<F, R>, &cfg) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -270,18 +300,19 @@ FsFusedPlan fsk_fused_plan(int64_t n, bool vec) {
     }
     if (f > 16) return p;
     const int F = f <= 2 ? 2 : f <= 4 ? 4 : f <= 8 ? 8 : 16;
-    int ns = (int)(200 * 1024 / (F * 4096));
+    const int R = F == 2 ? 8 : F == 4 ? 4 : F == 8 ? 2 : 1; // rows per stage: stages of 64 KB
+    int ns = (int)(200 * 1024 / (R * F * 4096));
     if (ns > 8) ns = 8;
     if (ns < 2) return p;
     int nc = 0;
     switch (F) {
-    case 2: nc = query_clusters<2>(S, ns); break;
-    case 4: nc = query_clusters<4>(S, ns); break;
-    case 8: nc = query_clusters<8>(S, ns); break;
-    default: nc = query_clusters<16>(S, ns); break;
+    case 2: nc = query_clusters<2, 8>(S, ns); break;
+    case 4: nc = query_clusters<4, 4>(S, ns); break;
+    case 8: nc = query_clusters<8, 2>(S, ns); break;
+    default: nc = query_clusters<16, 1>(S, ns); break;
     }
     if (nc < 1) return p;
-    p.enabled = true, p.S = S, p.F = F, p.nstages = ns, p.nclusters = nc, p.tile_rows = 32;
+    p.enabled = true, p.S = S, p.F = F, p.R = R, p.nstages = ns, p.nclusters = nc, p.tile_rows = 32;
     return p;
 }
 
@@ -291,9 +322,9 @@ cudaError_t fsk_fused_iteration(const FsFusedPlan &p, const float *K, int64_t ld
                                 int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials,
                                 float eta, FsDeviceStatus *status, cudaStream_t st) {
     switch (p.F) {
-    case 2: return launch_fused<2>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
-    case 4: return launch_fused<4>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
-    case 8: return launch_fused<8>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
-    default: return launch_fused<16>(p.S, p.nclusters, p.nstages, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
+    case 2: return launch_fused<2, 8>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
+    case 4: return launch_fused<4, 4>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
+    case 8: return launch_fused<8, 2>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
+    default: return launch_fused<16, 1>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
     }
 }

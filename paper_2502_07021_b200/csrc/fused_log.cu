@@ -311,7 +311,7 @@ FsFusedPlan fsk_fused_log_plan(int64_t n, bool vec) {
     default: nc = query_clusters<8>(S, ns); break;
     }
     if (nc < 1) return p;
-    p.enabled = true, p.S = S, p.F = F, p.nstages = ns, p.nclusters = nc, p.tile_rows = 32;
+    p.enabled = true, p.S = S, p.F = F, p.R = 1, p.nstages = ns, p.nclusters = nc, p.tile_rows = 32;
     return p;
 }
 
