@@ -45,8 +45,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (kernel name, n) -> bytes; a capture at n = 16384 is scaled by 4 for n = 32768 (traffic is proportional to n*n).
 TRAFFIC_BYTES_PER_LAUNCH = {
-    ("fused_iteration_kernel", 16384): 1.073985e9 + 4.69e6,
-    ("fused_iteration_kernel", 32768): 4 * (1.073985e9 + 4.69e6),
+    ("fused_iteration_kernel", 16384): 1.073989e9 + 4.5e6,
+    ("fused_iteration_kernel", 32768): 4 * (1.073989e9 + 4.5e6),
     ("log_row_pass_kernel", 16384): 1.074176e9 + 3.74e6,
     ("batched_tc_kernel", 8192): 272.67e6 + 4.5e6,
 }
