@@ -230,6 +230,78 @@ def time_config(fs, torch, dev, stream, w, steps=3):
             "final_row_marginal_l1_max": float(row.max()), "final_col_marginal_l1_max": float(col.max())}
 
 
+def run_sharded(args, rank, local_rank, world):
+    """Row-partitioned run (opt-in, --multi sharded): one shard of the SAME problem per GPU, one all-reduce
+    of n floats per iteration over NCCL; total work is fixed, so scaling is strong."""
+    import torch
+    from paper_2502_07021_b200 import binding as fs
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.Stream(device=dev)
+    n_total = args.n or workloads._SPECS[args.config]["n"]
+    lo, hi = fsdist.row_range(n_total, rank, world)
+    w = workloads.make(args.config, n=args.n, want_cost=False, rows=(lo, hi))
+    if w.domain != workloads.DOMAIN_SCALING or w.nbatch != 1:
+        raise RuntimeError("--multi sharded covers the single-problem scaling-domain configurations")
+    if args.iters is not None:
+        w.iters = args.iters
+    Kb = torch.from_numpy(w.K).to(dev)
+    a_loc = torch.from_numpy(w.a[lo:hi].copy()).to(dev)
+    b = torch.from_numpy(w.b).to(dev)
+    r_buf = torch.empty(w.n, dtype=torch.float32, device=dev)
+    ones_u = torch.ones(hi - lo, dtype=torch.float32, device=dev)
+    ones_v = torch.ones(w.n, dtype=torch.float32, device=dev)
+    torch.cuda.synchronize()
+    sh = fs.fs_shard_create(w.n, lo, hi - lo, Kb, w.n, fs.FS_MATRIX_KERNEL, w.eps, a_loc, b, stream)
+
+    def step():
+        fs.fs_shard_set_scalings(sh, ones_u, ones_v, stream)
+        fsdist.sharded_iterate(fs, sh, r_buf, w.iters, stream)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    stream.synchronize()
+    sampler = ClockSampler(visible_device_index(local_rank))
+    fsdist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    stream.synchronize()
+    torch.cuda.synchronize()
+    fsdist.barrier()
+    clocks = sampler.stop()
+    t_ms, _ = fsdist.aggregate(e0.elapsed_time(e1), 0.0, dev)
+    l1, _ = fs.fs_shard_row_error(sh, stream)
+    _, l1 = fsdist.aggregate(0.0, l1, dev)
+    fs.fs_shard_destroy(sh)
+    if rank != 0:
+        return
+    its = args.steps * w.iters
+    peaks, peak_kind = measured_peaks()
+    per_pass_bytes = (hi - lo) * w.n * 4
+    line = {"metric": METRIC, "value": its / (t_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": t_ms / args.steps, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": dict(config_dict(w, args, world), parallelism=f"{world} row shards of one problem, "
+                           "all-reduce of n floats per iteration (NCCL)"),
+            "gpu_launches": int(its * 5), "clocks": clocks, "e2e": None,
+            "roofline": {"bound": "hbm", "kernel": "row_pass_kernel + col_partial_kernel (per shard)",
+                         "achieved": 2 * per_pass_bytes * its / (t_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": 2 * per_pass_bytes * its / (t_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                         "peak_source": f"of {peak_kind}", "traffic": None,
+                         "note": "per-GPU rate over the whole iteration, collectives included"},
+            "cpu_baseline": None, "row_marginal_l1_before_last_iteration": l1}
+    print(json.dumps(line), flush=True)
+
+
 def run_ours(args, w, rank, local_rank, world):
     import torch
     from paper_2502_07021_b200 import binding as fs
@@ -388,6 +460,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-iters", type=int, default=1, help="--impl reference: iterations per step")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--multi", default="replicas", choices=["replicas", "sharded"],
+                    help="N > 1: independent replicas (default, weak scaling) or row shards of one problem")
     ap.add_argument("--headline-only", action="store_true", help="skip the short runs of configurations 1, 2, 3, 5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic-bytes", type=float, default=None,
@@ -405,6 +479,12 @@ def main():
         return 0
     if world > 1:
         fsdist.init()
+    if args.multi == "sharded":
+        try:
+            run_sharded(args, rank, local_rank, world)
+        finally:
+            fsdist.finalize()
+        return 0
     w = workloads.make(args.config, n=args.n, want_cost=None if args.config == 3 else False)
     if args.iters is not None:
         w.iters = args.iters

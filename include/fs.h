@@ -221,6 +221,33 @@ int fs_solve_host(int64_t n, int32_t c, const int64_t *row_offsets, const float 
 int fs_col_pass_static(const float *K_dev, int64_t ld, int64_t n, const float *u_dev, const float *b_dev,
                        float *v_dev, void *stream);
 
+/*
+ * Row-partitioned shards for several GPUs (Section 3.1: client j holds K_{I_j,:}, a_j and a copy of v;
+ * Algorithm 1 with the column sums assembled from per-client partial products, as in the appendix's 2D block
+ * baseline).  One process per GPU creates one shard for its contiguous rows [row_lo, row_lo + m) and runs,
+ * per iteration,
+ *      fs_shard_row_pass      u_I = a_I ./ (K_{I,:} v)                  local
+ *      fs_shard_col_partial   p   = (K_{I,:})^T u_I   (n floats)        local, written to r_dev_out
+ *      (all-reduce SUM of p over the shards: the caller's, e.g. torch.distributed / NCCL)
+ *      fs_shard_col_finish    v   = b ./ r                              redundantly on every shard
+ * Scaling domain only.  M_dev is the LOCAL m x n block (leading dimension ld >= n), borrowed; a_local_dev is
+ * [m], b_dev is the whole [n]; start u = v = 1.  The equal-mass condition spans all shards and is not checked
+ * here; positivity is.  fs_shard_row_error returns the local sums sum_i |d_i| and sum_i d_i^2 of the row residual
+ * d = u .* (K v) - a seen by the last row pass (add them over the shards; take the root of the second).
+ * All calls are asynchronous on `stream` except fs_shard_create, fs_shard_scalings and fs_shard_row_error,
+ * which synchronise it.
+ */
+typedef struct fs_shard fs_shard; /* opaque */
+int fs_shard_create(fs_shard **out, int64_t n, int64_t row_lo, int64_t m, const float *M_dev, int64_t ld,
+                    int matrix_kind, double eps, const float *a_local_dev, const float *b_dev, void *stream);
+int fs_shard_row_pass(fs_shard *s, void *stream);
+int fs_shard_col_partial(fs_shard *s, float *r_dev_out, void *stream);
+int fs_shard_col_finish(fs_shard *s, const float *r_total_dev, void *stream);
+int fs_shard_scalings(fs_shard *s, float *u_local_dev_out, float *v_dev_out, void *stream);
+int fs_shard_set_scalings(fs_shard *s, const float *u_local_dev, const float *v_dev, void *stream);
+int fs_shard_row_error(fs_shard *s, double *l1_out, double *sumsq_out, void *stream);
+int fs_shard_destroy(fs_shard *s);
+
 const char *fs_strerror(int code);
 
 /* Text of the last CUDA error seen by this thread's calls ("" if none). */

@@ -48,6 +48,14 @@ _SIGNATURES = {
     "fs_destroy": (_int, [_vp]),
     "fs_solve_host": (_int, [_i64, _i32, _vp, _vp, _i64, _int, _dbl, _vp, _vp, _i32, _int, _i32, _vp, _vp, _vp]),
     "fs_col_pass_static": (_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "fs_shard_create": (_int, [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp, _i64, _int, _dbl, _vp, _vp, _vp]),
+    "fs_shard_row_pass": (_int, [_vp, _vp]),
+    "fs_shard_col_partial": (_int, [_vp, _vp, _vp]),
+    "fs_shard_col_finish": (_int, [_vp, _vp, _vp]),
+    "fs_shard_scalings": (_int, [_vp, _vp, _vp, _vp]),
+    "fs_shard_set_scalings": (_int, [_vp, _vp, _vp, _vp]),
+    "fs_shard_row_error": (_int, [_vp, _vp, _vp, _vp]),
+    "fs_shard_destroy": (_int, [_vp]),
     "fs_strerror": (ctypes.c_char_p, [_int]),
     "fs_last_cuda_error": (ctypes.c_char_p, []),
 }
@@ -209,6 +217,44 @@ def fs_col_pass_static(K_dev, ld, n, u_dev, b_dev, v_dev, stream=None):
     """v = b / (K^T u) through the entry point that allocates nothing (n <= FS_STATIC_MAX_N)."""
     _check(lib().fs_col_pass_static(_dev(K_dev), ld, n, _dev(u_dev), _dev(b_dev), _dev(v_dev), _stream(stream)),
            "fs_col_pass_static")
+
+
+def fs_shard_create(n, row_lo, m, M_dev, ld, matrix_kind, eps, a_local_dev, b_dev, stream=None):
+    out = _vp()
+    _check(lib().fs_shard_create(ctypes.byref(out), n, row_lo, m, _dev(M_dev), ld, matrix_kind, float(eps),
+                                 _dev(a_local_dev), _dev(b_dev), _stream(stream)), "fs_shard_create")
+    return out
+
+
+def fs_shard_row_pass(s, stream=None):
+    _check(lib().fs_shard_row_pass(s, _stream(stream)), "fs_shard_row_pass")
+
+
+def fs_shard_col_partial(s, r_dev_out, stream=None):
+    _check(lib().fs_shard_col_partial(s, _dev(r_dev_out), _stream(stream)), "fs_shard_col_partial")
+
+
+def fs_shard_col_finish(s, r_total_dev, stream=None):
+    _check(lib().fs_shard_col_finish(s, _dev(r_total_dev), _stream(stream)), "fs_shard_col_finish")
+
+
+def fs_shard_scalings(s, u_local_dev_out, v_dev_out, stream=None):
+    _check(lib().fs_shard_scalings(s, _dev(u_local_dev_out), _dev(v_dev_out), _stream(stream)), "fs_shard_scalings")
+
+
+def fs_shard_set_scalings(s, u_local_dev, v_dev, stream=None):
+    _check(lib().fs_shard_set_scalings(s, _dev(u_local_dev), _dev(v_dev), _stream(stream)), "fs_shard_set_scalings")
+
+
+def fs_shard_row_error(s, stream=None):
+    """(sum |d|, sum d^2) of the local row residual seen by the last row pass."""
+    l1, sq = _dbl(0.0), _dbl(0.0)
+    _check(lib().fs_shard_row_error(s, ctypes.byref(l1), ctypes.byref(sq), _stream(stream)), "fs_shard_row_error")
+    return l1.value, sq.value
+
+
+def fs_shard_destroy(s):
+    _check(lib().fs_shard_destroy(s), "fs_shard_destroy")
 
 
 def fs_solve_host(n, c, row_offsets, M_host, ld, matrix_kind, eps, a_host, b_host, nbatch, domain, iters,

@@ -33,7 +33,9 @@ constexpr int64_t kFusedAutoMinN = 6144;
 constexpr int kTcMinBatch = 32;
 constexpr int kTcMinN = 512;
 
-FsPassPlan choose_plan(int64_t n, bool vec, int domain) {
+} // namespace
+
+FsPassPlan fsk_choose_plan(int64_t n, bool vec, int domain) {
     FsPassPlan p{};
     p.vec = vec;
     if (n >= 8192) {
@@ -46,6 +48,8 @@ FsPassPlan choose_plan(int64_t n, bool vec, int domain) {
     }
     return p;
 }
+
+namespace {
 
 // Row tiles of at most `h` rows that never cross a block boundary (Section 3.1: block j is the
 // unit a client owns).
@@ -122,7 +126,7 @@ void enqueue_row(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
                              st);
         launches += 1;
     } else if (s->domain == FS_DOMAIN_SCALING) {
-        fsk_row_pass(s->plan, s->mat, s->mat_ld, s->n, s->y, s->a, s->x, s->rowdiff, update, s->eta, s->status, st);
+        fsk_row_pass(s->plan, s->mat, s->mat_ld, s->n, s->n, s->y, s->a, s->x, s->rowdiff, update, s->eta, s->status, st);
         launches += fsk_pass_launches_row();
     } else {
         fsk_log_row_pass(s->plan, s->mat, s->mat_ld, s->n, s->eps, s->ys, s->a, s->loga, s->x, s->xs, s->rowdiff,
@@ -347,13 +351,13 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
     } else if (matrix_kind == FS_MATRIX_COST) {
         // set-up step: materialise the Gibbs kernel once (Section 1, K = exp(-C/eps))
         FS_CU(cudaMalloc(&s->K_owned, sizeof(float) * (size_t)n * (size_t)s->n_pad));
-        fsk_materialize_kernel(M_dev, ld, n, (float)(-1.0 / eps), s->K_owned, s->n_pad, st);
+        fsk_materialize_kernel(M_dev, ld, n, n, (float)(-1.0 / eps), s->K_owned, s->n_pad, st);
         s->mat = s->K_owned, s->mat_ld = s->n_pad;
     } else {
         s->mat = M_dev, s->mat_ld = ld;
     }
     const bool vec = (reinterpret_cast<uintptr_t>(s->mat) & 15) == 0 && (s->mat_ld & 3) == 0;
-    s->plan = choose_plan(n, vec, domain);
+    s->plan = fsk_choose_plan(n, vec, domain);
     int rc = upload_tiles(s);
     if (rc != FS_OK) return rc;
     if (nbatch == 1) {

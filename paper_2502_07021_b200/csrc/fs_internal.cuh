@@ -115,8 +115,13 @@ struct fs_solver {
 
 // ---- passes.cu ---------------------------------------------------------------------------
 // Row pass, scaling domain: q_i = sum_l K_il v_l; rowdiff_i = u_i q_i - a_i; if update u_i = a_i/q_i.
-void fsk_row_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, const float *v, const float *a,
-                  float *u, float *rowdiff, int update, float eta, FsDeviceStatus *status, cudaStream_t st);
+// K is nrows x n (nrows = n for a whole problem, fewer for a row shard).
+void fsk_row_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t nrows, const float *v,
+                  const float *a, float *u, float *rowdiff, int update, float eta, FsDeviceStatus *status,
+                  cudaStream_t st);
+void fsk_col_partial_sum(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
+                         int ntiles, const float *u, float *partials, float *r_out, cudaStream_t st);
+FsPassPlan fsk_choose_plan(int64_t n, bool vec, int domain);
 // Column pass, scaling domain, two deterministic stages.
 void fsk_col_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
                   int ntiles, const float *u, const float *b, float *v, float *partials, float *coldiff,
@@ -174,7 +179,8 @@ void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float 
                  FsDeviceStatus *status, cudaStream_t st);
 
 // ---- setup.cu ----------------------------------------------------------------------------
-void fsk_materialize_kernel(const float *C, int64_t ldc, int64_t n, float neg_inv_eps, float *K, int64_t ldk,
+// C and K are nrows x n.
+void fsk_materialize_kernel(const float *C, int64_t ldc, int64_t n, int64_t nrows, float neg_inv_eps, float *K, int64_t ldk,
                             cudaStream_t st);
 // out[p][0] = min, out[p][1] = sum (double) of x[p][0..n)
 void fsk_min_sum(const float *x, int64_t n, int nbatch, double *out, cudaStream_t st);

@@ -66,7 +66,7 @@ __device__ __forceinline__ float damped(float x_new, float x_old, float eta) {
 // Row pass, scaling domain.
 template <int L, int R, bool VEC>
 __global__ void __launch_bounds__(kThreads)
-row_pass_kernel(const float *__restrict__ K, int64_t ld, int n, const float *__restrict__ v,
+row_pass_kernel(const float *__restrict__ K, int64_t ld, int n, int nrows, const float *__restrict__ v,
                 const float *__restrict__ a, float *__restrict__ u, float *__restrict__ rowdiff, int update,
                 float eta, FsDeviceStatus *status) {
     constexpr int G = kThreads / L;
@@ -78,7 +78,7 @@ row_pass_kernel(const float *__restrict__ K, int64_t ld, int n, const float *__r
     const int row0 = (blockIdx.x * G + grp) * R;
     const float *rowp[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) rowp[r] = K + (int64_t)min(row0 + r, n - 1) * ld;
+    for (int r = 0; r < R; ++r) rowp[r] = K + (int64_t)min(row0 + r, nrows - 1) * ld;
     float acc[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) acc[r] = 0.f;
@@ -139,7 +139,7 @@ row_pass_kernel(const float *__restrict__ K, int64_t ld, int n, const float *__r
     if (threadIdx.x < G * R) {
         const int g = threadIdx.x / R, r = threadIdx.x % R;
         const int row = (blockIdx.x * G + g) * R + r;
-        if (row < n) {
+        if (row < nrows) {
             float q = 0.f;
 #pragma unroll
             for (int w = 0; w < W; ++w) q += red[g * W + w][r];
@@ -359,6 +359,17 @@ col_finish_kernel(int n, int64_t n_pad, int ntiles, const float *__restrict__ pa
     }
 }
 
+// Sum of the tile partials alone, in tile order.
+__global__ void __launch_bounds__(kThreads)
+sum_partials_kernel(int n, int64_t n_pad, int ntiles, const float *__restrict__ partials, float *__restrict__ r_out) {
+    const int l = blockIdx.x * kThreads + threadIdx.x;
+    if (l >= n) return;
+    float r = 0.f;
+#pragma unroll 8
+    for (int t = 0; t < ntiles; ++t) r += partials[(int64_t)t * n_pad + l];
+    r_out[l] = r;
+}
+
 // Log-domain column pass stage 1: per (tile, column) running (max, sum) pair.
 // partials: plane 0 = maxima [ntiles][n_pad], plane 1 = sums.
 template <int TX, int TY, bool VEC>
@@ -478,7 +489,7 @@ log_col_finish_kernel(int n, int64_t n_pad, int ntiles, float s2, double eps, co
 #define FS_ROW_DISPATCH(KERNEL, ...)                                                              \
     do {                                                                                          \
         const int G_ = kThreads / p.row_L;                                                        \
-        const unsigned grid_ = (unsigned)((n + (int64_t)G_ * p.row_R - 1) / ((int64_t)G_ * p.row_R)); \
+        const unsigned grid_ = (unsigned)((nrows + (int64_t)G_ * p.row_R - 1) / ((int64_t)G_ * p.row_R)); \
         FS_ROW_CASE(KERNEL, 32, 1, __VA_ARGS__)                                                   \
         FS_ROW_CASE(KERNEL, 32, 2, __VA_ARGS__)                                                   \
         FS_ROW_CASE(KERNEL, 64, 1, __VA_ARGS__)                                                   \
@@ -505,9 +516,10 @@ log_col_finish_kernel(int n, int64_t n_pad, int ntiles, float s2, double eps, co
         }                                                                                         \
     } while (0)
 
-void fsk_row_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, const float *v, const float *a,
-                  float *u, float *rowdiff, int update, float eta, FsDeviceStatus *status, cudaStream_t st) {
-    FS_ROW_DISPATCH(row_pass_kernel, K, ld, (int)n, v, a, u, rowdiff, update, eta, status);
+void fsk_row_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t nrows, const float *v,
+                  const float *a, float *u, float *rowdiff, int update, float eta, FsDeviceStatus *status,
+                  cudaStream_t st) {
+    FS_ROW_DISPATCH(row_pass_kernel, K, ld, (int)n, (int)nrows, v, a, u, rowdiff, update, eta, status);
 }
 
 void fsk_col_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
@@ -522,6 +534,7 @@ void fsk_log_row_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n
                       const float *a, const float *loga, float *f, float *xs, float *rowdiff, int update,
                       FsDeviceStatus *status, cudaStream_t st) {
     const float s2 = (float)(1.4426950408889634 / eps);
+    const int64_t nrows = n;
     FS_ROW_DISPATCH(log_row_pass_kernel, C, ld, (int)n, s2, eps, ys, a, loga, f, xs, rowdiff, update, status);
 }
 
@@ -533,6 +546,14 @@ void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n
     FS_COL_DISPATCH(log_col_partial_kernel, C, ld, (int)n, n_pad, s2, tiles, ntiles, nstrips, xs, partials);
     log_col_finish_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>(
         (int)n, n_pad, ntiles, s2, eps, partials, b, logb, g, ys, coldiff, update, status);
+}
+
+// Stage 1 followed by a plain sum of the tile partials: r_out[l] = sum over the given row tiles of
+// K_il u_i, without the divide (the shard's contribution to K^T u).
+void fsk_col_partial_sum(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
+                         int ntiles, const float *u, float *partials, float *r_out, cudaStream_t st) {
+    FS_COL_DISPATCH(col_partial_kernel, K, ld, (int)n, n_pad, tiles, nstrips, u, partials);
+    sum_partials_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>((int)n, n_pad, ntiles, partials, r_out);
 }
 
 void fsk_col_finish(int64_t n, int64_t n_pad, int ntiles, const float *partials, const float *b, float *v,

@@ -170,13 +170,13 @@ unsigned grid_for(int64_t count) {
 
 } // namespace
 
-void fsk_materialize_kernel(const float *C, int64_t ldc, int64_t n, float neg_inv_eps, float *K, int64_t ldk,
-                            cudaStream_t st) {
+void fsk_materialize_kernel(const float *C, int64_t ldc, int64_t n, int64_t nrows, float neg_inv_eps, float *K,
+                            int64_t ldk, cudaStream_t st) {
     int64_t gx = (n + kThreads - 1) / kThreads;
     if (gx > 64) gx = 64;
     // grid.y is limited to 65535 rows per launch
-    for (int64_t r0 = 0; r0 < n; r0 += 65535) {
-        const int64_t rows = n - r0 < 65535 ? n - r0 : 65535;
+    for (int64_t r0 = 0; r0 < nrows; r0 += 65535) {
+        const int64_t rows = nrows - r0 < 65535 ? nrows - r0 : 65535;
         dim3 grid((unsigned)gx, (unsigned)rows);
         materialize_kernel<<<grid, kThreads, 0, st>>>(C + r0 * ldc, ldc, (int)n, neg_inv_eps, K + r0 * ldk, ldk);
     }

@@ -1,0 +1,187 @@
+// Row-partitioned solver shard: the piece of the path one GPU runs when the kernel matrix is split
+// by rows over several devices, as in Section 3.1 (client j holds K_{I_j,:}, a_j and a copy of v).
+//
+// One iteration on G shards is
+//   row pass        u_I = a_I ./ (K_{I,:} v)                      local, no communication
+//   column partial  p   = (K_{I,:})^T u_I   (all n columns)       local
+//   all-reduce      r   = sum over shards of p                     n floats per iteration
+//   finish          v   = b ./ r                                   every shard, redundantly
+// which is the strict row-partition form (the column sums are assembled from per-shard partial
+// products, as in the appendix's 2D block baseline); for any K it gives the iterates of Algorithm 1 up
+// to the association of the column sums.  The all-reduce is the caller's (torch.distributed / NCCL in
+// paper_2502_07021_b200/distributed.py); this file only provides the three device steps.
+#include <math.h>
+
+#include <vector>
+
+#include "fs_internal.cuh"
+
+struct fs_shard {
+    int64_t n = 0, m = 0, row_lo = 0, ld = 0, n_pad = 0;
+    double eps = 0;
+    const float *mat = nullptr;
+    int64_t mat_ld = 0;
+    float *K_owned = nullptr;
+    float *a = nullptr, *b = nullptr, *u = nullptr, *v = nullptr, *rowdiff = nullptr, *coldiff = nullptr;
+    float *partials = nullptr;
+    FsRowTile *tiles_dev = nullptr;
+    int ntiles = 0;
+    double *err_dev = nullptr;
+    FsDeviceStatus *status = nullptr;
+    FsPassPlan plan{};
+    float eta = 1.f;
+};
+
+namespace {
+
+#define FS_SH(call)                                   \
+    do {                                              \
+        cudaError_t e_ = (call);                      \
+        if (e_ != cudaSuccess) {                      \
+            cudaGetLastError();                       \
+            return FS_ERR_CUDA;                       \
+        }                                             \
+    } while (0)
+
+void shard_free(fs_shard *s) {
+    if (!s) return;
+    cudaFree(s->K_owned), cudaFree(s->a), cudaFree(s->b), cudaFree(s->u), cudaFree(s->v), cudaFree(s->rowdiff);
+    cudaFree(s->coldiff), cudaFree(s->partials), cudaFree(s->tiles_dev), cudaFree(s->err_dev), cudaFree(s->status);
+    delete s;
+}
+
+} // namespace
+
+extern "C" {
+
+int fs_shard_create(fs_shard **out, int64_t n, int64_t row_lo, int64_t m, const float *M_dev, int64_t ld, int matrix_kind,
+                    double eps, const float *a_local_dev, const float *b_dev, void *stream) {
+    if (!out) return FS_ERR_NULL;
+    *out = nullptr;
+    if (!M_dev || !a_local_dev || !b_dev) return FS_ERR_NULL;
+    if (n < 1 || n > (int64_t(1) << 30) || m < 1 || row_lo < 0 || row_lo + m > n || ld < n) return FS_ERR_BAD_N;
+    if (matrix_kind != FS_MATRIX_KERNEL && matrix_kind != FS_MATRIX_COST) return FS_ERR_BAD_N;
+    if (!(eps > 0.0) || !isfinite(eps)) return FS_ERR_BAD_EPS;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    // positivity of the local marginals (the equal-mass condition spans all shards and is the caller's)
+    {
+        double *scan = nullptr;
+        FS_SH(cudaMalloc(&scan, sizeof(double) * 4));
+        fsk_min_sum(a_local_dev, m, 1, scan, st);
+        fsk_min_sum(b_dev, n, 1, scan + 2, st);
+        double h[4];
+        cudaError_t e = cudaMemcpyAsync(h, scan, sizeof(h), cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        cudaFree(scan);
+        if (e != cudaSuccess) return FS_ERR_CUDA;
+        if (!(h[0] > 0.0) || !(h[2] > 0.0) || !isfinite(h[1]) || !isfinite(h[3])) return FS_ERR_NONPOSITIVE_MARGINAL;
+    }
+
+    fs_shard *s = new fs_shard();
+    struct Guard {
+        fs_shard *s;
+        ~Guard() { shard_free(s); }
+    } guard{s};
+    s->n = n, s->m = m, s->row_lo = row_lo, s->ld = ld, s->eps = eps;
+    s->n_pad = (n + 3) & ~int64_t(3);
+    FS_SH(cudaMalloc(&s->a, sizeof(float) * m));
+    FS_SH(cudaMalloc(&s->u, sizeof(float) * m));
+    FS_SH(cudaMalloc(&s->rowdiff, sizeof(float) * m));
+    FS_SH(cudaMalloc(&s->b, sizeof(float) * n));
+    FS_SH(cudaMalloc(&s->v, sizeof(float) * n));
+    FS_SH(cudaMalloc(&s->coldiff, sizeof(float) * n));
+    FS_SH(cudaMalloc(&s->err_dev, sizeof(double) * 2));
+    FS_SH(cudaMalloc(&s->status, sizeof(FsDeviceStatus)));
+    FS_SH(cudaMemsetAsync(s->status, 0, sizeof(FsDeviceStatus), st));
+    FS_SH(cudaMemsetAsync(s->rowdiff, 0, sizeof(float) * m, st));
+    FS_SH(cudaMemcpyAsync(s->a, a_local_dev, sizeof(float) * m, cudaMemcpyDeviceToDevice, st));
+    FS_SH(cudaMemcpyAsync(s->b, b_dev, sizeof(float) * n, cudaMemcpyDeviceToDevice, st));
+    fsk_fill(s->u, m, 1.f, st);
+    fsk_fill(s->v, n, 1.f, st);
+    if (matrix_kind == FS_MATRIX_COST) {
+        FS_SH(cudaMalloc(&s->K_owned, sizeof(float) * (size_t)m * (size_t)s->n_pad));
+        fsk_materialize_kernel(M_dev, ld, n, m, (float)(-1.0 / eps), s->K_owned, s->n_pad, st);
+        s->mat = s->K_owned, s->mat_ld = s->n_pad;
+    } else {
+        s->mat = M_dev, s->mat_ld = ld;
+    }
+    const bool vec = (reinterpret_cast<uintptr_t>(s->mat) & 15) == 0 && (s->mat_ld & 3) == 0;
+    s->plan = fsk_choose_plan(n, vec, FS_DOMAIN_SCALING);
+    std::vector<FsRowTile> tiles;
+    for (int64_t r = 0; r < m; r += s->plan.col_tile_rows)
+        tiles.push_back(FsRowTile{(int32_t)r, (int32_t)(r + s->plan.col_tile_rows < m ? r + s->plan.col_tile_rows : m)});
+    s->ntiles = (int)tiles.size();
+    FS_SH(cudaMalloc(&s->tiles_dev, sizeof(FsRowTile) * tiles.size()));
+    FS_SH(cudaMemcpyAsync(s->tiles_dev, tiles.data(), sizeof(FsRowTile) * tiles.size(), cudaMemcpyHostToDevice, st));
+    FS_SH(cudaMalloc(&s->partials, sizeof(float) * tiles.size() * (size_t)s->n_pad));
+    FS_SH(cudaStreamSynchronize(st));
+    FS_SH(cudaGetLastError());
+    guard.s = nullptr;
+    *out = s;
+    return FS_OK;
+}
+
+int fs_shard_row_pass(fs_shard *s, void *stream) {
+    if (!s) return FS_ERR_NULL;
+    fsk_row_pass(s->plan, s->mat, s->mat_ld, s->n, s->m, s->v, s->a, s->u, s->rowdiff, 1, s->eta, s->status,
+                 (cudaStream_t)stream);
+    FS_SH(cudaGetLastError());
+    return FS_OK;
+}
+
+int fs_shard_col_partial(fs_shard *s, float *r_dev_out, void *stream) {
+    if (!s || !r_dev_out) return FS_ERR_NULL;
+    fsk_col_partial_sum(s->plan, s->mat, s->mat_ld, s->n, s->n_pad, s->tiles_dev, s->ntiles, s->u, s->partials, r_dev_out,
+                        (cudaStream_t)stream);
+    FS_SH(cudaGetLastError());
+    return FS_OK;
+}
+
+int fs_shard_col_finish(fs_shard *s, const float *r_total_dev, void *stream) {
+    if (!s || !r_total_dev) return FS_ERR_NULL;
+    // stage 2 over a single "partial" row: the residual v .* r - b and v = b ./ r
+    fsk_col_finish(s->n, s->n, 1, r_total_dev, s->b, s->v, s->coldiff, 1, s->eta, s->status, (cudaStream_t)stream);
+    FS_SH(cudaGetLastError());
+    return FS_OK;
+}
+
+int fs_shard_scalings(fs_shard *s, float *u_local_dev_out, float *v_dev_out, void *stream) {
+    if (!s) return FS_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (u_local_dev_out) FS_SH(cudaMemcpyAsync(u_local_dev_out, s->u, sizeof(float) * s->m, cudaMemcpyDeviceToDevice, st));
+    if (v_dev_out) FS_SH(cudaMemcpyAsync(v_dev_out, s->v, sizeof(float) * s->n, cudaMemcpyDeviceToDevice, st));
+    FsDeviceStatus h{};
+    FS_SH(cudaMemcpyAsync(&h, s->status, sizeof(h), cudaMemcpyDeviceToHost, st));
+    FS_SH(cudaStreamSynchronize(st));
+    return h.nonfinite ? FS_ERR_NONFINITE : FS_OK;
+}
+
+int fs_shard_set_scalings(fs_shard *s, const float *u_local_dev, const float *v_dev, void *stream) {
+    if (!s) return FS_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (u_local_dev) FS_SH(cudaMemcpyAsync(s->u, u_local_dev, sizeof(float) * s->m, cudaMemcpyDeviceToDevice, st));
+    if (v_dev) FS_SH(cudaMemcpyAsync(s->v, v_dev, sizeof(float) * s->n, cudaMemcpyDeviceToDevice, st));
+    return FS_OK;
+}
+
+int fs_shard_row_error(fs_shard *s, double *l1_out, double *sumsq_out, void *stream) {
+    if (!s) return FS_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    fsk_diff_norms(s->rowdiff, s->m, 1, s->err_dev, st);
+    double h[2];
+    FS_SH(cudaMemcpyAsync(h, s->err_dev, sizeof(h), cudaMemcpyDeviceToHost, st));
+    FS_SH(cudaStreamSynchronize(st));
+    if (l1_out) *l1_out = h[0];
+    if (sumsq_out) *sumsq_out = h[1];
+    return FS_OK;
+}
+
+int fs_shard_destroy(fs_shard *s) {
+    if (!s) return FS_ERR_NULL;
+    cudaDeviceSynchronize();
+    shard_free(s);
+    return FS_OK;
+}
+
+} // extern "C"

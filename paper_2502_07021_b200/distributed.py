@@ -1,8 +1,8 @@
 """Host-side plumbing for running the hot path on N GPUs of one node, one process per GPU.
 
 The single-GPU path has no inter-GPU exchange, so N processes are N independent solvers, each on
-its own problem instance (weak scaling: per-GPU work is fixed).  What the processes share is
-only measurement: a barrier on both sides of the timed region, the MAX over ranks of the
+its own problem instance (weak scaling: per-GPU work is fixed).  What the processes share there
+is only measurement: a barrier on both sides of the timed region, the MAX over ranks of the
 device-timed duration, and the SUM of the units of work.  This module holds exactly that, on top
 of ``torch.distributed`` (NCCL on GPUs, gloo on CPU for the tests).
 """
@@ -59,6 +59,35 @@ def shard_problems(total: int, rank: int, world: int):
     base, extra = divmod(total, world)
     lo = rank * base + min(rank, extra)
     return lo, lo + base + (1 if rank < extra else 0)
+
+
+def row_range(n: int, rank: int, world: int):
+    """Contiguous rows [lo, hi) of an n x n problem owned by `rank` (the paper's index set I_rank)."""
+    return shard_problems(n, rank, world)
+
+
+def sharded_iterate(api, shard, r_buf, k: int, stream=None, group=None):
+    """k Sinkhorn iterations of a row-partitioned problem, one shard per process (Algorithm 1 with the
+    column sums assembled by an all-reduce of the per-shard partial products, n floats per iteration).
+
+    `api` provides fs_shard_row_pass / fs_shard_col_partial / fs_shard_col_finish (the ctypes binding on
+    GPUs); `r_buf` is a length-n float32 tensor on the shard's device that receives the partial and then
+    the reduced column sums.  The collective is torch.distributed's (NCCL on GPUs, gloo on CPU); with a
+    CUDA `stream` the three steps and the collective are ordered on that stream.
+    """
+    import contextlib
+
+    import torch
+    import torch.distributed as dist
+    use_dist = dist.is_available() and dist.is_initialized()
+    ctx = torch.cuda.stream(stream) if (stream is not None and r_buf.is_cuda) else contextlib.nullcontext()
+    with ctx:
+        for _ in range(k):
+            api.fs_shard_row_pass(shard, stream)
+            api.fs_shard_col_partial(shard, r_buf, stream)
+            if use_dist:
+                dist.all_reduce(r_buf, op=dist.ReduceOp.SUM, group=group)
+            api.fs_shard_col_finish(shard, r_buf, stream)
 
 
 def finalize():

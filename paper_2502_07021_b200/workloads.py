@@ -99,9 +99,10 @@ def _sqdist_rows(X: np.ndarray, Y: np.ndarray, ynorm: np.ndarray, r0: int, r1: i
     return d
 
 
-def cost_and_kernel(X, Y, eps, normalize, want_cost=True, want_kernel=True, chunk=2048):
+def cost_and_kernel(X, Y, eps, normalize, want_cost=True, want_kernel=True, chunk=2048, rows=None):
     """Dense C_il = max(0, |x_i|^2 + |y_l|^2 - 2 x_i.y_l) (optionally divided by its maximum)
-    and K = exp(-C/eps), built in fp64 row chunks and rounded once to fp32."""
+    and K = exp(-C/eps), built in fp64 row chunks and rounded once to fp32.  With rows = (lo, hi) only
+    that row block is materialised (the maximum is still taken over the whole matrix)."""
     n = X.shape[0]
     ynorm = (Y * Y).sum(1)
     scale = 1.0
@@ -110,26 +111,28 @@ def cost_and_kernel(X, Y, eps, normalize, want_cost=True, want_kernel=True, chun
         cmax = max(cmax, float(_sqdist_rows(X, Y, ynorm, r0, min(n, r0 + chunk)).max()))
     if normalize:
         scale = 1.0 / cmax
-    C32 = np.empty((n, n), dtype=np.float32) if want_cost else None
-    K32 = np.empty((n, n), dtype=np.float32) if want_kernel else None
-    for r0 in range(0, n, chunk):
-        r1 = min(n, r0 + chunk)
+    lo, hi = (0, n) if rows is None else rows
+    C32 = np.empty((hi - lo, n), dtype=np.float32) if want_cost else None
+    K32 = np.empty((hi - lo, n), dtype=np.float32) if want_kernel else None
+    for r0 in range(lo, hi, chunk):
+        r1 = min(hi, r0 + chunk)
         d = _sqdist_rows(X, Y, ynorm, r0, r1)
         if normalize:
             d *= scale
         if want_cost:
-            C32[r0:r1] = d
+            C32[r0 - lo:r1 - lo] = d
         if want_kernel:
             d *= -1.0 / eps
             np.exp(d, out=d)
-            K32[r0:r1] = d
+            K32[r0 - lo:r1 - lo] = d
     return C32, K32, dict(raw_cost_max=cmax, cost_scale=scale)
 
 
 def make(cfg: int, n: int | None = None, nbatch: int | None = None, c: int | None = None,
-         offsets=None, want_cost: bool | None = None, want_kernel: bool | None = None) -> Workload:
+         offsets=None, want_cost: bool | None = None, want_kernel: bool | None = None, rows=None) -> Workload:
     """Build configuration `cfg` (1..5).  `n`, `nbatch`, `c`/`offsets` override the stated sizes
-    to get a smaller or differently partitioned copy of the same recipe."""
+    to get a smaller or differently partitioned copy of the same recipe.  `rows = (lo, hi)` materialises
+    only that row block of the matrices (a, b stay whole): what one shard of a row partition holds."""
     s = dict(_SPECS[cfg])
     n = int(s["n"] if n is None else n)
     nb = int(s["nbatch"] if nbatch is None else nbatch)
@@ -147,7 +150,7 @@ def make(cfg: int, n: int | None = None, nbatch: int | None = None, c: int | Non
         want_cost = True if log else n <= 8192
     if want_kernel is None:
         want_kernel = not log
-    C32, K32, meta = cost_and_kernel(X, Y, s["eps"], s["normalize"], want_cost, want_kernel)
+    C32, K32, meta = cost_and_kernel(X, Y, s["eps"], s["normalize"], want_cost, want_kernel, rows=rows)
 
     def marg(seed):
         if s["marg"] == "uniform":

@@ -71,3 +71,49 @@ def test_reference_arm_runs_only_on_rank_zero():
                           "--gpus", "2", "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True,
                          timeout=300)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_two_gloo_ranks_run_the_sharded_iteration(tmp_path):
+    """`sharded_iterate` with two gloo ranks: each rank owns a row block and a stand-in for the shard API
+    written with numpy (row pass, column partial, finish); the all-reduce is torch.distributed's.  The
+    stacked result must be the row-partition iterates of the oracle."""
+    script = tmp_path / "shard_rank.py"
+    script.write_text(textwrap.dedent(f"""
+        import sys
+        sys.path.insert(0, {ROOT!r})
+        import numpy as np, torch
+        import oracle
+        from paper_2502_07021_b200 import distributed as fsdist, workloads
+
+        class NumpyShardApi:
+            # host stand-in with the call pattern of the C ABI's fs_shard_* steps
+            def fs_shard_row_pass(self, s, stream=None):
+                s["u"] = s["a"] / (s["K"] @ s["v"])
+            def fs_shard_col_partial(self, s, r_buf, stream=None):
+                r_buf.copy_(torch.from_numpy((s["K"].T @ s["u"]).astype(np.float32)))
+            def fs_shard_col_finish(self, s, r_buf, stream=None):
+                s["v"] = s["b"] / r_buf.numpy().astype(np.float64)
+
+        rank, local_rank, world = fsdist.init(backend="gloo")
+        w = workloads.make(2, n=96)
+        lo, hi = fsdist.row_range(w.n, rank, world)
+        shard = dict(K=w.K[lo:hi].astype(np.float64), a=w.a[lo:hi].astype(np.float64), b=w.b.astype(np.float64),
+                     u=np.ones(hi - lo), v=np.ones(w.n))
+        r_buf = torch.empty(w.n, dtype=torch.float32)
+        fsdist.sharded_iterate(NumpyShardApi(), shard, r_buf, 6)
+        uo, vo = oracle.sinkhorn_rowpartition(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, [0, 48, 96], 6)
+        ok = np.max(np.abs(shard["u"] - uo[lo:hi]) / uo[lo:hi]) < 1e-5 and np.max(np.abs(shard["v"] - vo) / vo) < 1e-5
+        print(f"RESULT {{rank}} {{lo}} {{hi}} {{int(ok)}}", flush=True)
+        fsdist.finalize()
+    """))
+    port = free_port()
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port), OMP_NUM_THREADS="2")
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.STDOUT, text=True))
+    outs = [p.communicate(timeout=180)[0] for p in procs]
+    assert all(p.returncode == 0 for p in procs), outs
+    results = sorted(line.split()[1:] for out in outs for line in out.splitlines() if line.startswith("RESULT"))
+    assert results == [["0", "0", "48", "1"], ["1", "48", "96", "1"]]
