@@ -402,6 +402,20 @@ def run_ours(args, w, rank, local_rank, world):
                 others[f"config{cfg}"] = time_config(fs, torch, dev, stream, workloads.make(cfg, want_cost=None if cfg == 3 else False))
             except Exception as exc:  # a failure here must not lose the headline line
                 others[f"config{cfg}"] = {"error": repr(exc)}
+        # the one table the paper prints for this path (Table 1: 15 iterations, n = 5000; 1 problem 0.32 s,
+        # 500 targets vectorised 0.31 s, on an unnamed GPU in fp64): same shapes, our recipe, fp32
+        try:
+            t1 = {}
+            for label, nb in (("one_problem", 1), ("vectorized_500", 500)):
+                wt = workloads.make(5, n=5000, nbatch=nb, want_cost=False)
+                wt.iters = 15
+                r = time_config(fs, torch, dev, stream, wt, steps=5)
+                t1[label] = {"seconds_for_15_iterations": 15 * r["us_per_iteration"] * 1e-6,
+                             "paper_seconds": 0.32 if nb == 1 else 0.31,
+                             "final_row_marginal_l1_max": r["final_row_marginal_l1_max"]}
+            others["paper_table1_n5000"] = t1
+        except Exception as exc:
+            others["paper_table1_n5000"] = {"error": repr(exc)}
 
     # end-to-end through the host-buffer entry point
     e2e = None
@@ -419,16 +433,21 @@ def run_ours(args, w, rank, local_rank, world):
         fs.fs_solve_host(w.n, w.c, w.offsets, pin_M, w.n, w.kind, w.eps, pin_a, pin_b, w.nbatch, w.domain, w.iters,
                          out_u, out_v)  # warm-up
         fsdist.barrier()
-        t0 = time.perf_counter()
+        step_ms = []
         for _ in range(e2e_steps):
+            t0 = time.perf_counter()
             fs.fs_solve_host(w.n, w.c, w.offsets, pin_M, w.n, w.kind, w.eps, pin_a, pin_b, w.nbatch, w.domain,
                              w.iters, out_u, out_v)
-        dt_ms = (time.perf_counter() - t0) * 1e3
+            step_ms.append((time.perf_counter() - t0) * 1e3)
+        # the host is shared: the PCIe copy of one step can take several times longer than that of the next,
+        # so the reported rate uses the median step; the spread is reported beside it
+        dt_ms = statistics.median(step_ms) * e2e_steps
         dt_ms, its = fsdist.aggregate(dt_ms, e2e_steps * w.iters, dev)
         h2d = w.n * w.n * 4 + 2 * w.a.size * 4
         d2h = 2 * w.a.size * 4 + 8 * w.nbatch
         e2e = {"value": its / (dt_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "steps": e2e_steps, "ms_per_step": dt_ms / e2e_steps,
+               "steps": e2e_steps, "ms_per_step": dt_ms / e2e_steps, "ms_per_step_min": min(step_ms),
+               "ms_per_step_max": max(step_ms), "statistic": "median step",
                "note": "fs_solve_host: device allocation, H2D of the matrix and marginals from pinned memory, "
                        "all iterations, marginal error, D2H of the scalings, free -- every step"}
     if h is not None:
@@ -457,7 +476,7 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="workload 1..5 (4 = the n=32768 headline)")
     ap.add_argument("--n", type=int, default=None, help="override n (scaled-down copy of the recipe)")
     ap.add_argument("--iters", type=int, default=None, help="override the iterations per step (profiling runs)")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--ref-iters", type=int, default=1, help="--impl reference: iterations per step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--multi", default="replicas", choices=["replicas", "sharded"],
