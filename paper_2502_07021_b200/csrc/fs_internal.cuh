@@ -1,6 +1,13 @@
 // Internal declarations shared by the translation units of libfs_b200.so.
-// Kernels live in passes.cu (single-problem scaling and log passes), batched.cu (shared-K
-// passes) and setup.cu (one-off and O(n) helpers); fs_api.cu owns the handle and the C ABI.
+//   fs_api.cu          handle, validation, iteration driver (graphs), result calls: the C ABI
+//   passes.cu          single-problem row / column passes, scaling and log domain (two-pass path)
+//   fused.cu           single-read fused iteration, scaling domain (clusters, bulk copies, DSMEM)
+//   fused_log.cu       the same for the log domain (opt-in)
+//   resident.cu        K-resident persistent kernel for small n
+//   batched_tc.cu      shared-K batched passes on tcgen05 tensor cores;  batched.cu  fp32 FMA engine
+//   shard.cu           row-partitioned shards for several GPUs (fs_shard_*)
+//   col_pass_static.cu column half-step without any allocation
+//   setup.cu           one-off and O(n) helpers;  cluster_ptx.cuh  PTX wrappers of the cluster kernels
 #pragma once
 
 #include <cuda_runtime.h>
