@@ -217,6 +217,20 @@ def test_fused_log_is_reproducible_and_traces():
         assert l1[k] == pytest.approx(e["row_l1"], rel=2e-3, abs=1e-6)
 
 
+@pytest.mark.slow
+def test_fused_clusters_of_four_beyond_n_32768():
+    """Rows longer than 32768 columns are split over clusters of four CTAs (S = 4); this is the only
+    size class that takes that path, so it gets a (slow) case of its own: n = 36864, three iterations."""
+    w = workloads.make(4, n=36864, want_cost=False)
+    with GpuSolver(w.K, KK, w.eps, w.a, w.b, w.offsets, SC) as g:
+        before = fs.fs_launch_count(g.h)
+        g.iterate(3)
+        assert fs.fs_launch_count(g.h) - before == 6           # fused kernel + stage 2 per iteration
+        x, y = g.scalings()
+    u, v = oracle.sinkhorn_scaling(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, 3)
+    assert rel_err(x, u) <= TOL_UV and rel_err(y, v) <= TOL_UV
+
+
 def test_fused_is_reproducible_and_traces():
     w = workloads.make(4, n=4096)
     runs = []
