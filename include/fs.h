@@ -248,6 +248,17 @@ int fs_shard_set_scalings(fs_shard *s, const float *u_local_dev, const float *v_
 int fs_shard_row_error(fs_shard *s, double *l1_out, double *sumsq_out, void *stream);
 int fs_shard_destroy(fs_shard *s);
 
+/*
+ * fs_selftest_bounded_wait -- exercises the bounded wait that every kernel of this library uses when it waits
+ * on an mbarrier (asynchronous copies, tensor-core commits, exchanges between the CTAs of a cluster): a probe
+ * kernel waits at most `poll_limit` polls (1 .. 2^20) on a barrier that is completed only if `arrive` is
+ * non-zero.  *timed_out (HOST) receives 1 when the wait gave up, 0 when it was satisfied.  The kernel always
+ * returns normally; the CUDA context stays usable.  In the solver kernels the same expiry raises a status
+ * flag that the next result call reports as FS_ERR_TIMEOUT.  (Failure-detection self-test; no counterpart in
+ * the paper, which assumes no failures.)  Synchronises `stream`.
+ */
+int fs_selftest_bounded_wait(int32_t poll_limit, int32_t arrive, int32_t *timed_out, void *stream);
+
 const char *fs_strerror(int code);
 
 /* Text of the last CUDA error seen by this thread's calls ("" if none). */

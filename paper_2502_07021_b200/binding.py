@@ -56,6 +56,7 @@ _SIGNATURES = {
     "fs_shard_set_scalings": (_int, [_vp, _vp, _vp, _vp]),
     "fs_shard_row_error": (_int, [_vp, _vp, _vp, _vp]),
     "fs_shard_destroy": (_int, [_vp]),
+    "fs_selftest_bounded_wait": (_int, [_i32, _i32, ctypes.POINTER(_i32), _vp]),
     "fs_strerror": (ctypes.c_char_p, [_int]),
     "fs_last_cuda_error": (ctypes.c_char_p, []),
 }
@@ -255,6 +256,14 @@ def fs_shard_row_error(s, stream=None):
 
 def fs_shard_destroy(s):
     _check(lib().fs_shard_destroy(s), "fs_shard_destroy")
+
+
+def fs_selftest_bounded_wait(poll_limit, arrive, stream=None):
+    """True when the probe kernel's bounded wait ran out."""
+    out = _i32(-1)
+    _check(lib().fs_selftest_bounded_wait(poll_limit, 1 if arrive else 0, ctypes.byref(out), _stream(stream)),
+           "fs_selftest_bounded_wait")
+    return out.value == 1
 
 
 def fs_solve_host(n, c, row_offsets, M_host, ld, matrix_kind, eps, a_host, b_host, nbatch, domain, iters,

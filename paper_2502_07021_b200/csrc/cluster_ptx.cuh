@@ -32,13 +32,15 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+// Bounded wait: gives up after `limit` polls and returns false (the caller raises the status flag).
+__device__ __forceinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, uint32_t limit) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (it > 64) __nanosleep(40);
     }
     return false;
 }
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) { return mbar_wait_limited(bar, parity, kSpinLimit); }
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait_cluster(bar, parity)) return true;

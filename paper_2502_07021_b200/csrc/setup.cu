@@ -5,6 +5,7 @@
 // All reductions use a fixed order (no atomics), so every reported number is reproducible.
 #include <math.h>
 
+#include "cluster_ptx.cuh"
 #include "fs_internal.cuh"
 
 namespace {
@@ -163,6 +164,21 @@ __global__ void __launch_bounds__(kThreads) sum_rows_kernel(const double *__rest
     if (threadIdx.x == 0) out[blockIdx.x] = t;
 }
 
+// Self-test of the bounded wait used by the cluster and tensor-core kernels: one thread waits on an
+// mbarrier that is completed only when `arrive` is set; when the poll limit runs out the kernel records
+// it and returns normally, so the context stays usable.
+__global__ void bounded_wait_probe_kernel(uint32_t limit, int arrive, int *timed_out) {
+    __shared__ __align__(8) uint64_t bar;
+    const uint32_t b = fsptx::smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        fsptx::mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && arrive) fsptx::mbar_arrive(b);
+    if (threadIdx.x == 32) *timed_out = fsptx::mbar_wait_limited(b, 0, limit) ? 0 : 1;
+}
+
 unsigned grid_for(int64_t count) {
     int64_t g = (count + kThreads - 1) / kThreads;
     return (unsigned)(g < 1 ? 1 : (g > 148 * 16 ? 148 * 16 : g));
@@ -208,4 +224,24 @@ void fsk_transport_cost(int domain, const float *mat, int64_t ld, const float *C
     dim3 grid((unsigned)((n + 7) / 8), (unsigned)nbatch);
     cost_rows_kernel<<<grid, kThreads, 0, st>>>(domain, mat, ld, C, ldc, (int)n, x, y, s2, rowsum_scratch);
     sum_rows_kernel<<<nbatch, kThreads, 0, st>>>(rowsum_scratch, n, cost_dev);
+}
+
+extern "C" int fs_selftest_bounded_wait(int32_t poll_limit, int32_t arrive, int32_t *timed_out, void *stream) {
+    if (!timed_out) return FS_ERR_NULL;
+    if (poll_limit < 1 || poll_limit > (1 << 20)) return FS_ERR_BAD_N;
+    cudaStream_t st = (cudaStream_t)stream;
+    int *flag = nullptr;
+    if (cudaMalloc(&flag, sizeof(int)) != cudaSuccess) return FS_ERR_CUDA;
+    cudaMemsetAsync(flag, 0xff, sizeof(int), st);
+    bounded_wait_probe_kernel<<<1, 64, 0, st>>>((uint32_t)poll_limit, arrive, flag);
+    int h = -1;
+    cudaError_t e = cudaMemcpyAsync(&h, flag, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(flag);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return FS_ERR_CUDA;
+    }
+    *timed_out = h;
+    return FS_OK;
 }

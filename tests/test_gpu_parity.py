@@ -552,6 +552,17 @@ def test_nonfinite_is_flagged():
         assert ei.value.code == fs.FS_ERR_NONFINITE
 
 
+def test_bounded_wait_gives_up_and_the_context_survives():
+    """Failure detection without a fault: a wait that nothing satisfies runs out after its poll limit, the
+    kernel returns, the host reads the status, and the library keeps working afterwards."""
+    assert fs.fs_selftest_bounded_wait(2000, arrive=False) is True
+    assert fs.fs_selftest_bounded_wait(2000, arrive=True) is False
+    w = workloads.make(1, n=64)
+    x, y = run(w, 3)
+    u, v = oracle.sinkhorn_scaling(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, 3)
+    assert rel_err(x, u) <= TOL_UV and rel_err(y, v) <= TOL_UV
+
+
 def test_create_rejects_bad_marginals():
     import torch
     n = 32
