@@ -11,8 +11,9 @@
 // The product keeps three of the four cross terms, hi*hi + hi*lo + lo*hi, accumulated in fp32
 // in tensor memory; the dropped lo*lo term is <= 2^-18 relative.  K is constant over the
 // iterations, so its split is made once at set-up and costs exactly the bytes of the fp32 matrix
-// (2 + 2 bytes per entry); the small operand (the scalings) is re-split by the epilogue that
-// produces it.  Both passes use the same K-major kernel: the column pass reads a transposed
+// (2 + 2 bytes per entry) and is stored tile by tile, each 128 x 64 tile in 16 KB of consecutive
+// bytes, so that a TMA box is one contiguous read; the small operand (the scalings) is re-split into
+// the same tiled layout by the epilogue that produces it.  Both passes use the same K-major kernel: the column pass reads a transposed
 // split copy of K made at set-up.
 //
 // Kernel: one CTA per (128-row tile of the output, split of the contraction range).  Warp 0
@@ -112,6 +113,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
     for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
 }
 
+// Operand matrices live in HBM tile by tile: the 128 x 64 bf16 tile (row tile t, k-block kb) occupies
+// 16 KB of consecutive bytes, so that one TMA box is one contiguous read instead of 128 segments of 128
+// bytes from rows that are kilobytes apart.  Element (r, c) of a matrix with `kblocks` k-blocks per row:
+__host__ __device__ __forceinline__ int64_t tiled_index(int64_t r, int64_t c, int kblocks) {
+    return (((r / BM) * kblocks + c / BK) * BM + r % BM) * BK + c % BK;
+}
+
 // Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes with the 128-byte
 // swizzle: 8-row groups 1024 bytes apart (stride byte offset), descriptor version 1.
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
@@ -174,11 +182,11 @@ batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_const
                 const uint32_t full = bars + 8 * s;
                 const uint32_t dst = base + s * STAGE_BYTES;
                 mbar_expect_tx(full, STAGE_BYTES);
-                const int x = (kb0 + it) * BK;
-                tma_load_2d(&tmA_hi, dst, full, x, mtile * BM);
-                tma_load_2d(&tmA_lo, dst + TILE_BYTES, full, x, mtile * BM);
-                tma_load_2d(&tmB_hi, dst + 2 * TILE_BYTES, full, x, ntile * BN);
-                tma_load_2d(&tmB_lo, dst + 3 * TILE_BYTES, full, x, ntile * BN);
+                const int ya = (mtile * kblocks + kb0 + it) * BM, yb = (ntile * kblocks + kb0 + it) * BN;
+                tma_load_2d(&tmA_hi, dst, full, 0, ya);
+                tma_load_2d(&tmA_lo, dst + TILE_BYTES, full, 0, ya);
+                tma_load_2d(&tmB_hi, dst + 2 * TILE_BYTES, full, 0, yb);
+                tma_load_2d(&tmB_lo, dst + 3 * TILE_BYTES, full, 0, yb);
             }
         }
     } else if (warp == 1) {
@@ -263,7 +271,7 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bflo
 
 // blockIdx.x = (ntile * mtiles + mtile) * 16 + slice: 1024 outputs per CTA, 4 consecutive rows per thread.
 __global__ void __launch_bounds__(256)
-batched_tc_finish_kernel(const float *__restrict__ partials, int ksplit, int n, int nbatch, int64_t ldb, int mtiles,
+batched_tc_finish_kernel(const float *__restrict__ partials, int ksplit, int n, int nbatch, int kblocks, int mtiles,
                          const float *__restrict__ marg, float *__restrict__ out, float *__restrict__ diff,
                          __nv_bfloat16 *__restrict__ op_hi, __nv_bfloat16 *__restrict__ op_lo, int update, float eta,
                          FsDeviceStatus *status) {
@@ -291,8 +299,8 @@ batched_tc_finish_kernel(const float *__restrict__ partials, int ksplit, int n, 
             out[idx] = nv;
             __nv_bfloat16 hi, lo;
             split_bf16(nv, hi, lo);
-            op_hi[(int64_t)gp * ldb + gi + j] = hi;
-            op_lo[(int64_t)gp * ldb + gi + j] = lo;
+            op_hi[tiled_index(gp, gi + j, kblocks)] = hi;
+            op_lo[tiled_index(gp, gi + j, kblocks)] = lo;
             if (!(nv > 0.f) || isinf(nv)) status->nonfinite = 1;
         }
     }
@@ -302,7 +310,7 @@ batched_tc_finish_kernel(const float *__restrict__ partials, int ksplit, int n, 
 // hi/lo split of the n x n fp32 matrix, written both as stored and transposed (32 x 32 tiles
 // through shared memory so that both writes are coalesced).
 __global__ void __launch_bounds__(256)
-split_matrix_kernel(const float *__restrict__ K, int64_t ld, int n, int64_t ldb, __nv_bfloat16 *__restrict__ hi,
+split_matrix_kernel(const float *__restrict__ K, int64_t ld, int n, int kblocks, __nv_bfloat16 *__restrict__ hi,
                     __nv_bfloat16 *__restrict__ lo, __nv_bfloat16 *__restrict__ thi, __nv_bfloat16 *__restrict__ tlo) {
     __shared__ float tile[32][33];
     const int tx = threadIdx.x % 32, ty = threadIdx.x / 32; // 32 x 8
@@ -314,8 +322,8 @@ split_matrix_kernel(const float *__restrict__ K, int64_t ld, int n, int64_t ldb,
             v = K[(int64_t)r * ld + c];
             __nv_bfloat16 h, l;
             split_bf16(v, h, l);
-            hi[(int64_t)r * ldb + c] = h;
-            lo[(int64_t)r * ldb + c] = l;
+            hi[tiled_index(r, c, kblocks)] = h;
+            lo[tiled_index(r, c, kblocks)] = l;
         }
         tile[j][tx] = v;
     }
@@ -325,20 +333,20 @@ split_matrix_kernel(const float *__restrict__ K, int64_t ld, int n, int64_t ldb,
         if (r < n && c < n) {
             __nv_bfloat16 h, l;
             split_bf16(tile[tx][j], h, l);
-            thi[(int64_t)r * ldb + c] = h;
-            tlo[(int64_t)r * ldb + c] = l;
+            thi[tiled_index(r, c, kblocks)] = h;
+            tlo[tiled_index(r, c, kblocks)] = l;
         }
     }
 }
 
-__global__ void split_vectors_kernel(const float *__restrict__ x, int n, int nbatch, int64_t ldb,
+__global__ void split_vectors_kernel(const float *__restrict__ x, int n, int nbatch, int kblocks,
                                      __nv_bfloat16 *__restrict__ hi, __nv_bfloat16 *__restrict__ lo) {
     const int p = blockIdx.y;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
         __nv_bfloat16 h, l;
         split_bf16(x[(int64_t)p * n + i], h, l);
-        hi[(int64_t)p * ldb + i] = h;
-        lo[(int64_t)p * ldb + i] = l;
+        hi[tiled_index(p, i, kblocks)] = h;
+        lo[tiled_index(p, i, kblocks)] = l;
     }
 }
 
@@ -359,12 +367,13 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// rows x cols bf16 matrix, row pitch ldb elements; box = 64 columns x 128 rows, 128-byte swizzle
-bool make_map(CUtensorMap *map, const __nv_bfloat16 *ptr, int64_t rows, int64_t cols, int64_t ldb) {
+// tiled bf16 matrix of rows x cols elements seen as a (rows * cols / 64) x 64 array of 128-byte rows: tile
+// (t, kb) is rows [(t * kblocks + kb) * 128, +128); box = 64 columns x 128 rows, 128-byte swizzle
+bool make_map(CUtensorMap *map, const __nv_bfloat16 *ptr, int64_t rows, int64_t cols) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)ldb * 2};
+    cuuint64_t dims[2] = {(cuuint64_t)BK, (cuuint64_t)(rows * cols / BK)};
+    cuuint64_t strides[1] = {(cuuint64_t)BK * 2};
     cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16 *>(ptr), dims, strides, box, estr,
@@ -409,13 +418,13 @@ void *fsk_tc_create(const float *K, int64_t ld, int64_t n, int nbatch, cudaStrea
     ok = ok && cudaMalloc(&t->partials, part_bytes) == cudaSuccess;
     if (ok) {
         dim3 grid((unsigned)((n + 31) / 32), (unsigned)((n + 31) / 32));
-        split_matrix_kernel<<<grid, 256, 0, st>>>(K, ld, (int)n, t->ldb, t->K_hi, t->K_lo, t->Kt_hi, t->Kt_lo);
+        split_matrix_kernel<<<grid, 256, 0, st>>>(K, ld, (int)n, t->kblocks, t->K_hi, t->K_lo, t->Kt_hi, t->Kt_lo);
         ok = cudaGetLastError() == cudaSuccess;
     }
-    ok = ok && make_map(&t->tmK_hi, t->K_hi, t->rows_pad, t->ldb, t->ldb) && make_map(&t->tmK_lo, t->K_lo, t->rows_pad, t->ldb, t->ldb) &&
-         make_map(&t->tmKt_hi, t->Kt_hi, t->rows_pad, t->ldb, t->ldb) && make_map(&t->tmKt_lo, t->Kt_lo, t->rows_pad, t->ldb, t->ldb) &&
-         make_map(&t->tmU_hi, t->U_hi, t->nb_pad, t->ldb, t->ldb) && make_map(&t->tmU_lo, t->U_lo, t->nb_pad, t->ldb, t->ldb) &&
-         make_map(&t->tmV_hi, t->V_hi, t->nb_pad, t->ldb, t->ldb) && make_map(&t->tmV_lo, t->V_lo, t->nb_pad, t->ldb, t->ldb);
+    ok = ok && make_map(&t->tmK_hi, t->K_hi, t->rows_pad, t->ldb) && make_map(&t->tmK_lo, t->K_lo, t->rows_pad, t->ldb) &&
+         make_map(&t->tmKt_hi, t->Kt_hi, t->rows_pad, t->ldb) && make_map(&t->tmKt_lo, t->Kt_lo, t->rows_pad, t->ldb) &&
+         make_map(&t->tmU_hi, t->U_hi, t->nb_pad, t->ldb) && make_map(&t->tmU_lo, t->U_lo, t->nb_pad, t->ldb) &&
+         make_map(&t->tmV_hi, t->V_hi, t->nb_pad, t->ldb) && make_map(&t->tmV_lo, t->V_lo, t->nb_pad, t->ldb);
     ok = ok && cudaFuncSetAttribute(batched_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
@@ -429,8 +438,8 @@ void *fsk_tc_create(const float *K, int64_t ld, int64_t n, int nbatch, cudaStrea
 void fsk_tc_refresh(void *tc, const float *u, const float *v, cudaStream_t st) {
     TcState *t = static_cast<TcState *>(tc);
     dim3 grid((unsigned)((t->n + 255) / 256 > 64 ? 64 : (t->n + 255) / 256), (unsigned)t->nbatch);
-    if (u) split_vectors_kernel<<<grid, 256, 0, st>>>(u, (int)t->n, t->nbatch, t->ldb, t->U_hi, t->U_lo);
-    if (v) split_vectors_kernel<<<grid, 256, 0, st>>>(v, (int)t->n, t->nbatch, t->ldb, t->V_hi, t->V_lo);
+    if (u) split_vectors_kernel<<<grid, 256, 0, st>>>(u, (int)t->n, t->nbatch, t->kblocks, t->U_hi, t->U_lo);
+    if (v) split_vectors_kernel<<<grid, 256, 0, st>>>(v, (int)t->n, t->nbatch, t->kblocks, t->V_hi, t->V_lo);
 }
 
 // One batched pass on the tensor-core engine; two launches.
@@ -444,7 +453,7 @@ void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float 
     else
         batched_tc_kernel<<<grid, kTcThreads, SMEM_BYTES, st>>>(t->tmKt_hi, t->tmKt_lo, t->tmU_hi, t->tmU_lo, t->partials,
                                                               t->kblocks, t->ksplit, status);
-    batched_tc_finish_kernel<<<(unsigned)(t->mtiles * t->ntiles * 16), 256, 0, st>>>(t->partials, t->ksplit, (int)t->n, t->nbatch, t->ldb, t->mtiles, marg, out, diff,
+    batched_tc_finish_kernel<<<(unsigned)(t->mtiles * t->ntiles * 16), 256, 0, st>>>(t->partials, t->ksplit, (int)t->n, t->nbatch, t->kblocks, t->mtiles, marg, out, diff,
                                                    transposed ? t->V_hi : t->U_hi, transposed ? t->V_lo : t->U_lo, update, eta,
                                                    status);
 }
