@@ -47,8 +47,8 @@ FALLBACK_HBM_GBS = 6650.0
 TRAFFIC_BYTES_PER_LAUNCH = {
     ("fused_iteration_kernel", 16384): 1.073989e9 + 4.5e6,
     ("fused_iteration_kernel", 32768): 4 * (1.073989e9 + 4.5e6),
-    ("log_row_pass_kernel", 16384): 1.074176e9 + 3.74e6,
-    ("batched_tc_kernel", 8192): 272.67e6 + 4.5e6,
+    ("log_row_pass_kernel", 16384): 1.074043e9 + 3.39e6,
+    ("batched_tc_kernel", 8192): 272.67e6 + 3.86e6,
 }
 
 
