@@ -76,9 +76,14 @@ enum {
                                aligned matrix, n a multiple of 4): 0 = never, 1 = automatic (default: scaling domain with
                                n >= 6144; the log-domain variant is slower than the two passes and is opt-in),
                                2 = whenever it applies (FS_ERR_UNSUPPORTED if it does not) */
-    FS_OPT_RESIDENT = 6     /* K-resident persistent kernel for small n (scaling domain, one problem, K fits the shared
+    FS_OPT_RESIDENT = 6,    /* K-resident persistent kernel for small n (scaling domain, one problem, K fits the shared
                                memory of one cluster: n <= ~590 with 8 CTAs, ~720 with 16; used by fs_iterate when no
                                error trace is set): 0 = never, 1 = automatic (default) */
+    FS_OPT_PERSISTENT = 7   /* grid-persistent kernel for mid-size n (scaling domain, one problem, 16-byte aligned matrix,
+                               n a multiple of 4, above the K-resident limit and n <= 5120): fs_iterate without an error
+                               trace runs all its iterations in one cooperative launch that reads K once per iteration.
+                               0 = never, 1 = automatic (default), 2 = whenever it
+                               applies (FS_ERR_UNSUPPORTED if it does not) */
 };
 
 /*

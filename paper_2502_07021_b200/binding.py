@@ -19,7 +19,7 @@ FS_ERR_NULL, FS_ERR_BAD_N, FS_ERR_BAD_OFFSETS, FS_ERR_BAD_EPS = -1, -2, -3, -4
 FS_ERR_NONPOSITIVE_MARGINAL, FS_ERR_MASS_MISMATCH, FS_ERR_DOMAIN = -5, -6, -7
 FS_ERR_CUDA, FS_ERR_NONFINITE, FS_ERR_UNSUPPORTED, FS_ERR_TOO_LARGE, FS_ERR_TIMEOUT = -8, -9, -10, -11, -12
 FS_STATIC_MAX_N = 16384
-FS_OPT_USE_GRAPH, FS_OPT_BATCH_ENGINE, FS_OPT_ROW_SHAPE, FS_OPT_COL_SHAPE, FS_OPT_FUSED, FS_OPT_RESIDENT = 1, 2, 3, 4, 5, 6
+FS_OPT_USE_GRAPH, FS_OPT_BATCH_ENGINE, FS_OPT_ROW_SHAPE, FS_OPT_COL_SHAPE, FS_OPT_FUSED, FS_OPT_RESIDENT, FS_OPT_PERSISTENT = 1, 2, 3, 4, 5, 6, 7
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libfs_b200.so")
 

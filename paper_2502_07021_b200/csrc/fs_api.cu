@@ -30,6 +30,7 @@ constexpr double kLog2e = 1.4426950408889634;
 constexpr int kGraphChunk = 64;
 constexpr int kTraceCap = 1 << 16;
 constexpr int64_t kFusedAutoMinN = 6144;
+constexpr int64_t kPersistentAutoMaxN = 5120; // K of at most 105 MB: inside the 126 MB L2
 constexpr int kTcMinBatch = 32;
 constexpr int kTcMinN = 512;
 
@@ -89,6 +90,7 @@ void destroy_solver(fs_solver *s) {
     free_dev(s->tiles_dev);
     free_dev(s->fused_tiles_dev);
     free_dev(s->fused_partials);
+    free_dev(s->persistent_scratch);
     free_dev(s->offsets_dev);
     free_dev(s->block_err);
     free_dev(s->err_out);
@@ -374,6 +376,10 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
         }
     }
     if (domain == FS_DOMAIN_SCALING && nbatch == 1) s->resident = fsk_resident_plan(n);
+    if (domain == FS_DOMAIN_SCALING && nbatch == 1 && !s->resident.enabled) {
+        s->persistent = fsk_persistent_plan(n, vec);
+        if (s->persistent.enabled) FS_CU(cudaMalloc(&s->persistent_scratch, fsk_persistent_scratch_bytes(s->persistent, n)));
+    }
     // batched problems: tensor-core engine when the batch is wide enough to fill its 128-problem tiles
     if (nbatch >= kTcMinBatch && n >= kTcMinN) s->tc = fsk_tc_create(s->mat, s->mat_ld, n, nbatch, st);
     rc = set_initial_state(s, st);
@@ -422,6 +428,11 @@ int fs_set_option(fs_solver *s, int option, int64_t value) {
     case FS_OPT_RESIDENT:
         if (value < 0 || value > 1) return FS_ERR_BAD_N;
         s->resident_mode = (int)value;
+        return FS_OK;
+    case FS_OPT_PERSISTENT:
+        if (value < 0 || value > 2) return FS_ERR_BAD_N;
+        if (value == 2 && !s->persistent.enabled) return FS_ERR_UNSUPPORTED;
+        s->persistent_mode = (int)value;
         return FS_OK;
     case FS_OPT_ROW_SHAPE: {
         const int L = (int)(value / 1000), R = (int)(value % 1000);
@@ -476,6 +487,16 @@ int fs_iterate(fs_solver *s, int32_t k, void *stream) {
     if (k > 0 && s->resident.enabled && s->resident_mode != 0 && ce == 0) {
         FS_CU(fsk_resident_iterate(s->resident, s->mat, s->mat_ld, s->n, k, s->a, s->b, s->x, s->y, s->rowdiff, s->coldiff,
                                    s->eta, s->status, st));
+        s->launches += 1;
+        s->iter_done += k;
+        return FS_OK;
+    }
+    // mid-size problems without an error trace: all k iterations in one cooperative launch that reads K once
+    // per iteration (automatic while K fits the L2 cache)
+    if (k > 0 && s->persistent.enabled && ce == 0 &&
+        (s->persistent_mode == 2 || (s->persistent_mode == 1 && s->n <= kPersistentAutoMaxN))) {
+        FS_CU(fsk_persistent_iterate(s->persistent, s->mat, s->mat_ld, s->n, k, s->a, s->b, s->x, s->y, s->rowdiff,
+                                     s->coldiff, s->eta, s->persistent_scratch, s->status, st));
         s->launches += 1;
         s->iter_done += k;
         return FS_OK;

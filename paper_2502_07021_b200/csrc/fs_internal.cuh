@@ -4,6 +4,7 @@
 //   fused.cu           single-read fused iteration, scaling domain (clusters, bulk copies, DSMEM)
 //   fused_log.cu       the same for the log domain (opt-in)
 //   resident.cu        K-resident persistent kernel for small n
+//   persistent.cu      grid-persistent single-read iterations for mid-size n (cooperative launch)
 //   batched_tc.cu      shared-K batched passes on tcgen05 tensor cores;  batched.cu  fp32 FMA engine
 //   shard.cu           row-partitioned shards for several GPUs (fs_shard_*)
 //   col_pass_static.cu column half-step without any allocation
@@ -51,6 +52,15 @@ struct FsResidentPlan {
     bool enabled;
     int S;             // CTAs in the one cluster that holds K
     int m;             // rows (and owned columns) per CTA
+    size_t smem_bytes; // dynamic shared memory per CTA
+};
+
+// Configuration of the grid-persistent kernel (persistent.cu) for mid-size n.
+struct FsPersistentPlan {
+    bool enabled;
+    int G;             // CTAs = row slices (one per SM)
+    int kmax;          // 128-bit column groups per thread
+    int res_rows;      // rows per CTA kept in shared memory
     size_t smem_bytes; // dynamic shared memory per CTA
 };
 
@@ -104,6 +114,9 @@ struct fs_solver {
     int batch_engine = 0;
     FsResidentPlan resident{};
     int resident_mode = 1;                  // 0 = never, 1 = automatic
+    FsPersistentPlan persistent{};
+    int persistent_mode = 1;                // 0 = never, 1 = automatic, 2 = whenever it applies
+    void *persistent_scratch = nullptr;
     float eta = 1.f;                        // relaxation of the scaling updates (1 = plain Sinkhorn)
 
     // batched tensor-core path
@@ -162,6 +175,13 @@ FsResidentPlan fsk_resident_plan(int64_t n);
 cudaError_t fsk_resident_iterate(const FsResidentPlan &p, const float *K, int64_t ld, int64_t n, int iters, const float *a,
                                  const float *b, float *u, float *v, float *rowdiff, float *coldiff, float eta,
                                  FsDeviceStatus *status, cudaStream_t st);
+
+// ---- persistent.cu -----------------------------------------------------------------------
+FsPersistentPlan fsk_persistent_plan(int64_t n, bool vec);
+size_t fsk_persistent_scratch_bytes(const FsPersistentPlan &p, int64_t n);
+cudaError_t fsk_persistent_iterate(const FsPersistentPlan &p, const float *K, int64_t ld, int64_t n, int iters,
+                                   const float *a, const float *b, float *u, float *v, float *rowdiff, float *coldiff,
+                                   float eta, void *scratch, FsDeviceStatus *status, cudaStream_t st);
 
 // ---- fused_log.cu ------------------------------------------------------------------------
 FsFusedPlan fsk_fused_log_plan(int64_t n, bool vec);

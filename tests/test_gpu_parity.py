@@ -489,6 +489,53 @@ def test_resident_kernel_small_problems(n):
     assert abs(res[1][2] - res[0][2]) < 1e-6
 
 
+@pytest.mark.parametrize("cfg,n", [(1, 772), (1, 1024), (2, 1500), (2, 2048), (2, 3000), (2, 4096), (4, 5120)])
+def test_persistent_kernel_mid_size_problems(cfg, n):
+    """The grid-persistent kernel (one cooperative launch runs all iterations, one read of K per iteration,
+    grid barriers between the phases) against the oracle and the two-pass graph path, with unequal blocks."""
+    w = workloads.make(cfg, n=n)
+    off = some_offsets(n, 11 * n)
+    res = {}
+    for mode in (0, 2):
+        with GpuSolver(w.K, KK, w.eps, w.a, w.b, off, SC) as g:
+            fs.fs_set_option(g.h, fs.FS_OPT_PERSISTENT, mode)
+            fs.fs_set_option(g.h, fs.FS_OPT_FUSED, 0)
+            before = fs.fs_launch_count(g.h)
+            g.iterate(4)
+            g.iterate(6)
+            launches = fs.fs_launch_count(g.h) - before
+            assert launches == (30 if mode == 0 else 2), (mode, launches)
+            res[mode] = g.scalings() + tuple(e[0] for e in g.errors(1))
+    u, v = oracle.sinkhorn_scaling(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, 10)
+    for mode in (0, 2):
+        assert rel_err(res[mode][0], u) <= TOL_UV and rel_err(res[mode][1], v) <= TOL_UV
+    assert rel_err(res[2][0], res[0][0]) < 1e-5 and rel_err(res[2][1], res[0][1]) < 1e-5
+    assert abs(res[2][2] - res[0][2]) < 1e-6
+
+
+def test_persistent_kernel_is_reproducible_damped_and_flags_nonfinite():
+    w = workloads.make(2, n=2048)
+    runs = []
+    for _ in range(2):
+        with GpuSolver(w.K, KK, w.eps, w.a, w.b, w.offsets, SC) as g:
+            g.iterate(25)
+            runs.append(g.scalings())
+    assert np.array_equal(runs[0][0], runs[1][0]) and np.array_equal(runs[0][1], runs[1][1])
+    with GpuSolver(w.K, KK, w.eps, w.a, w.b, w.offsets, SC) as g:
+        fs.fs_set_damping(g.h, 0.5)
+        g.iterate(10)
+        ud, vd = g.scalings()
+    uo, vo = oracle.sinkhorn_damped(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, 0.5, 10)
+    assert rel_err(ud, uo) <= TOL_UV and rel_err(vd, vo) <= TOL_UV
+    K = w.K.copy()
+    K[100, :] = 0.0
+    with GpuSolver(K, KK, w.eps, w.a, w.b, w.offsets, SC) as g:
+        g.iterate(2)
+        with pytest.raises(fs.FsError) as ei:
+            g.scalings()
+        assert ei.value.code == fs.FS_ERR_NONFINITE
+
+
 def test_resident_kernel_converges_and_flags_nonfinite():
     w = workloads.make(1)
     check_converged(w, w.iters, w.C)                          # default path for n = 512 is the resident kernel
