@@ -62,7 +62,6 @@ __device__ __forceinline__ bool grid_barrier(unsigned *counter, unsigned target,
             if (it > 16) __nanosleep(32);
         }
         if (it == kPollLimit) *flag_s = 1;
-        __threadfence();
     }
     __syncthreads();
     return *flag_s == 0;
@@ -79,7 +78,7 @@ struct Params {
     FsDeviceStatus *status;
 };
 
-// Shared memory (floats): Kres[res_rows][n] | red[2][RG][kWarps] | us[2][mmax] | as[mmax] | flag
+// Shared memory (floats): Kres[res_rows][n] | red[2][RG][kWarps] | us[2][mmax] | as[mmax] | vsl[4 gmax] | bsl[4 gmax] | flag
 template <int KMAX>
 __global__ void __launch_bounds__(kThreads, 1) persistent_iterations_kernel(const Params P) {
     extern __shared__ __align__(16) float smem[];
@@ -92,7 +91,10 @@ __global__ void __launch_bounds__(kThreads, 1) persistent_iterations_kernel(cons
     float *red = Kres + (size_t)P.res_rows * n;
     float *us = red + 2 * RG * kWarps;
     float *as = us + 2 * mmax;
-    int *flag_s = reinterpret_cast<int *>(as + mmax);
+    const int gmax = (n4 + G - 1) / G + 1; // 128-bit column groups of a phase-B slice, at most
+    float *vsl = as + mmax;
+    float *bsl = vsl + 4 * gmax;
+    int *flag_s = reinterpret_cast<int *>(bsl + 4 * gmax);
 
     // one-off: resident rows, local a and u
     for (int i = warp; i < res; i += kWarps) {
@@ -113,28 +115,31 @@ __global__ void __launch_bounds__(kThreads, 1) persistent_iterations_kernel(cons
     bool bad = false, ok = true;
     unsigned barriers = 0;
 
-    // loads the K values of group g (rows 4g..4g+3 of this CTA) for this thread's columns
+    // streamed groups are first_streamed .. ngroups-1; S(k) = k-th of them
+    const int ns = ngroups - first_streamed;
+    // loads the K values of streamed group g (rows 4g..4g+3 of this CTA) for this thread's columns
     auto load_group = [&](float4 (&kv)[RG][KMAX], int g) {
 #pragma unroll
         for (int r = 0; r < RG; ++r) {
             const int i = min(g * RG + r, m - 1); // rows past the end repeat the last row; their u is 0
-            if (g < first_streamed) {
-                const float4 *src = reinterpret_cast<const float4 *>(Kres + (size_t)i * n);
+            const float *src = P.K + (int64_t)(row0 + i) * P.ld;
 #pragma unroll
-                for (int k = 0; k < KMAX; ++k) {
-                    const int c = t + k * kThreads;
-                    kv[r][k] = c < n4 ? src[c] : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-            } else {
-                const float *src = P.K + (int64_t)(row0 + i) * P.ld;
-#pragma unroll
-                for (int k = 0; k < KMAX; ++k) {
-                    const int c = t + k * kThreads;
-                    kv[r][k] = c < n4 ? ldg_stream(src + 4 * c) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
+            for (int k = 0; k < KMAX; ++k) {
+                const int c = t + k * kThreads;
+                kv[r][k] = c < n4 ? ldg_stream(src + 4 * c) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
     };
+    // this CTA's slice of v and b for phase B (columns 4 g0 .. 4 g1 - 1)
+    for (int l = t; l < 4 * (g1 - g0); l += kThreads) {
+        vsl[l] = P.v[4 * g0 + l];
+        bsl[l] = P.b[4 * g0 + l];
+    }
+    // the first two streamed groups are in flight before v is needed: K does not depend on the iterates
+    float4 kvA[RG][KMAX], kvB[RG][KMAX];
+    if (ns > 0) load_group(kvA, first_streamed);
+    if (ns > 1) load_group(kvB, first_streamed + 1);
+    __syncthreads();
 
     for (int it = 0; it < P.iters && ok; ++it) {
         const bool last = it == P.iters - 1;
@@ -148,21 +153,16 @@ __global__ void __launch_bounds__(kThreads, 1) persistent_iterations_kernel(cons
             vreg[k] = c < n4 ? __ldcg(reinterpret_cast<const float4 *>(P.v) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
             p[k] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        // ---- phase A: streamed groups first (their loads are prefetched one group ahead), then resident
-        auto process = [&](const float4 (&kv)[RG][KMAX], int g, int slot) {
-            float d[RG];
-#pragma unroll
-            for (int r = 0; r < RG; ++r) {
-                d[r] = 0.f;
-#pragma unroll
-                for (int k = 0; k < KMAX; ++k) d[r] = dot4(kv[r][k], vreg[k], d[r]);
-            }
+        int slot = 0;
+        // block reduction of the RG partial dot products in a fixed order, then the u update; un[r] = new
+        // u of row 4g + r (0 for rows past the end)
+        auto reduce_and_update = [&](float (&d)[RG], int g, float (&un)[RG]) {
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
 #pragma unroll
                 for (int r = 0; r < RG; ++r) d[r] += __shfl_xor_sync(0xffffffffu, d[r], off);
             }
-            float *rb = red + (size_t)(slot & 1) * RG * kWarps;
+            float *rb = red + (size_t)(slot++ & 1) * RG * kWarps;
             if (lane == 0) {
 #pragma unroll
                 for (int r = 0; r < RG; ++r) rb[r * kWarps + warp] = d[r];
@@ -174,32 +174,79 @@ __global__ void __launch_bounds__(kThreads, 1) persistent_iterations_kernel(cons
                 const float4 w1 = reinterpret_cast<const float4 *>(rb + r * kWarps)[1];
                 const float q = ((w0.x + w0.y) + (w0.z + w0.w)) + ((w1.x + w1.y) + (w1.z + w1.w));
                 const int i = g * RG + r;
-                float un = 0.f;
+                un[r] = 0.f;
                 if (i < m) {
                     const float uo = uo_s[i], ai = as[i];
-                    un = damped(ai / q, uo, P.eta);
+                    un[r] = damped(ai / q, uo, P.eta);
                     if (t == r) {
-                        un_s[i] = un;
+                        un_s[i] = un[r];
                         if (last) P.rowdiff[row0 + i] = fmaf(uo, q, -ai);
-                        if (!(un > 0.f) || isinf(un)) bad = true;
+                        if (!(un[r] > 0.f) || isinf(un[r])) bad = true;
                     }
                 }
-#pragma unroll
-                for (int k = 0; k < KMAX; ++k) axpy4(p[k], kv[r][k], un);
             }
         };
-        {
-            float4 kvA[RG][KMAX], kvB[RG][KMAX];
-            int slot = 0;
-            // processing order: streamed groups first_streamed..ngroups-1, then resident groups 0..first_streamed-1
-            auto group_at = [&](int s) { return s < ngroups - first_streamed ? first_streamed + s : s - (ngroups - first_streamed); };
-            if (ngroups > 0) load_group(kvA, group_at(0));
-            for (int s = 0; s < ngroups; s += 2) {
-                if (s + 1 < ngroups) load_group(kvB, group_at(s + 1));
-                process(kvA, group_at(s), slot++);
-                if (s + 2 < ngroups) load_group(kvA, group_at(s + 2));
-                if (s + 1 < ngroups) process(kvB, group_at(s + 1), slot++);
+        auto process_streamed = [&](const float4 (&kv)[RG][KMAX], int g) {
+            float d[RG], un[RG];
+#pragma unroll
+            for (int r = 0; r < RG; ++r) {
+                d[r] = 0.f;
+#pragma unroll
+                for (int k = 0; k < KMAX; ++k) d[r] = dot4(kv[r][k], vreg[k], d[r]);
             }
+            reduce_and_update(d, g, un);
+#pragma unroll
+            for (int r = 0; r < RG; ++r) {
+#pragma unroll
+                for (int k = 0; k < KMAX; ++k) axpy4(p[k], kv[r][k], un[r]);
+            }
+        };
+        // resident groups are whole (all RG rows exist) and are read from shared memory twice
+        auto process_resident = [&](int g) {
+            float d[RG], un[RG];
+            const float4 *src = reinterpret_cast<const float4 *>(Kres + (size_t)g * RG * n);
+#pragma unroll
+            for (int r = 0; r < RG; ++r) {
+                d[r] = 0.f;
+#pragma unroll
+                for (int k = 0; k < KMAX; ++k) {
+                    const int c = t + k * kThreads;
+                    if (c < n4) d[r] = dot4(src[(size_t)r * n4 + c], vreg[k], d[r]);
+                }
+            }
+            reduce_and_update(d, g, un);
+#pragma unroll
+            for (int r = 0; r < RG; ++r) {
+#pragma unroll
+                for (int k = 0; k < KMAX; ++k) {
+                    const int c = t + k * kThreads;
+                    if (c < n4) axpy4(p[k], src[(size_t)r * n4 + c], un[r]);
+                }
+            }
+        };
+        // ---- phase A.  Order: S(0), S(1) (already in flight), all resident groups (while S(2), S(3) load),
+        //      then the remaining streamed groups, each loaded two groups ahead into the buffer just freed.
+        if (ns > 0) {
+            process_streamed(kvA, first_streamed);
+            if (ns > 2) load_group(kvA, first_streamed + 2);
+        }
+        if (ns > 1) {
+            process_streamed(kvB, first_streamed + 1);
+            if (ns > 3) load_group(kvB, first_streamed + 3);
+        }
+        for (int g = 0; g < first_streamed; ++g) process_resident(g);
+        for (int k = 2; k < ns; k += 2) {
+            process_streamed(kvA, first_streamed + k);
+            if (k + 2 < ns) load_group(kvA, first_streamed + k + 2);
+            if (k + 1 < ns) {
+                process_streamed(kvB, first_streamed + k + 1);
+                if (k + 3 < ns) load_group(kvB, first_streamed + k + 3);
+            }
+        }
+        // next iteration's first two streamed groups travel during the barriers and phase B
+        if (!last) {
+            if (ns > 0) load_group(kvA, first_streamed);
+            if (ns > 1) load_group(kvB, first_streamed + 1);
         }
 #pragma unroll
         for (int k = 0; k < KMAX; ++k) {
@@ -225,9 +272,10 @@ __global__ void __launch_bounds__(kThreads, 1) persistent_iterations_kernel(cons
             }
             if (lane < 4) {
                 const float r = lane == 0 ? r4.x : lane == 1 ? r4.y : lane == 2 ? r4.z : r4.w;
-                const int l = 4 * g + lane;
-                const float vo = __ldcg(P.v + l), bl = P.b[l];
+                const int ls = 4 * (g - g0) + lane, l = 4 * g + lane;
+                const float vo = vsl[ls], bl = bsl[ls];
                 const float vn = damped(bl / r, vo, P.eta);
+                vsl[ls] = vn;
                 __stcg(P.v + l, vn);
                 if (last) P.coldiff[l] = fmaf(vo, r, -bl);
                 if (!(vn > 0.f) || isinf(vn)) bad = true;
@@ -296,7 +344,8 @@ FsPersistentPlan fsk_persistent_plan(int64_t n, bool vec) {
     p.G = (int)(n / 4 < sms ? n / 4 : sms);
     p.kmax = (int)((n / 4 + kThreads - 1) / kThreads);
     const int mmax = (int)((n + p.G - 1) / p.G);
-    const size_t fixed = sizeof(float) * (2 * RG * kWarps + 3 * (size_t)mmax) + 16;
+    const size_t gmax = (size_t)((n / 4 + p.G - 1) / p.G + 1);
+    const size_t fixed = sizeof(float) * (2 * RG * kWarps + 3 * (size_t)mmax + 8 * gmax) + 16;
     const size_t budget = 227 * 1024;
     int res = (int)((budget - fixed) / (sizeof(float) * (size_t)n));
     res = (res < mmax ? res : mmax + RG - 1) & ~(RG - 1);
