@@ -49,6 +49,8 @@ TRAFFIC_BYTES_PER_LAUNCH = {
     ("fused_iteration_kernel", 32768): 4 * (1.073989e9 + 4.5e6),
     ("log_row_pass_kernel", 16384): 1.074043e9 + 3.39e6,
     ("batched_tc_kernel", 8192): 272.67e6 + 3.86e6,
+    # captured on a 200-iteration launch; K is read from DRAM once per launch whatever the iteration count
+    ("persistent_iterations_kernel", 4096): 67.26e6 + 1.4e6,
 }
 
 
@@ -373,6 +375,16 @@ def run_ours(args, w, rank, local_rank, world):
         kernel, bytes_launch = "fused_iteration_kernel", n2
         note = ("one launch per iteration reads K once (n*n*4 bytes); the timed interval includes the "
                 "col_finish_kernel that follows it")
+    elif w.nbatch == 1 and w.domain == workloads.DOMAIN_SCALING and w.n <= 5120 and w.n % 4 == 0 and w.n >= 8:
+        # all iterations of a step in one launch of a persistent kernel; K is read from HBM once per launch
+        # and then served from shared memory (n <= ~720) or from L2 and shared memory
+        reps = 5
+        per_launch_s = timed(lambda: fs.fs_iterate(h, w.iters, stream))
+        kernel = "resident_iterations_kernel" if w.n <= 720 else "persistent_iterations_kernel"
+        bytes_launch = n2 * w.iters
+        note = ("one launch runs all %d iterations of a step; bytes = one read of K per iteration (n*n*4 each), served "
+                "from on-chip memory and L2, not HBM: the kernel is latency-bound and this fraction is not an HBM "
+                "utilisation" % w.iters)
     elif w.nbatch > 1:
         per_launch_s = timed(lambda: fs.fs_row_pass(h, stream))
         kernel, bytes_launch = "batched_tc_kernel", n2 + 4 * w.n * w.nbatch * 4
