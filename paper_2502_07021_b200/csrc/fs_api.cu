@@ -492,9 +492,9 @@ int fs_iterate(fs_solver *s, int32_t k, void *stream) {
         return FS_OK;
     }
     // mid-size problems without an error trace: all k iterations in one cooperative launch that reads K once
-    // per iteration (automatic while K fits the L2 cache)
+    // per iteration (automatic while K fits the L2 cache, unless the fused path was asked for explicitly)
     if (k > 0 && s->persistent.enabled && ce == 0 &&
-        (s->persistent_mode == 2 || (s->persistent_mode == 1 && s->n <= kPersistentAutoMaxN))) {
+        (s->persistent_mode == 2 || (s->persistent_mode == 1 && s->n <= kPersistentAutoMaxN && s->fused_mode != 2))) {
         FS_CU(fsk_persistent_iterate(s->persistent, s->mat, s->mat_ld, s->n, k, s->a, s->b, s->x, s->y, s->rowdiff,
                                      s->coldiff, s->eta, s->persistent_scratch, s->status, st));
         s->launches += 1;

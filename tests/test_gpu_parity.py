@@ -162,6 +162,8 @@ def test_fused_single_read_iteration(n, offsets):
     for mode in (0, 2):
         with GpuSolver(w.K, KK, w.eps, w.a, w.b, off, SC) as g:
             fs.fs_set_option(g.h, fs.FS_OPT_FUSED, mode)
+            if n <= 5120:
+                fs.fs_set_option(g.h, fs.FS_OPT_PERSISTENT, 0)     # mode 0 is to be the two-pass graph path
             before = fs.fs_launch_count(g.h)
             g.iterate(10)
             assert fs.fs_launch_count(g.h) - before == (30 if mode == 0 else 20)
@@ -185,6 +187,8 @@ def test_fused_single_read_iteration_log_domain(n, offsets):
     for mode in (0, 2):
         with GpuSolver(w.C, KC, w.eps, w.a, w.b, off, LG) as g:
             fs.fs_set_option(g.h, fs.FS_OPT_FUSED, mode)
+            if n <= 5120:
+                fs.fs_set_option(g.h, fs.FS_OPT_PERSISTENT, 0)     # mode 0 is to be the two-pass graph path
             before = fs.fs_launch_count(g.h)
             g.iterate(10)
             assert fs.fs_launch_count(g.h) - before == (30 if mode == 0 else 20)
