@@ -495,10 +495,15 @@ int fs_iterate(fs_solver *s, int32_t k, void *stream) {
     // per iteration (automatic while K fits the L2 cache, unless the fused path was asked for explicitly)
     if (k > 0 && s->persistent.enabled && ce == 0 &&
         (s->persistent_mode == 2 || (s->persistent_mode == 1 && s->n <= kPersistentAutoMaxN && s->fused_mode != 2))) {
-        FS_CU(fsk_persistent_iterate(s->persistent, s->mat, s->mat_ld, s->n, k, s->a, s->b, s->x, s->y, s->rowdiff,
-                                     s->coldiff, s->eta, s->persistent_scratch, s->status, st));
-        s->launches += 1;
-        s->iter_done += k;
+        // at most 2^20 iterations per launch: the grid barrier's 32-bit arrival counter must not wrap
+        for (int32_t done = 0; done < k;) {
+            const int32_t len = std::min<int32_t>(k - done, 1 << 20);
+            FS_CU(fsk_persistent_iterate(s->persistent, s->mat, s->mat_ld, s->n, len, s->a, s->b, s->x, s->y, s->rowdiff,
+                                         s->coldiff, s->eta, s->persistent_scratch, s->status, st));
+            s->launches += 1;
+            s->iter_done += len;
+            done += len;
+        }
         return FS_OK;
     }
     int64_t remaining = k;
