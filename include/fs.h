@@ -186,6 +186,12 @@ int64_t fs_iterations_done(const fs_solver *s);
 /* Number of kernel launches this handle has enqueued so far (graph replays count their nodes). */
 int64_t fs_launch_count(const fs_solver *s);
 
+/* Log domain, single-read fused path (FS_OPT_FUSED): number of iterations since creation / fs_reset whose
+ * marginals left the safe fp32 range of that path and that were therefore redone by the two-pass kernels
+ * (normally the first iteration from a cold start and none after it).  count_out: HOST.  Synchronises the
+ * stream.  The paper has no counterpart: it is a diagnostic of this implementation. */
+int fs_fused_log_fallbacks(fs_solver *s, int64_t *count_out, void *stream);
+
 int fs_destroy(fs_solver *s);
 
 /*

@@ -45,6 +45,7 @@ _SIGNATURES = {
     "fs_set_option": (_int, [_vp, _int, _i64]),
     "fs_iterations_done": (_i64, [_vp]),
     "fs_launch_count": (_i64, [_vp]),
+    "fs_fused_log_fallbacks": (_int, [_vp, ctypes.POINTER(_i64), _vp]),
     "fs_destroy": (_int, [_vp]),
     "fs_solve_host": (_int, [_i64, _i32, _vp, _vp, _i64, _int, _dbl, _vp, _vp, _i32, _int, _i32, _vp, _vp, _vp]),
     "fs_col_pass_static": (_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp]),
@@ -208,6 +209,12 @@ def fs_iterations_done(s):
 
 def fs_launch_count(s):
     return int(lib().fs_launch_count(s))
+
+
+def fs_fused_log_fallbacks(s, stream=None):
+    out = _i64(0)
+    _check(lib().fs_fused_log_fallbacks(s, ctypes.byref(out), _stream(stream)), "fs_fused_log_fallbacks")
+    return int(out.value)
 
 
 def fs_destroy(s):

@@ -90,6 +90,7 @@ void destroy_solver(fs_solver *s) {
     free_dev(s->tiles_dev);
     free_dev(s->fused_tiles_dev);
     free_dev(s->fused_partials);
+    free_dev(s->fused_log_tmp);
     free_dev(s->persistent_scratch);
     free_dev(s->offsets_dev);
     free_dev(s->block_err);
@@ -167,22 +168,37 @@ bool use_fused(const fs_solver *s) {
 }
 
 void enqueue_fused_rows(fs_solver *s, cudaStream_t st, int64_t &launches) {
-    if (s->domain == FS_DOMAIN_LOG)
-        fsk_fused_log_iteration(s->fused, s->mat, s->mat_ld, s->n, s->eps, s->fused_tiles_dev, s->fused_ntiles, s->ys, s->a,
-                                s->loga, s->x, s->xs, s->rowdiff, s->fused_partials, s->status, st);
-    else
-        fsk_fused_iteration(s->fused, s->mat, s->mat_ld, s->n, s->fused_tiles_dev, s->fused_ntiles, s->y, s->a, s->x,
-                            s->rowdiff, s->fused_partials, s->eta, s->status, st);
+    fsk_fused_iteration(s->fused, s->mat, s->mat_ld, s->n, s->fused_tiles_dev, s->fused_ntiles, s->y, s->a, s->x,
+                        s->rowdiff, s->fused_partials, s->eta, s->status, st);
     launches += 1;
 }
 
 void enqueue_fused_finish(fs_solver *s, cudaStream_t st, int64_t &launches) {
-    if (s->domain == FS_DOMAIN_LOG)
-        fsk_log_col_finish(s->n, s->n, s->fused.nclusters, s->eps, s->fused_partials, s->b, s->logb, s->y, s->ys,
-                           s->coldiff, 1, s->status, st);
-    else
-        fsk_col_finish(s->n, s->n, s->fused.nclusters, s->fused_partials, s->b, s->y, s->coldiff, 1, s->eta, s->status, st);
+    fsk_col_finish(s->n, s->n, s->fused.nclusters, s->fused_partials, s->b, s->y, s->coldiff, 1, s->eta, s->status, st);
     launches += 1;
+}
+
+void enqueue_trace(fs_solver *s, cudaStream_t st, int64_t &launches);
+
+// One log-domain iteration on the single-read path: the fused kernels write the new duals to temporaries;
+// the two-pass kernels follow as guarded launches that do nothing unless the fused iteration left the safe
+// range (then they redo it from the untouched duals); the commit kernel adopts the temporaries otherwise.
+void enqueue_fused_log_iteration(fs_solver *s, bool check, cudaStream_t st, int64_t &launches) {
+    float *tmp = s->fused_log_tmp;
+    const size_t n = (size_t)s->n;
+    const int *redo = &s->status->range;
+    fsk_fused_log_iteration(s->fused, s->mat, s->mat_ld, s->n, s->eps, s->fused_tiles_dev, s->fused_ntiles, s->xs, s->ys,
+                            s->a, s->b, tmp, tmp + n, tmp + 2 * n, tmp + 3 * n, s->rowdiff, s->coldiff, s->fused_partials,
+                            s->status, st);
+    fsk_log_row_pass(s->plan, s->mat, s->mat_ld, s->n, s->eps, s->ys, s->a, s->loga, s->x, s->xs, s->rowdiff, 1, s->status,
+                     st, redo);
+    launches += 3;
+    if (check) enqueue_trace(s, st, launches);
+    fsk_log_col_pass(s->plan, s->mat, s->mat_ld, s->n, s->n_pad, s->eps, s->tiles_dev, (int)s->tiles.size(), s->xs, s->b,
+                     s->logb, s->y, s->ys, s->partials, s->coldiff, 1, s->status, st, redo);
+    fsk_fused_log_commit(s->n, tmp, tmp + n, tmp + 2 * n, tmp + 3 * n, s->x, s->xs, s->y, s->ys, s->status,
+                         reinterpret_cast<int *>(tmp + 4 * n), st);
+    launches += 3;
 }
 
 void enqueue_trace(fs_solver *s, cudaStream_t st, int64_t &launches) {
@@ -200,9 +216,13 @@ void enqueue_range(fs_solver *s, int phase, int len, bool trace_first, bool fina
     const int ce = s->check_every;
     const bool fused = use_fused(s);
     for (int it = 0; it < len; ++it) {
+        const bool check = it == 0 ? trace_first : (ce > 0 && (phase + it) % ce == 0);
+        if (fused && s->domain == FS_DOMAIN_LOG) {
+            enqueue_fused_log_iteration(s, check, st, launches);
+            continue;
+        }
         if (fused) enqueue_fused_rows(s, st, launches);
         else enqueue_row(s, 1, st, launches);
-        const bool check = it == 0 ? trace_first : (ce > 0 && (phase + it) % ce == 0);
         if (check) enqueue_trace(s, st, launches);
         if (fused) enqueue_fused_finish(s, st, launches);
         else enqueue_col(s, 1, st, launches);
@@ -365,7 +385,7 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
     if (nbatch == 1) {
         s->fused = domain == FS_DOMAIN_LOG ? fsk_fused_log_plan(n, vec) : fsk_fused_plan(n, vec);
         if (s->fused.enabled) {
-            const size_t planes = domain == FS_DOMAIN_LOG ? 2 : 1;
+            const size_t planes = 1;
             const std::vector<FsRowTile> ft = build_tiles(s->offsets, s->fused.tile_rows);
             s->fused_ntiles = (int)ft.size();
             FS_CU(cudaMalloc(&s->fused_tiles_dev, sizeof(FsRowTile) * ft.size()));
@@ -373,6 +393,11 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
             const size_t pbytes = sizeof(float) * planes * (size_t)s->fused.nclusters * (size_t)n;
             FS_CU(cudaMalloc(&s->fused_partials, pbytes));
             FS_CU(cudaMemsetAsync(s->fused_partials, 0, pbytes, st));
+            if (domain == FS_DOMAIN_LOG) {
+                const size_t tbytes = sizeof(float) * 4 * (size_t)n + 64;
+                FS_CU(cudaMalloc(&s->fused_log_tmp, tbytes));
+                FS_CU(cudaMemsetAsync(s->fused_log_tmp, 0, tbytes, st));
+            }
         }
     }
     if (domain == FS_DOMAIN_SCALING && nbatch == 1) s->resident = fsk_resident_plan(n);
@@ -674,6 +699,16 @@ int fs_error_trace(fs_solver *s, double *l1_out, double *l2_out, int32_t cap, in
 
 int64_t fs_iterations_done(const fs_solver *s) { return s ? s->iter_done : -1; }
 int64_t fs_launch_count(const fs_solver *s) { return s ? s->launches : -1; }
+
+int fs_fused_log_fallbacks(fs_solver *s, int64_t *count_out, void *stream) {
+    if (!s || !count_out) return FS_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    FsDeviceStatus h{};
+    FS_CU(cudaMemcpyAsync(&h, s->status, sizeof(h), cudaMemcpyDeviceToHost, st));
+    FS_CU(cudaStreamSynchronize(st));
+    *count_out = h.fallbacks;
+    return FS_OK;
+}
 
 int fs_solve_host(int64_t n, int32_t c, const int64_t *row_offsets, const float *M_host, int64_t ld, int matrix_kind,
                   double eps, const float *a_host, const float *b_host, int32_t nbatch, int domain, int32_t iters,

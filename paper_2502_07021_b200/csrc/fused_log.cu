@@ -1,22 +1,28 @@
 // Single-read fused iteration, log domain, one problem.
 //
-// Same organisation as fused.cu (clusters of S CTAs, each CTA one column segment of every row in a
-// ring of shared-memory stages filled by bulk async copies; a "row" group and a "column" group of 8
-// warps each working on different rows at the same time), for the stabilised updates
+// The stabilised updates
+//   f_i <- eps log a_i - eps LSE_l((g_l - C_il)/eps),     g_l <- eps log b_l - eps LSE_i((f_i - C_il)/eps)
+// are evaluated with the current duals as stabilisers instead of running maxima.  With
+//   e_il = exp((f_i + g_l - C_il)/eps)      (an entry of the current plan),     s_i = sum_l e_il
+// the row update is exactly  f_i <- f_i + eps log(a_i / s_i), and the entries of the plan after it are
+// e_il * (a_i / s_i), so the column update is  g_l <- g_l + eps log(b_l / r_l),  r_l = sum_i e_il a_i / s_i:
+// ONE exponential per matrix element and iteration, and the column sums are plain multiply-adds with a
+// per-row factor -- the structure of the scaling-domain fused kernel (fused.cu) with e formed on the fly
+// from C.  s_i is the row marginal of the current plan and r_l the column marginal after the row update,
+// so both stay within a factor exp(+-delta/eps) of a_i, b_l, delta = the change of the duals in one
+// iteration; they leave the fp32 range only from a cold start or after a jump of the duals of more than
+// ~60 eps.  The kernels check s_i and r_l against [2^-90, 2^90]; outside it they raise status->range and
+// the driver's guarded two-pass kernels (running maxima, always safe) redo that iteration from the
+// untouched duals.  Results of this path are written to temporaries and committed only when in range.
 //
-//   f_i = eps log a_i - eps LSE_l((g_l - C_il)/eps),     g_l = eps log b_l - eps LSE_i((f_i - C_il)/eps).
-//
-// Exponents are kept in base 2: t = fma(C_il, -log2(e)/eps, g_l log2(e)/eps).
-//   - row group: a thread holds its slice of the scaled dual g in registers, forms its t values of a
-//     landed row segment, takes their maximum first and then one ex2 per element (no rescaling); the
-//     warp combines (max, sum) with one more ex2 per lane and sends the pair to every CTA of the
-//     cluster (st.async counted on the receiver's mbarrier);
-//   - column group: when the S*8 pairs of a row have arrived it combines them (maximum first, then one
-//     ex2 per pair), forms f_i, and folds the row into per-column running (max, sum) pairs held in
-//     registers.  The fold costs exactly one ex2 per element: 2^-|t - m| is either the rescale factor
-//     of the old sum (t is a new maximum) or the new term (it is not).
-// The cost matrix is read from HBM once per iteration instead of twice; per-cluster column pairs
-// are combined in cluster order by the ordinary stage-2 kernel.  Every wait is bounded.
+// Organisation: one persistent CTA of 1024 threads per SM owns whole rows (row tiles dealt round-robin; a row
+// of up to 16384 columns fits one shared-memory stage).  Thread 0 doubles as the producer and keeps a ring
+// of stages filled with bulk async copies.  Per step (R rows): every thread reads its columns of the stage
+// once, forms e (one ex2 per element) in REGISTERS and partial row sums; one block barrier completes the
+// sums and frees the stage for the next copy; then a_i/s_i is formed in a fixed order and e_il a_i/s_i is
+// accumulated into register-resident column sums.  32 warps per SM hide the latency of the special-function
+// unit; no cross-CTA exchange is needed.  Exponents are in base 2: xs = f log2(e)/eps, ys = g log2(e)/eps,
+// t = fma(C, -log2(e)/eps, ys_l) + xs_i.  Every wait is bounded.
 #include <math.h>
 
 #include "cluster_ptx.cuh"
@@ -26,305 +32,345 @@ namespace {
 
 using namespace fsptx;
 
-constexpr int kGroup = 256;
-constexpr int kThreadsLog = 2 * kGroup + 32;
-constexpr int kWarpsPerGroup = kGroup / 32;
-constexpr int kXchgStride = 64; // floats per exchange slot: S*8 (max, sum) pairs, S <= 4
-constexpr float kNegBig = -1.0e30f;
+constexpr int kThreadsLog = 1024;
+constexpr int kWarpsLog = kThreadsLog / 32;
+constexpr float kRangeLo = 8.0779357e-28f; // 2^-90
+constexpr float kRangeHi = 1.2379400e27f;  // 2^90
 
-template <int F>
+__device__ __forceinline__ bool in_range(float x) { return x >= kRangeLo && x <= kRangeHi; }
+
+// One stage = R whole rows of C (R * n floats).  Barriers: full[ns] (bulk copies of a stage landed).
+// FT = 128-bit column groups per thread: thread t of 1024 owns groups t, t + 1024, ... of every row: the same
+// columns when it forms e and when it accumulates the column sums.
+template <int FT, int R>
 __global__ void __launch_bounds__(kThreadsLog, 1)
-fused_log_iteration_kernel(const float *__restrict__ C, int64_t ld, int n, int S, int nclusters, int nstages, float s2,
-                           double eps, const FsRowTile *__restrict__ tiles, int ntiles, const float *__restrict__ ys,
-                           const float *__restrict__ a, const float *__restrict__ loga, float *__restrict__ f,
-                           float *__restrict__ xs, float *__restrict__ rowdiff, float *__restrict__ partials,
+fused_log_iteration_kernel(const float *__restrict__ C, int64_t ld, int n, int nctas, int nstages, float s2, double eps,
+                           const FsRowTile *__restrict__ tiles, int ntiles, const float *__restrict__ xs,
+                           const float *__restrict__ ys, const float *__restrict__ a, float *__restrict__ f_out,
+                           float *__restrict__ xs_out, float *__restrict__ rowdiff, float *__restrict__ partials,
                            FsDeviceStatus *status) {
     extern __shared__ uint8_t smem_raw[];
-    constexpr int W = F * 1024;
-    const uint32_t stage_bytes = W * 4;
+    const uint32_t row_bytes = (uint32_t)n * 4u;
+    const uint32_t stage_bytes = R * row_bytes;
     const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
-    const uint32_t xchg = base + (uint32_t)nstages * stage_bytes;
-    const uint32_t bars = xchg + (uint32_t)(2 * nstages) * kXchgStride * 4; // full[ns], empty[ns], qbar[2 ns]
-    const uint32_t rank = cluster_ctarank();
-    const int cluster = blockIdx.x / S;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int col0 = (int)rank * W;
-    const int seg = max(0, min(W, n - col0));
-    const int seg4 = seg >> 2;
+    const uint32_t red = base + (uint32_t)nstages * stage_bytes;   // [2][R][kWarpsLog] floats
+    const uint32_t bar_full = red + 2u * R * kWarpsLog * 4u;
+    const float *red_f = reinterpret_cast<const float *>(smem_raw + (red - smem_u32(smem_raw)));
+    float *red_w = const_cast<float *>(red_f);
+    __shared__ int fail_s;
+    const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
+    const int cta = blockIdx.x;
+    const int n4 = n >> 2;
     const float ns2 = -s2;
+    const bool cols_full = n4 == FT * kThreadsLog;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < nstages; ++s) {
-            mbar_init(bars + 8 * s, 1);
-            mbar_init(bars + 8 * (nstages + s), kWarpsPerGroup);
-        }
-        for (int s = 0; s < 2 * nstages; ++s) mbar_init(bars + 8 * (2 * nstages + s), 1);
+    if (t == 0) {
+        for (int s = 0; s < nstages; ++s) mbar_init(bar_full + 8 * s, 1);
+        fail_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    cluster_sync_all();
 
-    bool ok = true;
-    if (warp == 2 * kWarpsPerGroup) {
-        // ---------------- producer ----------------
-        if (lane == 0) {
-            int k = 0;
-            for (int t = cluster; t < ntiles && ok; t += nclusters) {
-                const FsRowTile tile = tiles[t];
-                for (int row = tile.begin; row < tile.end; ++row, ++k) {
-                    const int s = k % nstages;
-                    const uint32_t ph = (uint32_t)(k / nstages) & 1u;
-                    if (!mbar_wait(bars + 8 * (nstages + s), ph ^ 1u)) { ok = false; break; }
-                    const uint32_t full = bars + 8 * s;
-                    mbar_expect_tx(bars + 8 * (2 * nstages + k % (2 * nstages)), (uint32_t)(S * kWarpsPerGroup) * 8u);
-                    if (seg > 0) {
-                        mbar_expect_tx(full, (uint32_t)seg * 4u);
-                        const float *src = C + (int64_t)row * ld + col0;
-                        const uint32_t dst = base + (uint32_t)s * stage_bytes;
-                        for (int off = 0; off < seg; off += 4096) {
-                            const int cnt = min(4096, seg - off);
-                            bulk_load(dst + (uint32_t)off * 4u, src + off, (uint32_t)cnt * 4u, full);
-                        }
-                    } else {
-                        mbar_arrive(full);
+    // Steps of this CTA in order: tiles cta, cta + nctas, ...; within a tile R rows at a time.  Thread 0 is also
+    // the producer: it walks the same sequence `nstages` steps ahead.
+    int p_tile = cta, p_row = 0, p_end = 0, p_k = 0; // producer cursor (thread 0 only)
+    bool p_more = false;
+    auto producer_issue = [&]() { // issues the bulk copies of the producer cursor's step and advances it
+        if (!p_more) return;
+        const int cnt = min(R, p_end - p_row);
+        const int s = p_k % nstages;
+        const uint32_t full = bar_full + 8 * s;
+        mbar_expect_tx(full, (uint32_t)cnt * row_bytes);
+        for (int r = 0; r < cnt; ++r) {
+            const float *src = C + (int64_t)(p_row + r) * ld;
+            const uint32_t dst = base + (uint32_t)s * stage_bytes + (uint32_t)r * row_bytes;
+            for (int off = 0; off < n; off += 4096) { // 16 KB pieces
+                const int c = min(4096, n - off);
+                bulk_load(dst + (uint32_t)off * 4u, src + off, (uint32_t)c * 4u, full);
+            }
+        }
+        ++p_k;
+        p_row += R;
+        if (p_row >= p_end) {
+            p_tile += nctas;
+            p_more = p_tile < ntiles;
+            if (p_more) {
+                const FsRowTile tile = tiles[p_tile];
+                p_row = tile.begin, p_end = tile.end;
+            }
+        }
+    };
+    if (t == 0) {
+        p_more = p_tile < ntiles;
+        if (p_more) {
+            const FsRowTile tile = tiles[p_tile];
+            p_row = tile.begin, p_end = tile.end;
+        }
+        for (int s = 0; s < nstages; ++s) producer_issue();
+    }
+
+    float4 g4[FT], r4[FT];
+#pragma unroll
+    for (int j = 0; j < FT; ++j) {
+        const int c4 = j * kThreadsLog + t;
+        g4[j] = c4 < n4 ? __ldg(reinterpret_cast<const float4 *>(ys) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        r4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    bool out_of_range = false, ok = true;
+    int k = 0;
+    for (int tl = cta; tl < ntiles && ok; tl += nctas) {
+        const FsRowTile tile = tiles[tl];
+        // the tile's marginal entries and scaled row duals (at most 32 rows): lane i keeps row i
+        float a_lane = 1.f, xs_lane = 0.f;
+        if (tile.begin + lane < tile.end) {
+            a_lane = a[tile.begin + lane];
+            xs_lane = xs[tile.begin + lane];
+        }
+        for (int row = tile.begin; row < tile.end; row += R, ++k) {
+            const int cnt = min(R, tile.end - row);
+            const int s = k % nstages;
+            float fh[R], ar[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int src_lane = min(row + r, tile.end - 1) - tile.begin;
+                fh[r] = __shfl_sync(0xffffffffu, xs_lane, src_lane);
+                ar[r] = __shfl_sync(0xffffffffu, a_lane, src_lane);
+            }
+            if (!mbar_wait(bar_full + 8 * s, (uint32_t)(k / nstages) & 1u)) fail_s = 1; // seen by all after the barrier
+            // ---- e into registers (one ex2 per element), partial row sums
+            const uint32_t st = base + (uint32_t)s * stage_bytes + (uint32_t)t * 16u;
+            float4 e[FT][R];
+            float acc[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) acc[r] = 0.f;
+            if (cols_full && cnt == R) {
+                // the common step: every row and column exists, straight-line code without predicates
+#pragma unroll
+                for (int j = 0; j < FT; ++j) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) e[j][r] = lds4(st + (uint32_t)r * row_bytes + (uint32_t)j * (kThreadsLog * 16u));
+                }
+#pragma unroll
+                for (int j = 0; j < FT; ++j) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        float4 x;
+                        x.x = ex2(fmaf(e[j][r].x, ns2, g4[j].x) + fh[r]);
+                        x.y = ex2(fmaf(e[j][r].y, ns2, g4[j].y) + fh[r]);
+                        x.z = ex2(fmaf(e[j][r].z, ns2, g4[j].z) + fh[r]);
+                        x.w = ex2(fmaf(e[j][r].w, ns2, g4[j].w) + fh[r]);
+                        e[j][r] = x;
+                        acc[r] += (x.x + x.y) + (x.z + x.w);
                     }
                 }
-            }
-            if (!ok) {
-                for (int j = max(0, k - nstages); j < k; ++j)
-                    (void)mbar_wait(bars + 8 * (j % nstages), (uint32_t)(j / nstages) & 1u);
-            }
-        }
-    } else if (warp < kWarpsPerGroup) {
-        // ---------------- row group: (max, sum) of 2^t over this CTA's segment ----------------
-        const int t = threadIdx.x;
-        float4 y4[F];
+            } else {
 #pragma unroll
-        for (int j = 0; j < F; ++j) {
-            const int c4 = j * kGroup + t;
-            y4[j] = c4 < seg4 ? __ldg(reinterpret_cast<const float4 *>(ys + col0) + c4)
-                              : make_float4(kNegBig, kNegBig, kNegBig, kNegBig);
-        }
-        int k = 0;
-        for (int tl = cluster; tl < ntiles && ok; tl += nclusters) {
-            const FsRowTile tile = tiles[tl];
-            for (int row = tile.begin; row < tile.end; ++row, ++k) {
-                const int s = k % nstages;
-                const int slot = k % (2 * nstages);
-                if (!mbar_wait(bars + 8 * s, (uint32_t)(k / nstages) & 1u)) { ok = false; break; }
-                const uint32_t st = base + (uint32_t)s * stage_bytes + (uint32_t)t * 16u;
-                float tv[4 * F];
-                float m = kNegBig;
+                for (int j = 0; j < FT; ++j) {
 #pragma unroll
-                for (int j = 0; j < F; ++j) {
-                    if (j * kGroup + t < seg4) {
-                        const float4 cv = lds4(st + (uint32_t)j * (kGroup * 16u));
-                        tv[4 * j + 0] = fmaf(cv.x, ns2, y4[j].x);
-                        tv[4 * j + 1] = fmaf(cv.y, ns2, y4[j].y);
-                        tv[4 * j + 2] = fmaf(cv.z, ns2, y4[j].z);
-                        tv[4 * j + 3] = fmaf(cv.w, ns2, y4[j].w);
-                        m = fmaxf(m, fmaxf(fmaxf(tv[4 * j], tv[4 * j + 1]), fmaxf(tv[4 * j + 2], tv[4 * j + 3])));
-                    } else {
-                        tv[4 * j + 0] = tv[4 * j + 1] = tv[4 * j + 2] = tv[4 * j + 3] = kNegBig;
-                    }
-                }
-                float sum = 0.f;
-#pragma unroll
-                for (int j = 0; j < F; ++j) {
-                    if (j * kGroup + t < seg4)
-                        sum += (ex2(tv[4 * j] - m) + ex2(tv[4 * j + 1] - m)) + (ex2(tv[4 * j + 2] - m) + ex2(tv[4 * j + 3] - m));
-                }
-                // warp: maximum first, one rescale per lane, then a fixed-order sum
-                float wm = m;
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, off));
-                sum *= ex2(m - wm);
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-                if (lane < S) {
-                    const uint32_t cell = xchg + (uint32_t)(slot * kXchgStride + ((int)rank * kWarpsPerGroup + warp) * 2) * 4u;
-                    const uint32_t qb = bars + 8 * (2 * nstages + slot);
-                    st_async_v2f32(map_to_cta(cell, (uint32_t)lane), wm, sum, map_to_cta(qb, (uint32_t)lane));
-                }
-            }
-        }
-    } else {
-        // ---------------- column group: f_i, then per-column running (max, sum) ----------------
-        const int t = threadIdx.x - kGroup;
-        float cm[4 * F], cs[4 * F];
-#pragma unroll
-        for (int j = 0; j < 4 * F; ++j) {
-            cm[j] = kNegBig;
-            cs[j] = 0.f;
-        }
-        const double s2d = 1.4426950408889634 / eps, inv_eps = 1.0 / eps;
-        int k = 0;
-        for (int tl = cluster; tl < ntiles && ok; tl += nclusters) {
-            const FsRowTile tile = tiles[tl];
-            float a_lane = 1.f, la_lane = 0.f, fo_lane = 0.f;
-            if (tile.begin + lane < tile.end) {
-                a_lane = a[tile.begin + lane];
-                la_lane = loga[tile.begin + lane];
-                fo_lane = f[tile.begin + lane];
-            }
-            for (int row = tile.begin; row < tile.end; ++row, ++k) {
-                const int s = k % nstages;
-                const int slot = k % (2 * nstages);
-                if (!mbar_wait(bars + 8 * s, (uint32_t)(k / nstages) & 1u)) { ok = false; break; }
-                if (!mbar_wait_cluster(bars + 8 * (2 * nstages + slot), (uint32_t)(k / (2 * nstages)) & 1u)) { ok = false; break; }
-                // combine the S*8 pairs: lane j takes pair j
-                float pm = kNegBig, ps = 0.f;
-                if (lane < S * kWarpsPerGroup) {
-                    const float2 pr = lds2(xchg + (uint32_t)(slot * kXchgStride + lane * 2) * 4u);
-                    pm = pr.x, ps = pr.y;
-                }
-                float M = pm;
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
-                float Ssum = ps * ex2(pm - M);
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) Ssum += __shfl_xor_sync(0xffffffffu, Ssum, off);
-                const int r = row - tile.begin;
-                const double la = (double)__shfl_sync(0xffffffffu, la_lane, r);
-                // L_i in natural-log units, f_i = eps (log a_i - L_i); the scaled copy comes from the rounded f_i
-                const double Li = ((double)M + (double)log2f(Ssum)) * 0.6931471805599453;
-                const double fn = eps * (la - Li);
-                const float fnf = (float)fn;
-                const float xi = (float)((double)fnf * s2d);
-                const float fo_f = __shfl_sync(0xffffffffu, fo_lane, r);
-                const float ai_f = __shfl_sync(0xffffffffu, a_lane, r);
-                if (t == 0 && rank == 0) {
-                    // the difference of the duals in fp64 (fn is not yet rounded), the exponential in fp32
-                    rowdiff[row] = ai_f * expm1f((float)(((double)fo_f - fn) * inv_eps));
-                    f[row] = fnf;
-                    xs[row] = xi;
-                    if (!isfinite(fnf)) status->nonfinite = 1;
-                }
-                const uint32_t st = base + (uint32_t)s * stage_bytes + (uint32_t)t * 16u;
-#pragma unroll
-                for (int j = 0; j < F; ++j) {
-                    if (j * kGroup + t < seg4) {
-                        const float4 cv = lds4(st + (uint32_t)j * (kGroup * 16u));
-                        const float tt[4] = {fmaf(cv.x, ns2, xi), fmaf(cv.y, ns2, xi), fmaf(cv.z, ns2, xi), fmaf(cv.w, ns2, xi)};
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            // one ex2 serves both cases: 2^-|t - m| is the rescale factor of the old sum when t
-                            // is a new maximum (the new term is then 1) and the new term itself otherwise
-                            const float mo = cm[4 * j + q];
-                            const float e = ex2(-fabsf(tt[q] - mo));
-                            cs[4 * j + q] = tt[q] > mo ? fmaf(cs[4 * j + q], e, 1.f) : cs[4 * j + q] + e;
-                            cm[4 * j + q] = fmaxf(mo, tt[q]);
+                    for (int r = 0; r < R; ++r) {
+                        e[j][r] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (j * kThreadsLog + t < n4 && r < cnt) {
+                            const float4 c4 = lds4(st + (uint32_t)r * row_bytes + (uint32_t)j * (kThreadsLog * 16u));
+                            float4 x;
+                            x.x = ex2(fmaf(c4.x, ns2, g4[j].x) + fh[r]);
+                            x.y = ex2(fmaf(c4.y, ns2, g4[j].y) + fh[r]);
+                            x.z = ex2(fmaf(c4.z, ns2, g4[j].z) + fh[r]);
+                            x.w = ex2(fmaf(c4.w, ns2, g4[j].w) + fh[r]);
+                            e[j][r] = x;
+                            acc[r] += (x.x + x.y) + (x.z + x.w);
                         }
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bars + 8 * (nstages + s));
             }
-        }
-        if (ok) {
-            float4 *outm = reinterpret_cast<float4 *>(partials + (int64_t)cluster * n + col0);
-            float4 *outs = reinterpret_cast<float4 *>(partials + ((int64_t)nclusters + cluster) * n + col0);
 #pragma unroll
-            for (int j = 0; j < F; ++j) {
-                const int c4 = j * kGroup + t;
-                if (c4 < seg4) {
-                    outm[c4] = make_float4(cm[4 * j], cm[4 * j + 1], cm[4 * j + 2], cm[4 * j + 3]);
-                    outs[c4] = make_float4(cs[4 * j], cs[4 * j + 1], cs[4 * j + 2], cs[4 * j + 3]);
+            for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], off);
+            }
+            float *rb = red_w + (size_t)(k & 1) * R * kWarpsLog;
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) rb[r * kWarpsLog + warp] = acc[r];
+            }
+            // one block barrier per step: the per-warp sums are complete, and every thread has consumed the stage,
+            // which was only read and can be refilled
+            __syncthreads();
+            if (fail_s) { ok = false; break; }
+            if (t == 0) producer_issue();
+            // ---- row factor a_i / s_i (lane w holds the sum of warp w; a fixed butterfly gives every lane the
+            //      same total), column sums from the e kept in registers
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float wi = 0.f;
+                if (r < cnt) {
+                    float si = rb[r * kWarpsLog + lane];
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) si += __shfl_xor_sync(0xffffffffu, si, off);
+                    wi = ar[r] / si;
+                    if (t == 0) {
+                        rowdiff[row + r] = si - ar[r]; // s_i is the row marginal of the plan that was read
+                        const float xn = fh[r] + __log2f(wi);
+                        xs_out[row + r] = xn;
+                        f_out[row + r] = (float)((double)xn * eps * 0.6931471805599453);
+                        if (!in_range(si)) out_of_range = true;
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < FT; ++j) { // e of columns or rows that do not exist is zero
+                    r4[j].x = fmaf(e[j][r].x, wi, r4[j].x);
+                    r4[j].y = fmaf(e[j][r].y, wi, r4[j].y);
+                    r4[j].z = fmaf(e[j][r].z, wi, r4[j].z);
+                    r4[j].w = fmaf(e[j][r].w, wi, r4[j].w);
                 }
             }
         }
     }
-    if (!ok) status->timeout = 1;
-    __syncwarp();
-    cluster_sync_all();
+    if (out_of_range) status->range = 1;
+    if (ok) {
+        float4 *out = reinterpret_cast<float4 *>(partials + (int64_t)cta * n);
+#pragma unroll
+        for (int j = 0; j < FT; ++j) {
+            const int c4 = j * kThreadsLog + t;
+            if (c4 < n4) out[c4] = r4[j];
+        }
+    } else if (t == 0) {
+        status->timeout = 1;
+        // drain: copies already issued must land before this CTA's shared memory goes away
+        for (int j = max(k, p_k - nstages); j < p_k; ++j)
+            (void)mbar_wait(bar_full + 8 * (j % nstages), (uint32_t)(j / nstages) & 1u);
+    }
 }
 
-size_t log_smem_bytes(int F, int nstages) {
-    return (size_t)nstages * F * 4096 + (size_t)2 * nstages * kXchgStride * 4 + (size_t)8 * 4 * nstages + 256;
+// Stage 2 of the fused log iteration: r_l = sum of the per-cluster column sums in cluster order,
+// g_l <- g_l + eps log(b_l / r_l), written to the temporaries; coldiff = r_l - b_l.
+__global__ void __launch_bounds__(256)
+fused_log_finish_kernel(int n, int nclusters, double eps, const float *__restrict__ partials, const float *__restrict__ b,
+                        const float *__restrict__ ys, float *__restrict__ g_out, float *__restrict__ ys_out,
+                        float *__restrict__ coldiff, FsDeviceStatus *status) {
+    const int l = blockIdx.x * 256 + threadIdx.x;
+    if (l >= n) return;
+    float r = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < nclusters; ++k) r += partials[(int64_t)k * n + l];
+    const float bl = b[l];
+    coldiff[l] = r - bl;
+    const float yn = ys[l] + __log2f(bl / r);
+    ys_out[l] = yn;
+    g_out[l] = (float)((double)yn * eps * 0.6931471805599453);
+    if (!in_range(r)) status->range = 1;
 }
 
-template <int F>
-void fill_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int S, int nclusters, int nstages, cudaStream_t st) {
-    cfg = cudaLaunchConfig_t{};
-    cfg.gridDim = dim3((unsigned)(nclusters * S));
-    cfg.blockDim = dim3(kThreadsLog);
-    cfg.dynamicSmemBytes = log_smem_bytes(F, nstages);
-    cfg.stream = st;
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)S;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+// Commit: when the iteration stayed in range the temporaries become the duals; otherwise the guarded
+// two-pass kernels have already written the duals and only the flag is cleared (and counted).
+__global__ void __launch_bounds__(256)
+fused_log_commit_kernel(int n, const float *__restrict__ f_tmp, const float *__restrict__ xs_tmp,
+                        const float *__restrict__ g_tmp, const float *__restrict__ ys_tmp, float *__restrict__ f,
+                        float *__restrict__ xs, float *__restrict__ g, float *__restrict__ ys, FsDeviceStatus *status,
+                        int *done_blocks) {
+    const int l = blockIdx.x * 256 + threadIdx.x;
+    const bool failed = *reinterpret_cast<volatile int *>(&status->range) != 0;
+    if (!failed && l < n) {
+        f[l] = f_tmp[l];
+        xs[l] = xs_tmp[l];
+        g[l] = g_tmp[l];
+        ys[l] = ys_tmp[l];
+    }
+    // the last block to finish resets the flag for the next iteration (all blocks have read it by then)
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const int prev = atomicAdd(done_blocks, 1);
+        if (prev == (int)gridDim.x - 1) {
+            *done_blocks = 0;
+            if (failed) {
+                status->range = 0;
+                status->fallbacks += 1;
+            }
+            __threadfence();
+        }
+    }
 }
 
-template <int F>
-int query_clusters(int S, int nstages) {
-    if (cudaFuncSetAttribute(fused_log_iteration_kernel<F>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)log_smem_bytes(F, nstages)) != cudaSuccess) {
+size_t fused_log_smem_bytes(int64_t n, int R, int nstages) {
+    return (size_t)nstages * R * (size_t)n * 4 + (size_t)2 * R * kWarpsLog * 4 + (size_t)8 * nstages + 256;
+}
+
+template <int FT, int R>
+cudaError_t launch_fused_log(const FsFusedPlan &p, cudaStream_t st, const float *C, int64_t ld, int n, float s2, double eps,
+                             const FsRowTile *tiles, int ntiles, const float *xs, const float *ys, const float *a,
+                             float *f_out, float *xs_out, float *rowdiff, float *partials, FsDeviceStatus *status) {
+    fused_log_iteration_kernel<FT, R><<<(unsigned)p.nclusters, kThreadsLog, fused_log_smem_bytes(n, R, p.nstages), st>>>(
+        C, ld, n, p.nclusters, p.nstages, s2, eps, tiles, ntiles, xs, ys, a, f_out, xs_out, rowdiff, partials, status);
+    return cudaGetLastError();
+}
+
+template <int FT, int R>
+int query_ctas(int64_t n, int nstages) {
+    const size_t smem = fused_log_smem_bytes(n, R, nstages);
+    if (cudaFuncSetAttribute(fused_log_iteration_kernel<FT, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
-    cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
-    fill_config<F>(cfg, attr, S, 148, nstages, nullptr);
-    int nc = 0;
-    if (cudaOccupancyMaxActiveClusters(&nc, fused_log_iteration_kernel<F>, &cfg) != cudaSuccess) {
+    int per_sm = 0, dev = 0, sms = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_log_iteration_kernel<FT, R>, kThreadsLog, smem) !=
+            cudaSuccess ||
+        cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
-    return nc;
-}
-
-template <int F>
-cudaError_t launch(const FsFusedPlan &p, cudaStream_t st, const float *C, int64_t ld, int n, float s2, double eps,
-                   const FsRowTile *tiles, int ntiles, const float *ys, const float *a, const float *loga, float *f,
-                   float *xs, float *rowdiff, float *partials, FsDeviceStatus *status) {
-    cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
-    fill_config<F>(cfg, attr, p.S, p.nclusters, p.nstages, st);
-    return cudaLaunchKernelEx(&cfg, fused_log_iteration_kernel<F>, C, ld, n, p.S, p.nclusters, p.nstages, s2, eps, tiles,
-                              ntiles, ys, a, loga, f, xs, rowdiff, partials, status);
+    return per_sm >= 1 ? sms : 0;
 }
 
 } // namespace
 
-// Configuration of the fused log-domain iteration: at most 8 column groups per thread (the column
-// group keeps two registers per column), so S = 2 up to n = 16384 and S = 4 up to n = 32768.
+// Chooses the fused log-domain configuration for an n x n problem; enabled = false when it does not apply.
+// nclusters = number of persistent CTAs = rows of the column-partial matrix.
 FsFusedPlan fsk_fused_log_plan(int64_t n, bool vec) {
     FsFusedPlan p{};
-    if (!vec || (n & 3) != 0 || n < 2048) return p;
-    int S = 2;
-    int64_t fgroups = (n + 2047) / 2048;
-    if (fgroups > 8) {
-        S = 4;
-        fgroups = (n + 4095) / 4096;
-    }
-    if (fgroups > 8) return p;
-    const int F = fgroups <= 2 ? 2 : fgroups <= 4 ? 4 : 8;
-    int ns = (int)(200 * 1024 / (F * 4096));
+    if (!vec || (n & 3) != 0 || n < 2048 || n > 16384) return p; // a whole row must fit one 64 KB stage
+    const int FT = (int)((n / 4 + kThreadsLog - 1) / kThreadsLog); // 128-bit column groups per thread: 1..4
+    const int R = FT == 1 ? 4 : FT == 2 ? 2 : 1;                   // rows per stage: stages of at most 64 KB
+    int ns = (int)(200 * 1024 / ((size_t)R * (size_t)n * 4));
     if (ns > 8) ns = 8;
+    if (ns < 2) return p;
     int nc = 0;
-    switch (F) {
-    case 2: nc = query_clusters<2>(S, ns); break;
-    case 4: nc = query_clusters<4>(S, ns); break;
-    default: nc = query_clusters<8>(S, ns); break;
+    switch (FT) {
+    case 1: nc = query_ctas<1, 4>(n, ns); break;
+    case 2: nc = query_ctas<2, 2>(n, ns); break;
+    case 3: nc = query_ctas<3, 1>(n, ns); break;
+    default: nc = query_ctas<4, 1>(n, ns); break;
     }
     if (nc < 1) return p;
-    p.enabled = true, p.S = S, p.F = F, p.R = 1, p.nstages = ns, p.nclusters = nc, p.tile_rows = 32;
+    p.enabled = true, p.S = 1, p.F = FT, p.R = R, p.nstages = ns, p.nclusters = nc, p.tile_rows = 32;
     return p;
 }
 
-// One fused log-domain iteration minus stage 2: writes f, its scaled copy, rowdiff and the per-cluster
-// column pairs (plane 0: maxima [nclusters][n], plane 1: sums).
+// One fused log-domain iteration, uncommitted: reads the duals (xs, ys scaled copies), writes the new duals
+// to the temporaries, rowdiff / coldiff directly, and raises status->range when a marginal left the safe range.
 cudaError_t fsk_fused_log_iteration(const FsFusedPlan &p, const float *C, int64_t ld, int64_t n, double eps,
-                                    const FsRowTile *tiles, int ntiles, const float *ys, const float *a,
-                                    const float *loga, float *f, float *xs, float *rowdiff, float *partials,
-                                    FsDeviceStatus *status, cudaStream_t st) {
+                                    const FsRowTile *tiles, int ntiles, const float *xs, const float *ys, const float *a,
+                                    const float *b, float *f_tmp, float *xs_tmp, float *g_tmp, float *ys_tmp,
+                                    float *rowdiff, float *coldiff, float *partials, FsDeviceStatus *status,
+                                    cudaStream_t st) {
     const float s2 = (float)(1.4426950408889634 / eps);
+    cudaError_t e;
     switch (p.F) {
-    case 2: return launch<2>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, ys, a, loga, f, xs, rowdiff, partials, status);
-    case 4: return launch<4>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, ys, a, loga, f, xs, rowdiff, partials, status);
-    default: return launch<8>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, ys, a, loga, f, xs, rowdiff, partials, status);
+    case 1: e = launch_fused_log<1, 4>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
+    case 2: e = launch_fused_log<2, 2>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
+    case 3: e = launch_fused_log<3, 1>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
+    default: e = launch_fused_log<4, 1>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
     }
+    if (e != cudaSuccess) return e;
+    fused_log_finish_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>((int)n, p.nclusters, eps, partials, b, ys, g_tmp, ys_tmp,
+                                                                         coldiff, status);
+    return cudaGetLastError();
+}
+
+// Commits the temporaries (or, after a range failure, leaves the duals the guarded two-pass kernels wrote).
+void fsk_fused_log_commit(int64_t n, const float *f_tmp, const float *xs_tmp, const float *g_tmp, const float *ys_tmp,
+                          float *f, float *xs, float *g, float *ys, FsDeviceStatus *status, int *done_blocks, cudaStream_t st) {
+    fused_log_commit_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>((int)n, f_tmp, xs_tmp, g_tmp, ys_tmp, f, xs, g, ys, status,
+                                                                         done_blocks);
 }

@@ -179,8 +179,9 @@ def test_fused_single_read_iteration(n, offsets):
 
 @pytest.mark.parametrize("n,offsets", [(2048, None), (4100, None), (8192, [0, 5, 37, 4096, 4100, 8192]), (8200, None)])
 def test_fused_single_read_iteration_log_domain(n, offsets):
-    """The log-domain fused kernel (row LSE, then per-column running (max, sum) pairs from the same
-    on-chip row) against the two-pass log path and the oracle."""
+    """The log-domain fused iteration (one exponential per element with the current duals as stabilisers,
+    column sums from the same on-chip rows; out-of-range iterations redone by the guarded two-pass kernels)
+    against the two-pass log path and the oracle."""
     w = workloads.make(3, n=n)
     off = w.offsets if offsets is None else np.asarray(offsets, dtype=np.int64)
     res = {}
@@ -191,8 +192,12 @@ def test_fused_single_read_iteration_log_domain(n, offsets):
                 fs.fs_set_option(g.h, fs.FS_OPT_PERSISTENT, 0)     # mode 0 is to be the two-pass graph path
             before = fs.fs_launch_count(g.h)
             g.iterate(10)
-            assert fs.fs_launch_count(g.h) - before == (30 if mode == 0 else 20)
+            assert fs.fs_launch_count(g.h) - before == (30 if mode == 0 else 60)
             res[mode] = g.scalings()
+            if mode == 2:
+                # a cold start may be out of the fused kernels' range (then the two-pass kernels redo it); the
+                # fused kernels must carry the run after the first few iterations
+                assert fs.fs_fused_log_fallbacks(g.h, g.stream) <= 3
             row, col = g.errors(1)
             res[mode] += (row[0], col[0])
     f, gg = oracle.sinkhorn_log(w.C, w.eps, w.a, w.b, 10)
@@ -219,6 +224,28 @@ def test_fused_log_is_reproducible_and_traces():
         f, gg = oracle.sinkhorn_log(w.C, w.eps, w.a, w.b, t)
         e = oracle.marginal_errors(w.C, oracle.KIND_COST, w.eps, LG, f, gg, w.a, w.b)
         assert l1[k] == pytest.approx(e["row_l1"], rel=2e-3, abs=1e-6)
+
+
+def test_fused_log_falls_back_after_a_jump_of_the_duals():
+    """A jump of the duals by hundreds of eps between two iterations takes the marginals out of the fused
+    path's fp32 range: that iteration must be redone by the two-pass kernels, transparently."""
+    w = workloads.make(3, n=2048)
+    with GpuSolver(w.C, KC, w.eps, w.a, w.b, w.offsets, LG) as g:
+        fs.fs_set_option(g.h, fs.FS_OPT_FUSED, 2)
+        g.iterate(6)
+        before = fs.fs_fused_log_fallbacks(g.h, g.stream)
+        f6, g6 = g.scalings()
+        shift = np.where(np.arange(w.n) % 2 == 0, 3.0, -3.0).astype(np.float32)    # +-300 eps
+        g.set_scalings(f6, g6 + shift)
+        g.iterate(4)
+        assert fs.fs_fused_log_fallbacks(g.h, g.stream) > before
+        fj, gj = g.scalings()
+    with GpuSolver(w.C, KC, w.eps, w.a, w.b, w.offsets, LG) as g:
+        fs.fs_set_option(g.h, fs.FS_OPT_FUSED, 0)
+        g.set_scalings(f6, g6 + shift)
+        g.iterate(4)
+        f0, g0 = g.scalings()
+    assert np.max(np.abs(fj - f0)) / w.eps < TOL_UV and np.max(np.abs(gj - g0)) / w.eps < TOL_UV
 
 
 @pytest.mark.slow
