@@ -44,7 +44,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
             rebuilt = True
     if rebuilt or not os.path.exists(LIB):
         tmp = LIB + f".tmp{os.getpid()}"
-        subprocess.run([nvcc, "-shared", "-o", tmp, *objs], check=True)
+        subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp, *objs], check=True)
         os.replace(tmp, LIB)
     return LIB
 

@@ -51,7 +51,6 @@ struct TcState {
     int nbatch = 0, nb_pad = 0, mtiles = 0, ntiles = 0, kblocks = 0, ksplit = 1;
     __nv_bfloat16 *K_hi = nullptr, *K_lo = nullptr, *Kt_hi = nullptr, *Kt_lo = nullptr;
     __nv_bfloat16 *U_hi = nullptr, *U_lo = nullptr, *V_hi = nullptr, *V_lo = nullptr;
-    float *partials = nullptr;
     CUtensorMap tmK_hi, tmK_lo, tmKt_hi, tmKt_lo, tmU_hi, tmU_lo, tmV_hi, tmV_lo;
 };
 
@@ -135,12 +134,50 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
 // Instruction descriptor: D = fp32, A = B = bf16, both K-major, N = 128, M = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
-// ---- GEMM kernel -------------------------------------------------------------------------
-// blockIdx.x = output row tile, blockIdx.y = split of the contraction range, blockIdx.z = tile of problems.
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
+    hi = __float2bfloat16_rn(x);
+    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ float ld_shared_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+// ---- GEMM kernel with the update fused into its epilogue ------------------------------------
+// blockIdx.x = output row tile, blockIdx.z = tile of problems; the KS CTAs along y form one cluster and
+// split the contraction range among them (rank in the cluster = index of the split).  After the main
+// loop every CTA holds a 128 x 128 fp32 partial tile in registers.  The tile's 128 problems are dealt
+// W = 128 / KS to each rank: every rank stores its partial sums for rank q's problems into q's shared
+// memory (the ring is idle by then: a cluster barrier separates the two uses), and after a second
+// cluster barrier rank q adds the KS contributions in rank order and applies the divide, the marginal
+// residual and the bf16 re-split of the new scalings -- no partial tile goes through HBM and no second
+// kernel is launched.
+template <int KS>
 __global__ void __launch_bounds__(kTcThreads, 1)
 batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_constant__ CUtensorMap tmA_lo,
                   const __grid_constant__ CUtensorMap tmB_hi, const __grid_constant__ CUtensorMap tmB_lo,
-                  float *__restrict__ partials, int kblocks, int ksplit, FsDeviceStatus *status) {
+                  int kblocks, int n, int nbatch, const float *__restrict__ marg, float *out,
+                  float *__restrict__ diff, __nv_bfloat16 *__restrict__ op_hi, __nv_bfloat16 *__restrict__ op_lo,
+                  int update, float eta, FsDeviceStatus *status) {
+    constexpr int ksplit = KS;
+    constexpr int W = BN / KS;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bars = base + STAGES * STAGE_BYTES;
@@ -148,7 +185,7 @@ batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_const
     const uint32_t tmem_slot = bars + 8 * NUM_BARS;
     uint32_t *tmem_slot_ptr = reinterpret_cast<uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int mtile = blockIdx.x, ks = blockIdx.y, ntile = blockIdx.z;
+    const int mtile = blockIdx.x, ks = (int)cluster_ctarank(), ntile = blockIdx.z;
     const int kb0 = (int)((int64_t)kblocks * ks / ksplit), kb1 = (int)((int64_t)kblocks * (ks + 1) / ksplit);
     const int nkb = kb1 - kb0;
 
@@ -248,61 +285,66 @@ batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_const
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_empty + 8 * buf) : "memory");
         }
-        if (ok) {
-            const int unit = ((ntile * gridDim.x + mtile) * ksplit + ks);
-            float *out = partials + (size_t)unit * (BM * BN) + row;
+        // exchange.  Barrier 1: every CTA of the cluster has finished its main loop (its tensor-core reads of the
+        // ring are complete), so stage 0 of every ring can take the partial sums.
+        cluster_sync_all();
+        const uint32_t recv = base; // [KS][W][BM] floats = 64 KB = one ring stage
 #pragma unroll
-            for (int j = 0; j < BN; ++j) out[(size_t)j * BM] = sum[j];
+        for (int q = 0; q < KS; ++q) {
+            const uint32_t dst = map_to_cta(recv + (uint32_t)((ks * W) * BM + row) * 4u, (uint32_t)q);
+#pragma unroll
+            for (int jj = 0; jj < W; ++jj) st_cluster_f32(dst + (uint32_t)(jj * BM) * 4u, sum[q * W + jj]);
         }
+        // Barrier 2: all contributions have landed (release / acquire at cluster scope).
+        cluster_sync_all();
+        const int gi = mtile * BM + row;
+        if (ok && gi < n) {
+            constexpr int G = 8; // problems handled together so that their loads are in flight at once
+#pragma unroll 1
+            for (int j0 = 0; j0 < W; j0 += G) {
+                float q[G], mg[G], old[G];
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const int gp = ntile * BN + ks * W + j0 + g;
+                    const int64_t idx = (int64_t)gp * n + gi;
+                    const bool live = gp < nbatch;
+                    mg[g] = live ? marg[idx] : 1.f;
+                    old[g] = live ? out[idx] : 1.f;
+                    float acc = ld_shared_f32(recv + (uint32_t)((j0 + g) * BM + row) * 4u);
+#pragma unroll
+                    for (int r = 1; r < KS; ++r) acc += ld_shared_f32(recv + (uint32_t)((r * W + j0 + g) * BM + row) * 4u);
+                    q[g] = acc;
+                }
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const int gp = ntile * BN + ks * W + j0 + g;
+                    if (gp >= nbatch) continue;
+                    const int64_t idx = (int64_t)gp * n + gi;
+                    diff[idx] = fmaf(old[g], q[g], -mg[g]);
+                    if (update) {
+                        const float nv = eta == 1.f ? mg[g] / q[g] : fmaf(eta, mg[g] / q[g], (1.f - eta) * old[g]);
+                        out[idx] = nv;
+                        __nv_bfloat16 hi, lo;
+                        split_bf16(nv, hi, lo);
+                        const int64_t ti = tiled_index(gp, gi, kblocks);
+                        op_hi[ti] = hi;
+                        op_lo[ti] = lo;
+                        if (!(nv > 0.f) || isinf(nv)) status->nonfinite = 1;
+                    }
+                }
+            }
+        }
+    }
+    if (warp < 2) { // the two issuing warps take part in both cluster barriers
+        __syncwarp();
+        cluster_sync_all();
+        cluster_sync_all();
     }
     if (!ok) status->timeout = 1;
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
-    }
-}
-
-// ---- epilogue over the partial tiles -----------------------------------------------------
-__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
-    hi = __float2bfloat16_rn(x);
-    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
-}
-
-// blockIdx.x = (ntile * mtiles + mtile) * 16 + slice: 1024 outputs per CTA, 4 consecutive rows per thread.
-__global__ void __launch_bounds__(256)
-batched_tc_finish_kernel(const float *__restrict__ partials, int ksplit, int n, int nbatch, int kblocks, int mtiles,
-                         const float *__restrict__ marg, float *__restrict__ out, float *__restrict__ diff,
-                         __nv_bfloat16 *__restrict__ op_hi, __nv_bfloat16 *__restrict__ op_lo, int update, float eta,
-                         FsDeviceStatus *status) {
-    const int tile = blockIdx.x >> 4, slice = blockIdx.x & 15;
-    const int mtile = tile % mtiles, ntile = tile / mtiles;
-    const int e = (slice * 256 + threadIdx.x) * 4; // element index inside the 128 x 128 tile, [p][i] order
-    const int p = e / BM, i = e % BM;
-    const int gi = mtile * BM + i, gp = ntile * BN + p;
-    if (gi >= n || gp >= nbatch) return;
-    const float *base = partials + (size_t)tile * ksplit * (BM * BN) + e;
-    float4 q = *reinterpret_cast<const float4 *>(base);
-    for (int k = 1; k < ksplit; ++k) {
-        const float4 t = *reinterpret_cast<const float4 *>(base + (size_t)k * (BM * BN));
-        q.x += t.x, q.y += t.y, q.z += t.z, q.w += t.w;
-    }
-    const float qs[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        if (gi + j >= n) break;
-        const int64_t idx = (int64_t)gp * n + gi + j;
-        const float mg = marg[idx], old = out[idx];
-        diff[idx] = fmaf(old, qs[j], -mg);
-        if (update) {
-            const float nv = eta == 1.f ? mg / qs[j] : fmaf(eta, mg / qs[j], (1.f - eta) * old);
-            out[idx] = nv;
-            __nv_bfloat16 hi, lo;
-            split_bf16(nv, hi, lo);
-            op_hi[tiled_index(gp, gi + j, kblocks)] = hi;
-            op_lo[tiled_index(gp, gi + j, kblocks)] = lo;
-            if (!(nv > 0.f) || isinf(nv)) status->nonfinite = 1;
-        }
     }
 }
 
@@ -381,11 +423,50 @@ bool make_map(CUtensorMap *map, const __nv_bfloat16 *ptr, int64_t rows, int64_t 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+void fill_launch(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int ks, int mtiles, int ntiles, cudaStream_t st) {
+    cfg.gridDim = dim3((unsigned)mtiles, (unsigned)ks, (unsigned)ntiles);
+    cfg.blockDim = dim3(kTcThreads, 1, 1);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = st;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1, attr[0].val.clusterDim.y = (unsigned)ks, attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr, cfg.numAttrs = 1;
+}
+
+const void *kernel_for(int ks) {
+    switch (ks) {
+    case 1: return reinterpret_cast<const void *>(batched_tc_kernel<1>);
+    case 2: return reinterpret_cast<const void *>(batched_tc_kernel<2>);
+    case 4: return reinterpret_cast<const void *>(batched_tc_kernel<4>);
+    default: return reinterpret_cast<const void *>(batched_tc_kernel<8>);
+    }
+}
+
+bool set_smem_attr(int ks) {
+    return cudaFuncSetAttribute(kernel_for(ks), cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
+}
+
+// true when at least one cluster of `ks` CTAs of this kernel can be resident
+bool cluster_fits(int ks, int mtiles, int ntiles) {
+    if (!set_smem_attr(ks)) {
+        cudaGetLastError();
+        return false;
+    }
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    fill_launch(cfg, attr, ks, mtiles, ntiles, nullptr);
+    int nclusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&nclusters, kernel_for(ks), &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return nclusters >= 1;
+}
+
 void tc_free(TcState *t) {
     if (!t) return;
     cudaFree(t->K_hi), cudaFree(t->K_lo), cudaFree(t->Kt_hi), cudaFree(t->Kt_lo);
     cudaFree(t->U_hi), cudaFree(t->U_lo), cudaFree(t->V_hi), cudaFree(t->V_lo);
-    cudaFree(t->partials);
     delete t;
 }
 
@@ -403,19 +484,20 @@ void *fsk_tc_create(const float *K, int64_t ld, int64_t n, int nbatch, cudaStrea
     t->rows_pad = (n + BM - 1) / BM * BM;
     t->nb_pad = (nbatch + BN - 1) / BN * BN;
     t->mtiles = (int)(t->rows_pad / BM), t->ntiles = t->nb_pad / BN, t->kblocks = (int)(t->ldb / BK);
-    int ks = 148 / (t->mtiles * t->ntiles);
-    if (ks < 1) ks = 1;
-    if (ks > t->kblocks) ks = t->kblocks;
-    if (ks > 16) ks = 16;
+    // split of the contraction range = cluster size: the largest power of two (at most 8, the portable cluster
+    // limit) that keeps all CTAs in one wave and that the device can co-schedule
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int ks = 1;
+    while (ks < 8 && 2 * ks * t->mtiles * t->ntiles <= sms && 2 * ks <= t->kblocks) ks *= 2;
+    while (ks > 1 && !cluster_fits(ks, t->mtiles, t->ntiles)) ks /= 2;
     t->ksplit = ks;
     const size_t mat_bytes = (size_t)t->rows_pad * t->ldb * 2, vec_bytes = (size_t)t->nb_pad * t->ldb * 2;
-    const size_t part_bytes = (size_t)t->mtiles * t->ntiles * t->ksplit * BM * BN * sizeof(float);
     bool ok = true;
     __nv_bfloat16 **mats[4] = {&t->K_hi, &t->K_lo, &t->Kt_hi, &t->Kt_lo};
     __nv_bfloat16 **vecs[4] = {&t->U_hi, &t->U_lo, &t->V_hi, &t->V_lo};
     for (auto m : mats) ok = ok && cudaMalloc(m, mat_bytes) == cudaSuccess && cudaMemsetAsync(*m, 0, mat_bytes, st) == cudaSuccess;
     for (auto v : vecs) ok = ok && cudaMalloc(v, vec_bytes) == cudaSuccess && cudaMemsetAsync(*v, 0, vec_bytes, st) == cudaSuccess;
-    ok = ok && cudaMalloc(&t->partials, part_bytes) == cudaSuccess;
     if (ok) {
         dim3 grid((unsigned)((n + 31) / 32), (unsigned)((n + 31) / 32));
         split_matrix_kernel<<<grid, 256, 0, st>>>(K, ld, (int)n, t->kblocks, t->K_hi, t->K_lo, t->Kt_hi, t->Kt_lo);
@@ -425,7 +507,7 @@ void *fsk_tc_create(const float *K, int64_t ld, int64_t n, int nbatch, cudaStrea
          make_map(&t->tmKt_hi, t->Kt_hi, t->rows_pad, t->ldb) && make_map(&t->tmKt_lo, t->Kt_lo, t->rows_pad, t->ldb) &&
          make_map(&t->tmU_hi, t->U_hi, t->nb_pad, t->ldb) && make_map(&t->tmU_lo, t->U_lo, t->nb_pad, t->ldb) &&
          make_map(&t->tmV_hi, t->V_hi, t->nb_pad, t->ldb) && make_map(&t->tmV_lo, t->V_lo, t->nb_pad, t->ldb);
-    ok = ok && cudaFuncSetAttribute(batched_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
+    ok = ok && set_smem_attr(t->ksplit);
     if (!ok) {
         cudaGetLastError();
         tc_free(t);
@@ -442,18 +524,20 @@ void fsk_tc_refresh(void *tc, const float *u, const float *v, cudaStream_t st) {
     if (v) split_vectors_kernel<<<grid, 256, 0, st>>>(v, (int)t->n, t->nbatch, t->kblocks, t->V_hi, t->V_lo);
 }
 
-// One batched pass on the tensor-core engine; two launches.
+// One batched pass on the tensor-core engine: one launch (clusters of `ksplit` CTAs).
 void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float *diff, int update, float eta,
                  FsDeviceStatus *status, cudaStream_t st) {
     TcState *t = static_cast<TcState *>(tc);
-    dim3 grid((unsigned)t->mtiles, (unsigned)t->ksplit, (unsigned)t->ntiles);
-    if (!transposed)
-        batched_tc_kernel<<<grid, kTcThreads, SMEM_BYTES, st>>>(t->tmK_hi, t->tmK_lo, t->tmV_hi, t->tmV_lo, t->partials,
-                                                              t->kblocks, t->ksplit, status);
-    else
-        batched_tc_kernel<<<grid, kTcThreads, SMEM_BYTES, st>>>(t->tmKt_hi, t->tmKt_lo, t->tmU_hi, t->tmU_lo, t->partials,
-                                                              t->kblocks, t->ksplit, status);
-    batched_tc_finish_kernel<<<(unsigned)(t->mtiles * t->ntiles * 16), 256, 0, st>>>(t->partials, t->ksplit, (int)t->n, t->nbatch, t->kblocks, t->mtiles, marg, out, diff,
-                                                   transposed ? t->V_hi : t->U_hi, transposed ? t->V_lo : t->U_lo, update, eta,
-                                                   status);
+    const CUtensorMap &a_hi = transposed ? t->tmKt_hi : t->tmK_hi, &a_lo = transposed ? t->tmKt_lo : t->tmK_lo;
+    const CUtensorMap &b_hi = transposed ? t->tmU_hi : t->tmV_hi, &b_lo = transposed ? t->tmU_lo : t->tmV_lo;
+    __nv_bfloat16 *op_hi = transposed ? t->V_hi : t->U_hi, *op_lo = transposed ? t->V_lo : t->U_lo;
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    fill_launch(cfg, attr, t->ksplit, t->mtiles, t->ntiles, st);
+    switch (t->ksplit) {
+    case 1: cudaLaunchKernelEx(&cfg, batched_tc_kernel<1>, a_hi, a_lo, b_hi, b_lo, t->kblocks, (int)t->n, t->nbatch, marg, out, diff, op_hi, op_lo, update, eta, status); break;
+    case 2: cudaLaunchKernelEx(&cfg, batched_tc_kernel<2>, a_hi, a_lo, b_hi, b_lo, t->kblocks, (int)t->n, t->nbatch, marg, out, diff, op_hi, op_lo, update, eta, status); break;
+    case 4: cudaLaunchKernelEx(&cfg, batched_tc_kernel<4>, a_hi, a_lo, b_hi, b_lo, t->kblocks, (int)t->n, t->nbatch, marg, out, diff, op_hi, op_lo, update, eta, status); break;
+    default: cudaLaunchKernelEx(&cfg, batched_tc_kernel<8>, a_hi, a_lo, b_hi, b_lo, t->kblocks, (int)t->n, t->nbatch, marg, out, diff, op_hi, op_lo, update, eta, status); break;
+    }
 }
