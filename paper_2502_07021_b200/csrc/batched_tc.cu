@@ -41,7 +41,7 @@ constexpr int TILE_BYTES = BM * BK * 2;     // one operand tile: 128 rows of 128
 constexpr int STAGE_BYTES = 4 * TILE_BYTES; // A_hi, A_lo, B_hi, B_lo
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 128;
 constexpr int NUM_BARS = 2 * STAGES + 4;    // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 320;          // TMA warp, MMA warp, eight epilogue warps
 constexpr int TMEM_COLS = 256;              // two 128-column fp32 accumulators
 constexpr int CHUNK_KB = 8;                 // k-blocks accumulated in TMEM before the chunk is drained
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -151,6 +151,15 @@ __device__ __forceinline__ float ld_shared_f32(uint32_t addr) {
     asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
     return v;
 }
+__device__ __forceinline__ void st_shared_b16(uint32_t addr, __nv_bfloat16 v) {
+    asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(__bfloat16_as_ushort(v)) : "memory");
+}
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -196,7 +205,7 @@ batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_const
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full + 8 * b, 1);
-            mbar_init(acc_empty + 8 * b, 4); // one arrival per epilogue warp
+            mbar_init(acc_empty + 8 * b, 8); // one arrival per epilogue warp
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -260,22 +269,40 @@ batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_const
             }
         }
     } else {
-        // epilogue warps 2..5: TMEM lane quarter = warp % 4; running sums of the chunks in registers
-        const int quarter = warp & 3;
+        // epilogue warps 2..9: TMEM lane quarter = warp % 4 (the lanes a warp may read), column half = (warp - 2) / 4;
+        // each thread keeps the running sums of one output row x 64 problems in registers
+        const int quarter = warp & 3, half = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;
-        float sum[BN];
+        constexpr int HN = BN / 2;
+        float sum[HN];
 #pragma unroll
-        for (int j = 0; j < BN; ++j) sum[j] = 0.f;
+        for (int j = 0; j < HN; ++j) sum[j] = 0.f;
         const int nchunks = (nkb + CHUNK_KB - 1) / CHUNK_KB;
+        constexpr int WH = W / 2 > 0 ? W / 2 : 1; // problems per thread in the final update (W >= 16 here)
         for (int c = 0; c < nchunks && ok; ++c) {
             const int buf = c & 1;
+            if (c == nchunks - 1) {
+                // the final update's operands (marginal and old scaling of this thread's problems) are asked
+                // into L2 while the last chunk is being computed
+                const int gi_pf = mtile * BM + row;
+                if (lane == 0 && gi_pf < n) {
+#pragma unroll 4
+                    for (int jj = 0; jj < WH; ++jj) {
+                        const int gp = ntile * BN + ks * W + half * WH + jj;
+                        if (gp < nbatch) {
+                            prefetch_l2(marg + (int64_t)gp * n + gi_pf);
+                            prefetch_l2(out + (int64_t)gp * n + gi_pf);
+                        }
+                    }
+                }
+            }
             ok = mbar_wait(acc_full + 8 * buf, (uint32_t)(c >> 1) & 1u);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + half * HN);
 #pragma unroll
-            for (int cc = 0; cc < BN / 32; ++cc) {
+            for (int cc = 0; cc < HN / 32; ++cc) {
                 float v[32];
                 tmem_ld32(taddr + (uint32_t)(cc * 32), v);
 #pragma unroll
@@ -289,48 +316,78 @@ batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_const
         // ring are complete), so stage 0 of every ring can take the partial sums.
         cluster_sync_all();
         const uint32_t recv = base; // [KS][W][BM] floats = 64 KB = one ring stage
+        const uint32_t stage_hi = base + STAGE_BYTES, stage_lo = stage_hi + (uint32_t)(2 * W * BK * 2);
+        if (KS == 1) {
 #pragma unroll
-        for (int q = 0; q < KS; ++q) {
-            const uint32_t dst = map_to_cta(recv + (uint32_t)((ks * W) * BM + row) * 4u, (uint32_t)q);
+            for (int jj = 0; jj < HN; ++jj) st_cluster_f32(recv + (uint32_t)((half * HN + jj) * BM + row) * 4u, sum[jj]);
+        } else {
+            // column j = half * 64 + jj of the tile belongs to rank j / W, as its problem j % W
+            constexpr int RPH = HN / W > 0 ? HN / W : 1; // ranks served by one column half
 #pragma unroll
-            for (int jj = 0; jj < W; ++jj) st_cluster_f32(dst + (uint32_t)(jj * BM) * 4u, sum[q * W + jj]);
+            for (int qq = 0; qq < RPH; ++qq) {
+                const uint32_t dst = map_to_cta(recv + (uint32_t)((ks * W) * BM + row) * 4u, (uint32_t)(half * RPH + qq));
+#pragma unroll
+                for (int jj = 0; jj < W && jj < HN; ++jj) st_cluster_f32(dst + (uint32_t)(jj * BM) * 4u, sum[(qq * W + jj) % HN]);
+            }
         }
-        // Barrier 2: all contributions have landed (release / acquire at cluster scope).
-        cluster_sync_all();
+        // The marginal and the old scaling of this thread's problems are fetched before the second barrier so
+        // that their latency overlaps the exchange.  Barrier 2: all contributions have landed (release /
+        // acquire at cluster scope).
         const int gi = mtile * BM + row;
-        if (ok && gi < n) {
-            constexpr int G = 8; // problems handled together so that their loads are in flight at once
+        const bool act = ok && gi < n;
+        constexpr int G = WH < 32 ? WH : 32; // problems per batch: 2 G values in registers (the sums are dead by now)
 #pragma unroll 1
-            for (int j0 = 0; j0 < W; j0 += G) {
-                float q[G], mg[G], old[G];
+        for (int j0 = 0; j0 < WH; j0 += G) {
+            float mg[G], old[G];
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const int gp = ntile * BN + ks * W + j0 + g;
+            for (int g = 0; g < G; ++g) {
+                const int gp = ntile * BN + ks * W + half * WH + j0 + g;
+                const int64_t idx = (int64_t)gp * n + gi;
+                const bool live = act && gp < nbatch;
+                mg[g] = live ? __ldg(marg + idx) : 1.f;
+                old[g] = live ? out[idx] : 1.f;
+            }
+            if (j0 == 0) cluster_sync_all();
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const int pj = half * WH + j0 + g; // problem of this rank, 0..W-1
+                const int gp = ntile * BN + ks * W + pj;
+                __nv_bfloat16 hi = __float2bfloat16_rn(0.f), lo = hi; // padding rows and problems stay zero
+                if (act && gp < nbatch) {
+                    float q = ld_shared_f32(recv + (uint32_t)(pj * BM + row) * 4u);
+#pragma unroll
+                    for (int r = 1; r < KS; ++r) q += ld_shared_f32(recv + (uint32_t)((r * W + pj) * BM + row) * 4u);
                     const int64_t idx = (int64_t)gp * n + gi;
-                    const bool live = gp < nbatch;
-                    mg[g] = live ? marg[idx] : 1.f;
-                    old[g] = live ? out[idx] : 1.f;
-                    float acc = ld_shared_f32(recv + (uint32_t)((j0 + g) * BM + row) * 4u);
-#pragma unroll
-                    for (int r = 1; r < KS; ++r) acc += ld_shared_f32(recv + (uint32_t)((r * W + j0 + g) * BM + row) * 4u);
-                    q[g] = acc;
-                }
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const int gp = ntile * BN + ks * W + j0 + g;
-                    if (gp >= nbatch) continue;
-                    const int64_t idx = (int64_t)gp * n + gi;
-                    diff[idx] = fmaf(old[g], q[g], -mg[g]);
+                    diff[idx] = fmaf(old[g], q, -mg[g]);
                     if (update) {
-                        const float nv = eta == 1.f ? mg[g] / q[g] : fmaf(eta, mg[g] / q[g], (1.f - eta) * old[g]);
+                        const float nv = eta == 1.f ? mg[g] / q : fmaf(eta, mg[g] / q, (1.f - eta) * old[g]);
                         out[idx] = nv;
-                        __nv_bfloat16 hi, lo;
                         split_bf16(nv, hi, lo);
-                        const int64_t ti = tiled_index(gp, gi, kblocks);
-                        op_hi[ti] = hi;
-                        op_lo[ti] = lo;
                         if (!(nv > 0.f) || isinf(nv)) status->nonfinite = 1;
                     }
+                }
+                // the new operand terms are collected in shared memory (ring stage 1, idle by now) in the
+                // layout of the operand tiles: [k-block of the row][problem][row % 64]
+                const uint32_t so = (uint32_t)((((row >> 6) * W + pj) * BK + (row & 63)) * 2);
+                st_shared_b16(stage_hi + so, hi);
+                st_shared_b16(stage_lo + so, lo);
+            }
+        }
+        if (update) {
+            // The W problems x 64 rows of one k-block are W * 128 consecutive bytes of the tiled operand:
+            // written with 16-byte stores, 512 consecutive bytes per warp instruction.
+            asm volatile("bar.sync 1, 256;" ::: "memory"); // the eight epilogue warps
+            const int et = threadIdx.x - 64;               // 0..255
+#pragma unroll
+            for (int kbl = 0; kbl < 2; ++kbl) {
+                const int kb = 2 * mtile + kbl;
+                if (kb >= kblocks) continue;
+                const int64_t elem = (((int64_t)ntile * kblocks + kb) * BN + ks * W) * BK;
+                uint4 *g_hi = reinterpret_cast<uint4 *>(op_hi + elem), *g_lo = reinterpret_cast<uint4 *>(op_lo + elem);
+                const uint32_t s_hi = stage_hi + (uint32_t)(kbl * W * BK * 2), s_lo = stage_lo + (uint32_t)(kbl * W * BK * 2);
+                for (int v = et; v < W * BK * 2 / 16; v += 256) {
+                    g_hi[v] = ld_shared_v4(s_hi + (uint32_t)v * 16u);
+                    g_lo[v] = ld_shared_v4(s_lo + (uint32_t)v * 16u);
                 }
             }
         }

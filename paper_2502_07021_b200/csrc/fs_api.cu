@@ -30,6 +30,7 @@ constexpr double kLog2e = 1.4426950408889634;
 constexpr int kGraphChunk = 64;
 constexpr int kTraceCap = 1 << 16;
 constexpr int64_t kFusedAutoMinN = 6144;
+constexpr int64_t kFusedLogAutoMinN = 8192;
 constexpr int64_t kPersistentAutoMaxN = 5120; // K of at most 105 MB: inside the 126 MB L2
 constexpr int kTcMinBatch = 32;
 constexpr int kTcMinN = 512;
@@ -161,10 +162,11 @@ void enqueue_col(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
 bool use_fused(const fs_solver *s) {
     if (!s->fused.enabled || s->fused_mode == 0) return false;
     if (s->fused_mode == 2) return true;
-    // automatic: only where it is measured faster.  The log-domain fused kernel is bound by instruction
-    // issue and the ex2 unit rather than by HBM (440 us against 327 us for the two passes at n = 16384),
-    // so it is opt-in.
-    return s->domain == FS_DOMAIN_SCALING && s->n >= kFusedAutoMinN;
+    // automatic: only where it is measured faster.  The log-domain fused iteration costs six launches
+    // (fused kernels, guarded two-pass kernels, commit) and wins from n = 8192 on (n = 16384: 260 us per
+    // iteration against 349 us for the two passes; n = 4096: 41 against 34 us).
+    if (s->domain == FS_DOMAIN_LOG) return s->n >= kFusedLogAutoMinN;
+    return s->n >= kFusedAutoMinN;
 }
 
 void enqueue_fused_rows(fs_solver *s, cudaStream_t st, int64_t &launches) {
