@@ -74,7 +74,7 @@ enum {
                                columns, row tiles of at most H <= 256 rows */
     FS_OPT_FUSED = 5,       /* single-read fused iteration in fs_iterate (scaling or log domain, one problem, 16-byte
                                aligned matrix, n a multiple of 4): 0 = never, 1 = automatic (default: scaling domain with
-                               n >= 6144; log domain with 8192 <= n <= 16384, where a whole row fits one stage),
+                               n >= 6144; log domain with 4096 <= n <= 16384, where a whole row fits one stage),
                                2 = whenever it applies (FS_ERR_UNSUPPORTED if it does not) */
     FS_OPT_RESIDENT = 6,    /* K-resident persistent kernel for small n (scaling domain, one problem, K fits the shared
                                memory of one cluster: n <= ~590 with 8 CTAs, ~720 with 16; used by fs_iterate when no

@@ -16,19 +16,23 @@
 // the same tiled layout by the epilogue that produces it.  Both passes use the same K-major kernel: the column pass reads a transposed
 // split copy of K made at set-up.
 //
-// Kernel: one CTA per (128-row tile of the output, split of the contraction range).  Warp 0
-// issues TMA tile loads (128 x 64 bf16, 128-byte swizzle) into a 3-stage shared-memory ring,
-// warp 1 issues the tcgen05.mma instructions (M = N = 128, K = 16, three per k-step) into a
-// 128-column TMEM accumulator and releases ring slots with tcgen05.commit, warps 2-5 read the
-// accumulator back with tcgen05.ld and store the fp32 partial tile.  The tensor core adds into its
-// fp32 accumulator without round-to-nearest, a bias that grows with the number of accumulated
-// MMAs (a uniform ~2e-5 relative deficit was measured after the 6144 MMAs of a full n = 8192
-// contraction in one accumulator); so the contraction is cut into chunks of 8 k-blocks (96 MMAs)
-// that alternate between two TMEM accumulators, and the epilogue warps add each finished chunk
-// into fp32 registers with round-to-nearest while the next chunk is being computed.  A second small kernel adds
-// the partial tiles of the splits in a fixed order and applies the divide, the marginal residual
-// and the bf16 re-split of the new scalings.  Every mbarrier wait is bounded: on expiry the
-// kernel raises a status flag, stops issuing work, drains what it had in flight and exits.
+// Kernel: one CTA per (128-row tile of the output, split of the contraction range); the KS CTAs that
+// split one tile form a thread-block cluster.  Warp 0 issues TMA tile loads (128 x 64 bf16, 128-byte
+// swizzle) into a 3-stage shared-memory ring, warp 1 issues the tcgen05.mma instructions (M = N = 128,
+// K = 16, three per k-step) into a 128-column TMEM accumulator and releases ring slots with
+// tcgen05.commit, warps 2-9 read the accumulator back with tcgen05.ld (two warps per TMEM lane quarter,
+// 64 columns each).  The tensor core adds into its fp32 accumulator without round-to-nearest, a bias
+// that grows with the number of accumulated MMAs (a uniform ~2e-5 relative deficit was measured after
+// the 6144 MMAs of a full n = 8192 contraction in one accumulator); so the contraction is cut into
+// chunks of 8 k-blocks (96 MMAs) that alternate between two TMEM accumulators, and the epilogue warps
+// add each finished chunk into fp32 registers with round-to-nearest while the next chunk is being
+// computed.  After the main loop the CTAs of a cluster exchange their partial tiles through distributed
+// shared memory (each rank receives the columns of its 128 / KS problems from every rank into an idle
+// ring stage), add them in rank order and apply the divide, the marginal residual and the bf16 re-split
+// of the new scalings; the re-split operand is collected in shared memory and written with 16-byte
+// stores.  One launch per pass; nothing but K, the operand and the result vectors touches HBM.  Every
+// mbarrier wait is bounded: on expiry the kernel raises a status flag, stops issuing work, drains what it
+// had in flight and still takes part in the cluster barriers before it exits.
 #include <cuda.h>
 #include <cuda_bf16.h>
 

@@ -30,7 +30,7 @@ constexpr double kLog2e = 1.4426950408889634;
 constexpr int kGraphChunk = 64;
 constexpr int kTraceCap = 1 << 16;
 constexpr int64_t kFusedAutoMinN = 6144;
-constexpr int64_t kFusedLogAutoMinN = 8192;
+constexpr int64_t kFusedLogAutoMinN = 4096;
 constexpr int64_t kPersistentAutoMaxN = 5120; // K of at most 105 MB: inside the 126 MB L2
 constexpr int kTcMinBatch = 32;
 constexpr int kTcMinN = 512;
@@ -124,7 +124,7 @@ bool use_tc(const fs_solver *s) { return s->tc != nullptr && s->batch_engine != 
 void enqueue_row(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
     if (s->nbatch > 1 && use_tc(s)) {
         fsk_tc_pass(s->tc, 0, s->a, s->x, s->rowdiff, update, s->eta, s->status, st);
-        launches += 2;
+        launches += 1;
     } else if (s->nbatch > 1) {
         fsk_batched_pass_fma(s->mat, s->mat_ld, s->n, s->nbatch, 0, s->y, s->a, s->x, s->rowdiff, update, s->eta, s->status,
                              st);
@@ -142,7 +142,7 @@ void enqueue_row(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
 void enqueue_col(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
     if (s->nbatch > 1 && use_tc(s)) {
         fsk_tc_pass(s->tc, 1, s->b, s->y, s->coldiff, update, s->eta, s->status, st);
-        launches += 2;
+        launches += 1;
     } else if (s->nbatch > 1) {
         fsk_batched_pass_fma(s->mat, s->mat_ld, s->n, s->nbatch, 1, s->x, s->b, s->y, s->coldiff, update, s->eta, s->status,
                              st);
@@ -163,8 +163,8 @@ bool use_fused(const fs_solver *s) {
     if (!s->fused.enabled || s->fused_mode == 0) return false;
     if (s->fused_mode == 2) return true;
     // automatic: only where it is measured faster.  The log-domain fused iteration costs six launches
-    // (fused kernels, guarded two-pass kernels, commit) and wins from n = 8192 on (n = 16384: 260 us per
-    // iteration against 349 us for the two passes; n = 4096: 41 against 34 us).
+    // (fused kernels, guarded two-pass kernels, commit) and wins from n = 4096 on (n = 16384: 204 us per
+    // iteration against 349 us for the two passes; n = 4096: 31 against 34 us; n = 2048: 28 against 16 us).
     if (s->domain == FS_DOMAIN_LOG) return s->n >= kFusedLogAutoMinN;
     return s->n >= kFusedAutoMinN;
 }
