@@ -296,6 +296,22 @@ def test_batched_engines_agree(n, nb):
     assert rel_err(res[2][0], res[1][0]) < 5e-5 and rel_err(res[2][1], res[1][1]) < 5e-5
 
 
+@pytest.mark.parametrize("n,nb", [(1024, 128), (4000, 100), (640, 1300), (1100, 1030)])
+def test_batched_tensor_core_cluster_sizes(n, nb):
+    """The tensor-core engine splits the contraction over a cluster of 8, 4, 2 or 1 CTAs depending on the
+    number of output tiles (here: 8 tiles -> 8, 32 -> 4, 5 x 11 -> 2, 9 x 9 -> 1); every size goes through
+    the exchange and the in-kernel update, with ragged row and problem tiles, and must match the oracle on
+    sampled problems (the problems of a batch are independent)."""
+    w = workloads.make(5, n=n, nbatch=nb)
+    with GpuSolver(w.K, KK, w.eps, w.a, w.b, w.offsets, SC) as g:
+        g.iterate(10)
+        U, V = g.scalings()
+        row, col = g.errors(1)
+    assert np.all(np.isfinite(U)) and np.all(U > 0) and np.all(np.isfinite(V)) and np.all(V > 0)
+    assert row.shape == (nb,) and np.all(col < 1e-5)      # right after a column update its marginal is exact
+    batched_sample(w, U, V, 10, sorted({0, 1, 63, 64, nb // 2, nb - 2, nb - 1}))
+
+
 def test_batched_tensor_core_engine_converges():
     w = workloads.make(5, n=1024, nbatch=64)
     check_converged(w, w.iters, w.C, problems=(0, 33, 63))
