@@ -312,7 +312,17 @@ FsFusedPlan fsk_fused_plan(int64_t n, bool vec) {
     default: nc = query_clusters<16, 1>(S, ns); break;
     }
     if (nc < 1) return p;
-    p.enabled = true, p.S = S, p.F = F, p.R = R, p.nstages = ns, p.nclusters = nc, p.tile_rows = 32;
+    // Row tiles are dealt round-robin to the clusters, so the busiest cluster gets ceil(tiles / clusters) of them:
+    // the tile height (a multiple of R, at most 32) is the one that gives it the fewest rows (n = 8192 on 74
+    // clusters: 16 rows -> 112 rows, where 32 rows -> 128 rows against an average of 110.7).
+    int best = 32;
+    int64_t best_rows = INT64_MAX;
+    for (int tr = 32; tr >= R && tr >= 4; tr >>= 1) {
+        const int64_t tiles = (n + tr - 1) / tr;
+        const int64_t rows = (tiles + nc - 1) / nc * tr;
+        if (rows * 50 < best_rows * 49) best_rows = rows, best = tr; // a smaller tile must save more than 2 %
+    }
+    p.enabled = true, p.S = S, p.F = F, p.R = R, p.nstages = ns, p.nclusters = nc, p.tile_rows = best;
     return p;
 }
 
