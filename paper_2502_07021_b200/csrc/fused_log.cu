@@ -365,8 +365,8 @@ FsFusedPlan fsk_fused_log_plan(int64_t n, bool vec) {
     // the fewest rows -- at n = 16384, 16 rows (7 tiles = 112 rows) rather than 32 (4 tiles = 128 rows against
     // an average of 110.7).
     int best = 32;
-    int64_t best_rows = INT64_MAX;
-    for (int tr = 32; tr >= R && tr >= 4; tr >>= 1) {
+    int64_t best_rows = ((n + 31) / 32 + nc - 1) / nc * 32;
+    for (int tr = 16; tr >= R && tr >= 4; tr >>= 1) {
         const int64_t tiles = (n + tr - 1) / tr;
         const int64_t rows = (tiles + nc - 1) / nc * tr;
         if (rows * 50 < best_rows * 49) best_rows = rows, best = tr; // a smaller tile must save more than 2 %
