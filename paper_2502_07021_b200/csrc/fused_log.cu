@@ -199,16 +199,21 @@ fused_log_iteration_kernel(const float *__restrict__ C, int64_t ld, int n, int n
             __syncthreads();
             if (fail_s) { ok = false; break; }
             if (t == 0) producer_issue();
-            // ---- row factor a_i / s_i (lane w holds the sum of warp w; a fixed butterfly gives every lane the
-            //      same total), column sums from the e kept in registers
+            // ---- row factor a_i / s_i, column sums from the e kept in registers
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 float wi = 0.f;
                 if (r < cnt) {
-                    float si = lane < kWarpsLog ? rb[r * kWarpsLog + lane] : 0.f;
+                    // every thread adds the per-warp sums itself, in a fixed order (broadcast 128-bit reads: shorter
+                    // than a second shuffle butterfly); the factor needs no correctly rounded division
+                    const float4 *rb4 = reinterpret_cast<const float4 *>(rb + r * kWarpsLog);
+                    float si = 0.f;
 #pragma unroll
-                    for (int off = 16; off > 0; off >>= 1) si += __shfl_xor_sync(0xffffffffu, si, off);
-                    wi = ar[r] / si;
+                    for (int q = 0; q < kWarpsLog / 4; ++q) {
+                        const float4 w4 = rb4[q];
+                        si += (w4.x + w4.y) + (w4.z + w4.w);
+                    }
+                    wi = __fdividef(ar[r], si);
                     if (t == 0) {
                         rowdiff[row + r] = si - ar[r]; // s_i is the row marginal of the plan that was read
                         const float xn = fh[r] + __log2f(wi);
