@@ -186,10 +186,11 @@ int64_t fs_iterations_done(const fs_solver *s);
 /* Number of kernel launches this handle has enqueued so far (graph replays count their nodes). */
 int64_t fs_launch_count(const fs_solver *s);
 
-/* Log domain, single-read fused path (FS_OPT_FUSED): number of iterations since creation / fs_reset whose
- * marginals left the safe fp32 range of that path and that were therefore redone by the two-pass kernels
- * (normally the first iteration from a cold start and none after it).  count_out: HOST.  Synchronises the
- * stream.  The paper has no counterpart: it is a diagnostic of this implementation. */
+/* Log domain, single-read fused path (FS_OPT_FUSED): number of iterations since creation / fs_reset in which
+ * a marginal left the safe fp32 range of that path's fast form, so that the rows or columns concerned were
+ * redone inside its kernels with a maximum as stabiliser (normally the first one or two iterations from a cold
+ * start and none after them).  count_out: HOST.  Synchronises the stream.  The paper has no counterpart: it is a
+ * diagnostic of this implementation. */
 int fs_fused_log_fallbacks(fs_solver *s, int64_t *count_out, void *stream);
 
 int fs_destroy(fs_solver *s);

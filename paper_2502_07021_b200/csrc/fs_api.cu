@@ -162,8 +162,7 @@ void enqueue_col(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
 bool use_fused(const fs_solver *s) {
     if (!s->fused.enabled || s->fused_mode == 0) return false;
     if (s->fused_mode == 2) return true;
-    // automatic: only where it is measured faster.  The log-domain fused iteration costs six launches
-    // (fused kernels, guarded two-pass kernels, commit) and wins from n = 4096 on (n = 16384: 204 us per
+    // automatic: only where it is measured faster.  The log-domain fused iteration wins from n = 4096 on (n = 16384: 204 us per
     // iteration against 349 us for the two passes; n = 4096: 31 against 34 us; n = 2048: 28 against 16 us).
     if (s->domain == FS_DOMAIN_LOG) return s->n >= kFusedLogAutoMinN;
     return s->n >= kFusedAutoMinN;
@@ -182,25 +181,13 @@ void enqueue_fused_finish(fs_solver *s, cudaStream_t st, int64_t &launches) {
 
 void enqueue_trace(fs_solver *s, cudaStream_t st, int64_t &launches);
 
-// One log-domain iteration on the single-read path: the fused kernels write the new duals to temporaries;
-// the two-pass kernels follow as guarded launches that do nothing unless the fused iteration left the safe
-// range (then they redo it from the untouched duals); the commit kernel adopts the temporaries otherwise.
+// One log-domain iteration on the single-read path: two launches, duals updated in place.
 void enqueue_fused_log_iteration(fs_solver *s, bool check, cudaStream_t st, int64_t &launches) {
-    float *tmp = s->fused_log_tmp;
-    const size_t n = (size_t)s->n;
-    const int *redo = &s->status->range;
-    fsk_fused_log_iteration(s->fused, s->mat, s->mat_ld, s->n, s->eps, s->fused_tiles_dev, s->fused_ntiles, s->xs, s->ys,
-                            s->a, s->b, tmp, tmp + n, tmp + 2 * n, tmp + 3 * n, s->rowdiff, s->coldiff, s->fused_partials,
-                            s->status, st);
-    fsk_log_row_pass(s->plan, s->mat, s->mat_ld, s->n, s->eps, s->ys, s->a, s->loga, s->x, s->xs, s->rowdiff, 1, s->status,
-                     st, redo);
-    launches += 3;
+    fsk_fused_log_iteration(s->fused, s->mat, s->mat_ld, s->n, s->eps, s->fused_tiles_dev, s->fused_ntiles, s->a, s->b, s->x,
+                            s->xs, s->y, s->ys, s->rowdiff, s->coldiff, s->fused_partials, s->status,
+                            reinterpret_cast<int *>(s->fused_log_tmp), st);
+    launches += 2;
     if (check) enqueue_trace(s, st, launches);
-    fsk_log_col_pass(s->plan, s->mat, s->mat_ld, s->n, s->n_pad, s->eps, s->tiles_dev, (int)s->tiles.size(), s->xs, s->b,
-                     s->logb, s->y, s->ys, s->partials, s->coldiff, 1, s->status, st, redo);
-    fsk_fused_log_commit(s->n, tmp, tmp + n, tmp + 2 * n, tmp + 3 * n, s->x, s->xs, s->y, s->ys, s->status,
-                         reinterpret_cast<int *>(tmp + 4 * n), st);
-    launches += 3;
 }
 
 void enqueue_trace(fs_solver *s, cudaStream_t st, int64_t &launches) {
@@ -396,7 +383,7 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
             FS_CU(cudaMalloc(&s->fused_partials, pbytes));
             FS_CU(cudaMemsetAsync(s->fused_partials, 0, pbytes, st));
             if (domain == FS_DOMAIN_LOG) {
-                const size_t tbytes = sizeof(float) * 4 * (size_t)n + 64;
+                const size_t tbytes = 64; // stage 2's count of finished CTAs
                 FS_CU(cudaMalloc(&s->fused_log_tmp, tbytes));
                 FS_CU(cudaMemsetAsync(s->fused_log_tmp, 0, tbytes, st));
             }

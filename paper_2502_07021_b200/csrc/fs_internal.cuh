@@ -68,8 +68,8 @@ struct FsDeviceStatus {
     int nonfinite;   // set by any kernel that produced a non-finite or non-positive scaling
     int trace_count; // number of trace entries appended so far
     int timeout;     // a bounded device-side wait ran out (tensor-core engine)
-    int range;       // fused log iteration: a marginal left the safe fp32 range; the guarded two-pass kernels redo it
-    int fallbacks;   // number of iterations redone that way
+    int range;       // fused log iteration: a marginal left the safe fp32 range and its row or column was redone
+    int fallbacks;   // number of iterations in which that happened
 };
 
 struct fs_solver {
@@ -110,7 +110,7 @@ struct fs_solver {
     FsRowTile *fused_tiles_dev = nullptr;
     int fused_ntiles = 0;
     float *fused_partials = nullptr;
-    float *fused_log_tmp = nullptr;         // fused log iteration: uncommitted f, xs, g, ys ([4][n]) + a block counter
+    float *fused_log_tmp = nullptr;         // fused log iteration: stage 2's count of finished CTAs (one int)
     int64_t iter_done = 0;
     int64_t launches = 0;
     bool use_graph = true;
@@ -153,11 +153,11 @@ void fsk_col_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, in
 // ys = g * log2(e)/eps on input; writes f and xs = f * log2(e)/eps when update.
 void fsk_log_row_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n, double eps, const float *ys,
                       const float *a, const float *loga, float *f, float *xs, float *rowdiff, int update,
-                      FsDeviceStatus *status, cudaStream_t st, const int *run_if = nullptr);
+                      FsDeviceStatus *status, cudaStream_t st);
 void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n, int64_t n_pad, double eps,
                       const FsRowTile *tiles, int ntiles, const float *xs, const float *b, const float *logb,
                       float *g, float *ys, float *partials, float *coldiff, int update,
-                      FsDeviceStatus *status, cudaStream_t st, const int *run_if = nullptr);
+                      FsDeviceStatus *status, cudaStream_t st);
 // Stage 2 of the column pass alone: r_l = sum over `ntiles` partial rows of pitch n_pad, residual, divide.
 void fsk_col_finish(int64_t n, int64_t n_pad, int ntiles, const float *partials, const float *b, float *v,
                     float *coldiff, int update, float eta, FsDeviceStatus *status, cudaStream_t st);
@@ -188,14 +188,12 @@ cudaError_t fsk_persistent_iterate(const FsPersistentPlan &p, const float *K, in
 
 // ---- fused_log.cu ------------------------------------------------------------------------
 FsFusedPlan fsk_fused_log_plan(int64_t n, bool vec);
-// One fused log-domain iteration (row kernel + stage 2), uncommitted: new duals go to the temporaries.
+// One fused log-domain iteration (row kernel + stage 2), in place; out-of-range rows and columns are redone
+// inside the two kernels.  done_blocks: one zero-initialised int of scratch.
 cudaError_t fsk_fused_log_iteration(const FsFusedPlan &p, const float *C, int64_t ld, int64_t n, double eps,
-                                    const FsRowTile *tiles, int ntiles, const float *xs, const float *ys, const float *a,
-                                    const float *b, float *f_tmp, float *xs_tmp, float *g_tmp, float *ys_tmp,
-                                    float *rowdiff, float *coldiff, float *partials, FsDeviceStatus *status,
-                                    cudaStream_t st);
-void fsk_fused_log_commit(int64_t n, const float *f_tmp, const float *xs_tmp, const float *g_tmp, const float *ys_tmp,
-                          float *f, float *xs, float *g, float *ys, FsDeviceStatus *status, int *done_blocks, cudaStream_t st);
+                                    const FsRowTile *tiles, int ntiles, const float *a, const float *b, float *f, float *xs,
+                                    float *g, float *ys, float *rowdiff, float *coldiff, float *partials,
+                                    FsDeviceStatus *status, int *done_blocks, cudaStream_t st);
 
 // ---- batched.cu --------------------------------------------------------------------------
 // out[p][i] = marg[p][i] / sum_l Mat(i,l) in[p][l], Mat(i,l) = K[i][l] (transposed = 0) or K[l][i].

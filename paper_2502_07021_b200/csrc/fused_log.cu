@@ -11,9 +11,13 @@
 // from C.  s_i is the row marginal of the current plan and r_l the column marginal after the row update,
 // so both stay within a factor exp(+-delta/eps) of a_i, b_l, delta = the change of the duals in one
 // iteration; they leave the fp32 range only from a cold start or after a jump of the duals of more than
-// ~60 eps.  The kernels check s_i and r_l against [2^-90, 2^90]; outside it they raise status->range and
-// the driver's guarded two-pass kernels (running maxima, always safe) redo that iteration from the
-// untouched duals.  Results of this path are written to temporaries and committed only when in range.
+// ~60 eps.  Both are checked against [2^-90, 2^90].  A row whose s_i is outside is redone on the spot by the
+// whole CTA from the copy of the row that is still in shared memory, with the row maximum as stabiliser (two
+// more sweeps: maximum, then sum; its plan entries e_il a_i / s_i are at most a_i, so they always fit).  A
+// column whose r_l is outside is redone by the stage-2 kernel directly from C and the new row duals with a
+// running maximum (a CTA re-reads its 32 columns: n reads of 128 bytes).  Either way the iteration's
+// results are those of the stabilised updates, written in place; status->fallbacks counts the iterations
+// in which this happened (normally the first one or two from a cold start and none after them).
 //
 // Organisation: one persistent CTA of 512 threads per SM owns whole rows (row tiles dealt round-robin; a row
 // of up to 16384 columns fits one shared-memory stage).  Thread 0 doubles as the producer and keeps a ring
@@ -47,16 +51,15 @@ __device__ __forceinline__ bool in_range(float x) { return x >= kRangeLo && x <=
 template <int FT, int R>
 __global__ void __launch_bounds__(kThreadsLog, 1)
 fused_log_iteration_kernel(const float *__restrict__ C, int64_t ld, int n, int nctas, int nstages, float s2, double eps,
-                           const FsRowTile *__restrict__ tiles, int ntiles, const float *__restrict__ xs,
+                           const FsRowTile *__restrict__ tiles, int ntiles, float *xs,
                            const float *__restrict__ ys, const float *__restrict__ a, float *__restrict__ f_out,
-                           float *__restrict__ xs_out, float *__restrict__ rowdiff, float *__restrict__ partials,
-                           FsDeviceStatus *status) {
+                           float *__restrict__ rowdiff, float *__restrict__ partials, FsDeviceStatus *status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t row_bytes = (uint32_t)n * 4u;
     const uint32_t stage_bytes = R * row_bytes;
     const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
-    const uint32_t red = base + (uint32_t)nstages * stage_bytes;   // [2][R][kWarpsLog] floats
-    const uint32_t bar_full = red + 2u * R * kWarpsLog * 4u;
+    const uint32_t red = base + (uint32_t)nstages * stage_bytes;   // [2][R][kWarpsLog] floats, then [2][kWarpsLog] for a redone row
+    const uint32_t bar_full = red + (2u * R + 2u) * kWarpsLog * 4u;
     const float *red_f = reinterpret_cast<const float *>(smem_raw + (red - smem_u32(smem_raw)));
     float *red_w = const_cast<float *>(red_f);
     __shared__ int fail_s;
@@ -198,7 +201,6 @@ fused_log_iteration_kernel(const float *__restrict__ C, int64_t ld, int n, int n
             // which was only read and can be refilled
             __syncthreads();
             if (fail_s) { ok = false; break; }
-            if (t == 0) producer_issue();
             // ---- row factor a_i / s_i, column sums from the e kept in registers
 #pragma unroll
             for (int r = 0; r < R; ++r) {
@@ -213,13 +215,62 @@ fused_log_iteration_kernel(const float *__restrict__ C, int64_t ld, int n, int n
                         const float4 w4 = rb4[q];
                         si += (w4.x + w4.y) + (w4.z + w4.w);
                     }
-                    wi = __fdividef(ar[r], si);
+                    float xn;
+                    if (in_range(si)) { // the same value in every thread, so the branch is uniform over the CTA
+                        wi = __fdividef(ar[r], si);
+                        xn = fh[r] + __log2f(wi);
+                    } else {
+                        // The row is redone from shared memory with the maximum m of t0 = ys_l - C_il log2(e)/eps as
+                        // stabiliser: s' = sum_l 2^(t0 - m), new dual log2(a_i / s') - m, plan entries 2^(t0 - m) a_i / s'.
+                        out_of_range = true;
+                        float *sb = red_w + 2 * R * kWarpsLog; // [2][kWarpsLog]
+                        float m = -INFINITY;
+#pragma unroll
+                        for (int j = 0; j < FT; ++j) {
+                            if (j * kThreadsLog + t < n4) {
+                                const float4 c4 = lds4(st + (uint32_t)r * row_bytes + (uint32_t)j * (kThreadsLog * 16u));
+                                m = fmaxf(m, fmaxf(fmaxf(fmaf(c4.x, ns2, g4[j].x), fmaf(c4.y, ns2, g4[j].y)),
+                                                   fmaxf(fmaf(c4.z, ns2, g4[j].z), fmaf(c4.w, ns2, g4[j].w))));
+                            }
+                        }
+#pragma unroll
+                        for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+                        if (lane == 0) sb[warp] = m;
+                        __syncthreads();
+                        m = sb[0];
+#pragma unroll
+                        for (int q = 1; q < kWarpsLog; ++q) m = fmaxf(m, sb[q]);
+                        float part = 0.f;
+#pragma unroll
+                        for (int j = 0; j < FT; ++j) {
+                            e[j][r] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (j * kThreadsLog + t < n4) {
+                                const float4 c4 = lds4(st + (uint32_t)r * row_bytes + (uint32_t)j * (kThreadsLog * 16u));
+                                float4 x;
+                                x.x = ex2(fmaf(c4.x, ns2, g4[j].x) - m);
+                                x.y = ex2(fmaf(c4.y, ns2, g4[j].y) - m);
+                                x.z = ex2(fmaf(c4.z, ns2, g4[j].z) - m);
+                                x.w = ex2(fmaf(c4.w, ns2, g4[j].w) - m);
+                                e[j][r] = x;
+                                part += (x.x + x.y) + (x.z + x.w);
+                            }
+                        }
+#pragma unroll
+                        for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+                        if (lane == 0) sb[kWarpsLog + warp] = part;
+                        __syncthreads();
+                        float sp = 0.f;
+#pragma unroll
+                        for (int q = 0; q < kWarpsLog; ++q) sp += sb[kWarpsLog + q];
+                        wi = ar[r] / sp; // sp >= 1: the maximum itself contributes 2^0
+                        xn = __log2f(wi) - m;
+                        __syncthreads(); // sb may be rewritten by the next redone row
+                    }
                     if (t == 0) {
                         rowdiff[row + r] = si - ar[r]; // s_i is the row marginal of the plan that was read
-                        const float xn = fh[r] + __log2f(wi);
-                        xs_out[row + r] = xn;
+                        xs[row + r] = xn;
                         f_out[row + r] = (float)((double)xn * eps * 0.6931471805599453);
-                        if (!in_range(si)) out_of_range = true;
+                        if (!(fabsf(xn) <= 3.0e38f)) status->nonfinite = 1;
                     }
                 }
 #pragma unroll
@@ -230,6 +281,8 @@ fused_log_iteration_kernel(const float *__restrict__ C, int64_t ld, int n, int n
                     r4[j].w = fmaf(e[j][r].w, wi, r4[j].w);
                 }
             }
+            // every thread is done with the stage (a redone row re-reads it, hence only now): refill it
+            if (t == 0) producer_issue();
         }
     }
     if (out_of_range) status->range = 1;
@@ -248,15 +301,20 @@ fused_log_iteration_kernel(const float *__restrict__ C, int64_t ld, int n, int n
     }
 }
 
-// Stage 2 of the fused log iteration: r_l = sum of the per-CTA column sums, g_l <- g_l + eps log(b_l / r_l),
-// written to the temporaries; coldiff = r_l - b_l.  A CTA serves 32 columns: thread (c, k) of 32 x 8 adds
-// the rows k, k + 8, ... of the partial matrix for column c (128-byte coalesced reads), and the eight
-// group sums of a column are added in group order -- a fixed order, so the result is reproducible.
+// Stage 2 of the fused log iteration: r_l = sum of the per-CTA column sums, g_l <- g_l + eps log(b_l / r_l);
+// coldiff = r_l - b_l.  A CTA serves 32 columns: thread (c, k) of 32 x 8 adds the rows k, k + 8, ... of the
+// partial matrix for column c (128-byte coalesced reads), and the eight group sums of a column are added in
+// group order -- a fixed order, so the result is reproducible.  If one of its columns has r_l outside the
+// safe range, the CTA recomputes its columns from C and the new row duals: thread (c, k) folds the rows
+// k, k + 8, ... into a running (maximum, sum) pair, the eight pairs of a column are merged in group order,
+// and g_l = eps (log2 b_l - M - log2 S) ln 2 is the stabilised update itself.  The last CTA to finish counts
+// the iteration as a fallback if any row or column was redone, and clears the flag.
 __global__ void __launch_bounds__(256)
-fused_log_finish_kernel(int n, int nclusters, double eps, const float *__restrict__ partials, const float *__restrict__ b,
-                        const float *__restrict__ ys, float *__restrict__ g_out, float *__restrict__ ys_out,
-                        float *__restrict__ coldiff, FsDeviceStatus *status) {
-    __shared__ float part[8][32];
+fused_log_finish_kernel(int n, int nclusters, double eps, float s2, const float *__restrict__ C, int64_t ld,
+                        const float *__restrict__ partials, const float *__restrict__ b, const float *__restrict__ xs,
+                        float *ys, float *__restrict__ g_out, float *__restrict__ coldiff, FsDeviceStatus *status,
+                        int *done_blocks) {
+    __shared__ float part[8][32], pmax[8][32];
     const int c = threadIdx.x & 31, k0 = threadIdx.x >> 5;
     const int l = blockIdx.x * 32 + c;
     float acc = 0.f;
@@ -266,41 +324,56 @@ fused_log_finish_kernel(int n, int nclusters, double eps, const float *__restric
     }
     part[k0][c] = acc;
     __syncthreads();
-    if (k0 != 0 || l >= n) return;
     float r = part[0][c];
 #pragma unroll
     for (int k = 1; k < 8; ++k) r += part[k][c];
-    const float bl = b[l];
-    coldiff[l] = r - bl;
-    const float yn = ys[l] + __log2f(bl / r);
-    ys_out[l] = yn;
-    g_out[l] = (float)((double)yn * eps * 0.6931471805599453);
-    if (!in_range(r)) status->range = 1;
-}
-
-// Commit: when the iteration stayed in range the temporaries become the duals; otherwise the guarded
-// two-pass kernels have already written the duals and only the flag is cleared (and counted).
-__global__ void __launch_bounds__(256)
-fused_log_commit_kernel(int n, const float *__restrict__ f_tmp, const float *__restrict__ xs_tmp,
-                        const float *__restrict__ g_tmp, const float *__restrict__ ys_tmp, float *__restrict__ f,
-                        float *__restrict__ xs, float *__restrict__ g, float *__restrict__ ys, FsDeviceStatus *status,
-                        int *done_blocks) {
-    const int l = blockIdx.x * 256 + threadIdx.x;
-    const bool failed = *reinterpret_cast<volatile int *>(&status->range) != 0;
-    if (!failed && l < n) {
-        f[l] = f_tmp[l];
-        xs[l] = xs_tmp[l];
-        g[l] = g_tmp[l];
-        ys[l] = ys_tmp[l];
+    const bool bad = l < n && !in_range(r);
+    const int any_bad = __syncthreads_or(bad ? 1 : 0); // also orders the reads of part[] before its reuse
+    const float bl = l < n ? b[l] : 1.f;
+    float yn = 0.f;
+    if (!bad && l < n) yn = ys[l] + __log2f(bl / r);
+    if (any_bad) {
+        // running (maximum, sum) of t = xs_i - C_il log2(e)/eps over this thread's rows
+        float m = -INFINITY, sum = 0.f;
+        if (l < n) {
+            for (int i = k0; i < n; i += 8) {
+                const float t = fmaf(__ldg(C + (int64_t)i * ld + l), -s2, __ldg(xs + i));
+                if (t > m) {
+                    sum = sum * ex2(m - t) + 1.f; // first row: 0 * 2^-inf + 1
+                    m = t;
+                } else {
+                    sum += ex2(t - m);
+                }
+            }
+        }
+        pmax[k0][c] = m, part[k0][c] = sum;
+        __syncthreads();
+        float M = pmax[0][c], S = part[0][c];
+#pragma unroll
+        for (int k = 1; k < 8; ++k) {
+            const float mk = pmax[k][c], sk = part[k][c];
+            const float mm = fmaxf(M, mk);
+            S = (M == -INFINITY ? 0.f : S * ex2(M - mm)) + (mk == -INFINITY ? 0.f : sk * ex2(mk - mm));
+            M = mm;
+        }
+        if (bad) yn = __log2f(bl) - M - __log2f(S);
     }
-    // the last block to finish resets the flag for the next iteration (all blocks have read it by then)
+    if (k0 == 0 && l < n) {
+        coldiff[l] = r - bl;
+        ys[l] = yn;
+        g_out[l] = (float)((double)yn * eps * 0.6931471805599453);
+        if (!(fabsf(yn) <= 3.0e38f)) status->nonfinite = 1;
+        if (bad) status->range = 1;
+    }
+    // the last CTA to finish counts and clears the flag (all CTAs have written it by then)
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
         const int prev = atomicAdd(done_blocks, 1);
         if (prev == (int)gridDim.x - 1) {
             *done_blocks = 0;
-            if (failed) {
+            __threadfence();
+            if (*reinterpret_cast<volatile int *>(&status->range) != 0) {
                 status->range = 0;
                 status->fallbacks += 1;
             }
@@ -310,15 +383,15 @@ fused_log_commit_kernel(int n, const float *__restrict__ f_tmp, const float *__r
 }
 
 size_t fused_log_smem_bytes(int64_t n, int R, int nstages) {
-    return (size_t)nstages * R * (size_t)n * 4 + (size_t)2 * R * kWarpsLog * 4 + (size_t)8 * nstages + 256;
+    return (size_t)nstages * R * (size_t)n * 4 + (size_t)(2 * R + 2) * kWarpsLog * 4 + (size_t)8 * nstages + 256;
 }
 
 template <int FT, int R>
 cudaError_t launch_fused_log(const FsFusedPlan &p, cudaStream_t st, const float *C, int64_t ld, int n, float s2, double eps,
-                             const FsRowTile *tiles, int ntiles, const float *xs, const float *ys, const float *a,
-                             float *f_out, float *xs_out, float *rowdiff, float *partials, FsDeviceStatus *status) {
+                             const FsRowTile *tiles, int ntiles, float *xs, const float *ys, const float *a,
+                             float *f_out, float *rowdiff, float *partials, FsDeviceStatus *status) {
     fused_log_iteration_kernel<FT, R><<<(unsigned)p.nclusters, kThreadsLog, fused_log_smem_bytes(n, R, p.nstages), st>>>(
-        C, ld, n, p.nclusters, p.nstages, s2, eps, tiles, ntiles, xs, ys, a, f_out, xs_out, rowdiff, partials, status);
+        C, ld, n, p.nclusters, p.nstages, s2, eps, tiles, ntiles, xs, ys, a, f_out, rowdiff, partials, status);
     return cudaGetLastError();
 }
 
@@ -380,34 +453,30 @@ FsFusedPlan fsk_fused_log_plan(int64_t n, bool vec) {
     return p;
 }
 
-// One fused log-domain iteration, uncommitted: reads the duals (xs, ys scaled copies), writes the new duals
-// to the temporaries, rowdiff / coldiff directly, and raises status->range when a marginal left the safe range.
+// One fused log-domain iteration, in place: the row kernel updates f / xs and writes rowdiff and the per-CTA
+// column partials, stage 2 updates g / ys and writes coldiff.  `done_blocks` is one zero-initialised int of
+// scratch (stage 2's count of finished CTAs; it leaves it zero).
 cudaError_t fsk_fused_log_iteration(const FsFusedPlan &p, const float *C, int64_t ld, int64_t n, double eps,
-                                    const FsRowTile *tiles, int ntiles, const float *xs, const float *ys, const float *a,
-                                    const float *b, float *f_tmp, float *xs_tmp, float *g_tmp, float *ys_tmp,
-                                    float *rowdiff, float *coldiff, float *partials, FsDeviceStatus *status,
-                                    cudaStream_t st) {
+                                    const FsRowTile *tiles, int ntiles, const float *a, const float *b, float *f, float *xs,
+                                    float *g, float *ys, float *rowdiff, float *coldiff, float *partials,
+                                    FsDeviceStatus *status, int *done_blocks, cudaStream_t st) {
     const float s2 = (float)(1.4426950408889634 / eps);
     cudaError_t e;
     switch (p.F) {
-    case 1: e = launch_fused_log<1, 4>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
-    case 2: e = launch_fused_log<2, 4>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
-    case 3: e = launch_fused_log<3, 2>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
-    case 4: e = launch_fused_log<4, 2>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
-    case 5: e = launch_fused_log<5, 1>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
-    case 6: e = launch_fused_log<6, 1>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
-    case 7: e = launch_fused_log<7, 1>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
-    default: e = launch_fused_log<8, 1>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f_tmp, xs_tmp, rowdiff, partials, status); break;
+#define FS_LOG_CASE(F_, R_) \
+    case F_: e = launch_fused_log<F_, R_>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f, rowdiff, partials, status); break;
+        FS_LOG_CASE(1, 4)
+        FS_LOG_CASE(2, 4)
+        FS_LOG_CASE(3, 2)
+        FS_LOG_CASE(4, 2)
+        FS_LOG_CASE(5, 1)
+        FS_LOG_CASE(6, 1)
+        FS_LOG_CASE(7, 1)
+    default: e = launch_fused_log<8, 1>(p, st, C, ld, (int)n, s2, eps, tiles, ntiles, xs, ys, a, f, rowdiff, partials, status); break;
+#undef FS_LOG_CASE
     }
     if (e != cudaSuccess) return e;
-    fused_log_finish_kernel<<<(unsigned)((n + 31) / 32), 256, 0, st>>>((int)n, p.nclusters, eps, partials, b, ys, g_tmp, ys_tmp,
-                                                                         coldiff, status);
+    fused_log_finish_kernel<<<(unsigned)((n + 31) / 32), 256, 0, st>>>((int)n, p.nclusters, eps, s2, C, ld, partials, b, xs, ys, g,
+                                                                       coldiff, status, done_blocks);
     return cudaGetLastError();
-}
-
-// Commits the temporaries (or, after a range failure, leaves the duals the guarded two-pass kernels wrote).
-void fsk_fused_log_commit(int64_t n, const float *f_tmp, const float *xs_tmp, const float *g_tmp, const float *ys_tmp,
-                          float *f, float *xs, float *g, float *ys, FsDeviceStatus *status, int *done_blocks, cudaStream_t st) {
-    fused_log_commit_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>((int)n, f_tmp, xs_tmp, g_tmp, ys_tmp, f, xs, g, ys, status,
-                                                                         done_blocks);
 }

@@ -155,24 +155,19 @@ row_pass_kernel(const float *__restrict__ K, int64_t ld, int n, int nrows, const
 }
 
 // Row pass, log domain.
-template <int L, int R, bool VEC, bool LOOP>
+template <int L, int R, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 log_row_pass_kernel(const float *__restrict__ C, int64_t ld, int n, float s2, double eps,
                     const float *__restrict__ ys, const float *__restrict__ a, const float *__restrict__ loga,
                     float *__restrict__ f, float *__restrict__ xs, float *__restrict__ rowdiff, int update,
-                    FsDeviceStatus *status, const int *run_if, int nblocks) {
-    // guarded launch: the whole grid leaves at once unless *run_if is set (redo of a fused iteration)
-    if (run_if != nullptr && *reinterpret_cast<const volatile int *>(run_if) == 0) return;
+                    FsDeviceStatus *status) {
     constexpr int G = kThreads / L;
     constexpr int W = L / 32;
     constexpr int U = (R >= 4) ? 2 : (R >= 2 ? 4 : 8); // column chunks in flight per thread
     __shared__ float red_m[kThreads / 32][R], red_s[kThreads / 32][R];
 
     const int grp = threadIdx.x / L, lane = threadIdx.x % L;
-    // LOOP (guarded launches): a small grid walks the row blocks; otherwise one block per CTA
-    int bid = blockIdx.x;
-    do {
-    const int row0 = (bid * G + grp) * R;
+    const int row0 = (blockIdx.x * G + grp) * R;
     const float *rowp[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) rowp[r] = C + (int64_t)min(row0 + r, n - 1) * ld;
@@ -251,7 +246,7 @@ log_row_pass_kernel(const float *__restrict__ C, int64_t ld, int n, float s2, do
     __syncthreads();
     if (threadIdx.x < G * R) {
         const int g = threadIdx.x / R, r = threadIdx.x % R;
-        const int row = (bid * G + g) * R + r;
+        const int row = (blockIdx.x * G + g) * R + r;
         if (row < n) {
             float mm = red_m[g * W][r], ss = red_s[g * W][r];
 #pragma unroll
@@ -270,8 +265,6 @@ log_row_pass_kernel(const float *__restrict__ C, int64_t ld, int n, float s2, do
             }
         }
     }
-    if (LOOP) __syncthreads(); // the reduction buffers are reused by the next row block
-    } while (LOOP && (bid += gridDim.x) < nblocks);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -379,20 +372,17 @@ sum_partials_kernel(int n, int64_t n_pad, int ntiles, const float *__restrict__ 
 
 // Log-domain column pass stage 1: per (tile, column) running (max, sum) pair.
 // partials: plane 0 = maxima [ntiles][n_pad], plane 1 = sums.
-template <int TX, int TY, bool VEC, bool LOOP>
+template <int TX, int TY, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 log_col_partial_kernel(const float *__restrict__ C, int64_t ld, int n, int64_t n_pad, float s2,
                        const FsRowTile *__restrict__ tiles, int ntiles, int nstrips, const float *__restrict__ xs,
-                       float *__restrict__ partials, const int *run_if, int nblocks) {
+                       float *__restrict__ partials) {
     static_assert(TX * TY == kThreads, "CTA shape");
-    if (run_if != nullptr && *reinterpret_cast<const volatile int *>(run_if) == 0) return;
     constexpr int U = 8;
     __shared__ float x_s[kMaxTileRows];
     __shared__ float4 red_m[TY > 1 ? kThreads : 1], red_s[TY > 1 ? kThreads : 1];
 
-    int bid = blockIdx.x; // see log_row_pass_kernel
-    do {
-    const int tile_idx = bid / nstrips, strip = bid % nstrips;
+    const int tile_idx = blockIdx.x / nstrips, strip = blockIdx.x % nstrips;
     const FsRowTile tile = tiles[tile_idx];
     const int rows = tile.end - tile.begin;
     for (int i = threadIdx.x; i < rows; i += kThreads) x_s[i] = xs[tile.begin + i];
@@ -462,16 +452,12 @@ log_col_partial_kernel(const float *__restrict__ C, int64_t ld, int n, int64_t n
         *reinterpret_cast<float4 *>(partials + (int64_t)tile_idx * n_pad + col) = m4;
         *reinterpret_cast<float4 *>(partials + ((int64_t)ntiles + tile_idx) * n_pad + col) = s4;
     }
-    if (LOOP) __syncthreads(); // shared buffers are reused by the next block
-    } while (LOOP && (bid += gridDim.x) < nblocks);
 }
 
 __global__ void __launch_bounds__(kThreads)
 log_col_finish_kernel(int n, int64_t n_pad, int ntiles, float s2, double eps, const float *__restrict__ partials,
                       const float *__restrict__ b, const float *__restrict__ logb, float *__restrict__ g,
-                      float *__restrict__ ys, float *__restrict__ coldiff, int update, FsDeviceStatus *status,
-                      const int *run_if) {
-    if (run_if != nullptr && *reinterpret_cast<const volatile int *>(run_if) == 0) return;
+                      float *__restrict__ ys, float *__restrict__ coldiff, int update, FsDeviceStatus *status) {
     const int l = blockIdx.x * kThreads + threadIdx.x;
     if (l >= n) return;
     float mm = partials[l], ss = partials[(int64_t)ntiles * n_pad + l];
@@ -494,25 +480,16 @@ log_col_finish_kernel(int n, int64_t n_pad, int ntiles, float s2, double eps, co
 // ------------------------------------------------------------------------------------------
 // Host-side dispatch.
 
-constexpr unsigned kGuardedGrid = 148 * 4; // CTAs of a guarded launch
-
-// Kernel names as the dispatch macros use them: (shape, shape, vectorised) -> instantiation
-#define FS_K_ROW(L_, R_, V_) row_pass_kernel<L_, R_, V_>
-#define FS_K_COL(TX_, TY_, V_) col_partial_kernel<TX_, TY_, V_>
-#define FS_K_LOG_ROW(L_, R_, V_) log_row_pass_kernel<L_, R_, V_, false>
-#define FS_K_LOG_COL(TX_, TY_, V_) log_col_partial_kernel<TX_, TY_, V_, false>
-
 #define FS_ROW_CASE(KERNEL, L_, R_, ...)                                                          \
     if (p.row_L == L_ && p.row_R == R_) {                                                         \
-        if (p.vec) KERNEL(L_, R_, true)<<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                  \
-        else KERNEL(L_, R_, false)<<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                       \
+        if (p.vec) KERNEL<L_, R_, true><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                  \
+        else KERNEL<L_, R_, false><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                       \
     } else
 
 #define FS_ROW_DISPATCH(KERNEL, ...)                                                              \
     do {                                                                                          \
         const int G_ = kThreads / p.row_L;                                                        \
-        const unsigned nblk_ = (unsigned)((nrows + (int64_t)G_ * p.row_R - 1) / ((int64_t)G_ * p.row_R)); \
-        const unsigned grid_ = grid_cap != 0 && grid_cap < nblk_ ? grid_cap : nblk_;              \
+        const unsigned grid_ = (unsigned)((nrows + (int64_t)G_ * p.row_R - 1) / ((int64_t)G_ * p.row_R)); \
         FS_ROW_CASE(KERNEL, 32, 1, __VA_ARGS__)                                                   \
         FS_ROW_CASE(KERNEL, 32, 2, __VA_ARGS__)                                                   \
         FS_ROW_CASE(KERNEL, 64, 1, __VA_ARGS__)                                                   \
@@ -526,89 +503,56 @@ constexpr unsigned kGuardedGrid = 148 * 4; // CTAs of a guarded launch
     do {                                                                                          \
         const int strip_ = 4 * p.col_TX;                                                          \
         const int nstrips = (int)((n + strip_ - 1) / strip_);                                     \
-        const unsigned nblk_ = (unsigned)((int64_t)nstrips * ntiles);                             \
-        const unsigned grid_ = grid_cap != 0 && grid_cap < nblk_ ? grid_cap : nblk_;              \
+        const unsigned grid_ = (unsigned)((int64_t)nstrips * ntiles);                             \
         if (p.col_TX == 32) {                                                                     \
-            if (p.vec) KERNEL(32, 8, true)<<<grid_, kThreads, 0, st>>>(__VA_ARGS__);               \
-            else KERNEL(32, 8, false)<<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                    \
+            if (p.vec) KERNEL<32, 8, true><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);               \
+            else KERNEL<32, 8, false><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                    \
         } else if (p.col_TX == 64) {                                                              \
-            if (p.vec) KERNEL(64, 4, true)<<<grid_, kThreads, 0, st>>>(__VA_ARGS__);               \
-            else KERNEL(64, 4, false)<<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                    \
+            if (p.vec) KERNEL<64, 4, true><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);               \
+            else KERNEL<64, 4, false><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                    \
         } else {                                                                                  \
-            if (p.vec) KERNEL(256, 1, true)<<<grid_, kThreads, 0, st>>>(__VA_ARGS__);              \
-            else KERNEL(256, 1, false)<<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                   \
+            if (p.vec) KERNEL<256, 1, true><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);              \
+            else KERNEL<256, 1, false><<<grid_, kThreads, 0, st>>>(__VA_ARGS__);                   \
         }                                                                                         \
     } while (0)
 
 void fsk_row_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t nrows, const float *v,
                   const float *a, float *u, float *rowdiff, int update, float eta, FsDeviceStatus *status,
                   cudaStream_t st) {
-    const unsigned grid_cap = 0;
-    FS_ROW_DISPATCH(FS_K_ROW, K, ld, (int)n, (int)nrows, v, a, u, rowdiff, update, eta, status);
+    FS_ROW_DISPATCH(row_pass_kernel, K, ld, (int)n, (int)nrows, v, a, u, rowdiff, update, eta, status);
 }
 
 void fsk_col_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
                   int ntiles, const float *u, const float *b, float *v, float *partials, float *coldiff,
                   int update, float eta, FsDeviceStatus *status, cudaStream_t st) {
-    const unsigned grid_cap = 0;
-    FS_COL_DISPATCH(FS_K_COL, K, ld, (int)n, n_pad, tiles, nstrips, u, partials);
+    FS_COL_DISPATCH(col_partial_kernel, K, ld, (int)n, n_pad, tiles, nstrips, u, partials);
     col_finish_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>(
         (int)n, n_pad, ntiles, partials, b, v, coldiff, update, eta, status);
 }
 
 void fsk_log_row_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n, double eps, const float *ys,
                       const float *a, const float *loga, float *f, float *xs, float *rowdiff, int update,
-                      FsDeviceStatus *status, cudaStream_t st, const int *run_if) {
+                      FsDeviceStatus *status, cudaStream_t st) {
     const float s2 = (float)(1.4426950408889634 / eps);
     const int64_t nrows = n;
-    if (run_if != nullptr) {
-        // guarded launch (redo of a fused iteration; normally nothing to do): one fixed shape, a small grid that
-        // walks the row blocks
-        constexpr int L = 128, R = 2, G = kThreads / L;
-        const unsigned nblk = (unsigned)((n + (int64_t)G * R - 1) / ((int64_t)G * R));
-        const unsigned grid = nblk < kGuardedGrid ? nblk : kGuardedGrid;
-        if (p.vec)
-            log_row_pass_kernel<L, R, true, true><<<grid, kThreads, 0, st>>>(C, ld, (int)n, s2, eps, ys, a, loga, f, xs, rowdiff,
-                                                                         update, status, run_if, (int)nblk);
-        else
-            log_row_pass_kernel<L, R, false, true><<<grid, kThreads, 0, st>>>(C, ld, (int)n, s2, eps, ys, a, loga, f, xs, rowdiff,
-                                                                          update, status, run_if, (int)nblk);
-        return;
-    }
-    const unsigned grid_cap = 0;
-    FS_ROW_DISPATCH(FS_K_LOG_ROW, C, ld, (int)n, s2, eps, ys, a, loga, f, xs, rowdiff, update, status, nullptr, 0);
+    FS_ROW_DISPATCH(log_row_pass_kernel, C, ld, (int)n, s2, eps, ys, a, loga, f, xs, rowdiff, update, status);
 }
 
 void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n, int64_t n_pad, double eps,
                       const FsRowTile *tiles, int ntiles, const float *xs, const float *b, const float *logb,
                       float *g, float *ys, float *partials, float *coldiff, int update,
-                      FsDeviceStatus *status, cudaStream_t st, const int *run_if) {
+                      FsDeviceStatus *status, cudaStream_t st) {
     const float s2 = (float)(1.4426950408889634 / eps);
-    if (run_if != nullptr) {
-        constexpr int TX = 64, TY = 4; // see fsk_log_row_pass
-        const int nstrips = (int)((n + 4 * TX - 1) / (4 * TX));
-        const unsigned nblk = (unsigned)((int64_t)nstrips * ntiles);
-        const unsigned grid = nblk < kGuardedGrid ? nblk : kGuardedGrid;
-        if (p.vec)
-            log_col_partial_kernel<TX, TY, true, true><<<grid, kThreads, 0, st>>>(C, ld, (int)n, n_pad, s2, tiles, ntiles, nstrips, xs,
-                                                                              partials, run_if, (int)nblk);
-        else
-            log_col_partial_kernel<TX, TY, false, true><<<grid, kThreads, 0, st>>>(C, ld, (int)n, n_pad, s2, tiles, ntiles, nstrips,
-                                                                               xs, partials, run_if, (int)nblk);
-    } else {
-        const unsigned grid_cap = 0;
-        FS_COL_DISPATCH(FS_K_LOG_COL, C, ld, (int)n, n_pad, s2, tiles, ntiles, nstrips, xs, partials, nullptr, 0);
-    }
+    FS_COL_DISPATCH(log_col_partial_kernel, C, ld, (int)n, n_pad, s2, tiles, ntiles, nstrips, xs, partials);
     log_col_finish_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>(
-        (int)n, n_pad, ntiles, s2, eps, partials, b, logb, g, ys, coldiff, update, status, run_if);
+        (int)n, n_pad, ntiles, s2, eps, partials, b, logb, g, ys, coldiff, update, status);
 }
 
 // Stage 1 followed by a plain sum of the tile partials: r_out[l] = sum over the given row tiles of
 // K_il u_i, without the divide (the shard's contribution to K^T u).
 void fsk_col_partial_sum(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
                          int ntiles, const float *u, float *partials, float *r_out, cudaStream_t st) {
-    const unsigned grid_cap = 0;
-    FS_COL_DISPATCH(FS_K_COL, K, ld, (int)n, n_pad, tiles, nstrips, u, partials);
+    FS_COL_DISPATCH(col_partial_kernel, K, ld, (int)n, n_pad, tiles, nstrips, u, partials);
     sum_partials_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>((int)n, n_pad, ntiles, partials, r_out);
 }
 
@@ -623,7 +567,7 @@ void fsk_log_col_finish(int64_t n, int64_t n_pad, int ntiles, double eps, const 
                         cudaStream_t st) {
     const float s2 = (float)(1.4426950408889634 / eps);
     log_col_finish_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>(
-        (int)n, n_pad, ntiles, s2, eps, partials, b, logb, g, ys, coldiff, update, status, nullptr);
+        (int)n, n_pad, ntiles, s2, eps, partials, b, logb, g, ys, coldiff, update, status);
 }
 
 int fsk_pass_launches_row() { return 1; }
