@@ -371,12 +371,11 @@ def run_ours(args, w, rank, local_rank, world):
     fused_log = w.nbatch == 1 and w.domain == workloads.DOMAIN_LOG and 4096 <= w.n <= 16384 and w.n % 4 == 0
     n2 = w.n * w.n * 4
     if fused_log:
-        # one launch of the fused log kernel per iteration; the interval also holds its stage-2 kernel, the
-        # three guarded two-pass launches (no-ops in range) and the commit kernel
+        # one launch of the fused log kernel per iteration; the interval also holds its stage-2 kernel
         per_launch_s = timed(lambda: fs.fs_iterate(h, 1, stream))
         kernel, bytes_launch = "fused_log_iteration_kernel", n2
         note = ("one launch per iteration reads C once (n*n*4 bytes), one ex2 per element; the timed interval "
-                "includes the stage-2, guard and commit kernels that follow it (about 15 us)")
+                "includes the stage-2 kernel that follows it")
     elif fused:
         # one launch of the fused kernel per iteration; the interval also holds the stage-2 kernel
         # that follows it (a few microseconds), so the kernel's own rate is slightly understated
