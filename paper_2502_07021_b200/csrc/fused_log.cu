@@ -302,31 +302,33 @@ fused_log_iteration_kernel(const float *__restrict__ C, int64_t ld, int n, int n
 }
 
 // Stage 2 of the fused log iteration: r_l = sum of the per-CTA column sums, g_l <- g_l + eps log(b_l / r_l);
-// coldiff = r_l - b_l.  A CTA serves 32 columns: thread (c, k) of 32 x 8 adds the rows k, k + 8, ... of the
-// partial matrix for column c (128-byte coalesced reads), and the eight group sums of a column are added in
-// group order -- a fixed order, so the result is reproducible.  If one of its columns has r_l outside the
-// safe range, the CTA recomputes its columns from C and the new row duals: thread (c, k) folds the rows
-// k, k + 8, ... into a running (maximum, sum) pair, the eight pairs of a column are merged in group order,
+// coldiff = r_l - b_l.  A CTA serves 32 columns: thread (c, k) of 32 x 16 adds the rows k, k + 16, ... of the
+// partial matrix for column c (128-byte coalesced reads, all of a thread's loads in flight at once), and the
+// sixteen group sums of a column are added in group order -- a fixed order, so the result is reproducible.
+// If one of its columns has r_l outside the safe range, the CTA recomputes its columns from C and the new row
+// duals: thread (c, k) folds the rows k, k + 16, ... into a running (maximum, sum) pair, the pairs of a column
+// are merged in group order,
 // and g_l = eps (log2 b_l - M - log2 S) ln 2 is the stabilised update itself.  The last CTA to finish counts
 // the iteration as a fallback if any row or column was redone, and clears the flag.
-__global__ void __launch_bounds__(256)
+constexpr int kFinishGroups = 16;
+__global__ void __launch_bounds__(32 * kFinishGroups)
 fused_log_finish_kernel(int n, int nclusters, double eps, float s2, const float *__restrict__ C, int64_t ld,
                         const float *__restrict__ partials, const float *__restrict__ b, const float *__restrict__ xs,
                         float *ys, float *__restrict__ g_out, float *__restrict__ coldiff, FsDeviceStatus *status,
                         int *done_blocks) {
-    __shared__ float part[8][32], pmax[8][32];
+    __shared__ float part[kFinishGroups][32], pmax[kFinishGroups][32];
     const int c = threadIdx.x & 31, k0 = threadIdx.x >> 5;
     const int l = blockIdx.x * 32 + c;
     float acc = 0.f;
     if (l < n) {
-#pragma unroll 4
-        for (int k = k0; k < nclusters; k += 8) acc += __ldcg(partials + (int64_t)k * n + l);
+#pragma unroll 10
+        for (int k = k0; k < nclusters; k += kFinishGroups) acc += __ldcg(partials + (int64_t)k * n + l);
     }
     part[k0][c] = acc;
     __syncthreads();
     float r = part[0][c];
 #pragma unroll
-    for (int k = 1; k < 8; ++k) r += part[k][c];
+    for (int k = 1; k < kFinishGroups; ++k) r += part[k][c];
     const bool bad = l < n && !in_range(r);
     const int any_bad = __syncthreads_or(bad ? 1 : 0); // also orders the reads of part[] before its reuse
     const float bl = l < n ? b[l] : 1.f;
@@ -336,7 +338,7 @@ fused_log_finish_kernel(int n, int nclusters, double eps, float s2, const float 
         // running (maximum, sum) of t = xs_i - C_il log2(e)/eps over this thread's rows
         float m = -INFINITY, sum = 0.f;
         if (l < n) {
-            for (int i = k0; i < n; i += 8) {
+            for (int i = k0; i < n; i += kFinishGroups) {
                 const float t = fmaf(__ldg(C + (int64_t)i * ld + l), -s2, __ldg(xs + i));
                 if (t > m) {
                     sum = sum * ex2(m - t) + 1.f; // first row: 0 * 2^-inf + 1
@@ -350,7 +352,7 @@ fused_log_finish_kernel(int n, int nclusters, double eps, float s2, const float 
         __syncthreads();
         float M = pmax[0][c], S = part[0][c];
 #pragma unroll
-        for (int k = 1; k < 8; ++k) {
+        for (int k = 1; k < kFinishGroups; ++k) {
             const float mk = pmax[k][c], sk = part[k][c];
             const float mm = fmaxf(M, mk);
             S = (M == -INFINITY ? 0.f : S * ex2(M - mm)) + (mk == -INFINITY ? 0.f : sk * ex2(mk - mm));
@@ -476,7 +478,7 @@ cudaError_t fsk_fused_log_iteration(const FsFusedPlan &p, const float *C, int64_
 #undef FS_LOG_CASE
     }
     if (e != cudaSuccess) return e;
-    fused_log_finish_kernel<<<(unsigned)((n + 31) / 32), 256, 0, st>>>((int)n, p.nclusters, eps, s2, C, ld, partials, b, xs, ys, g,
+    fused_log_finish_kernel<<<(unsigned)((n + 31) / 32), 32 * kFinishGroups, 0, st>>>((int)n, p.nclusters, eps, s2, C, ld, partials, b, xs, ys, g,
                                                                        coldiff, status, done_blocks);
     return cudaGetLastError();
 }

@@ -340,16 +340,35 @@ col_partial_kernel(const float *__restrict__ K, int64_t ld, int n, int64_t n_pad
         *reinterpret_cast<float4 *>(partials + (int64_t)tile_idx * n_pad + col) = acc;
 }
 
-// Column pass stage 2: r_l = sum over tiles in tile order; residual; divide.
+// Sum of the tile partials of the CTA's 32 columns: thread (c, k) of 32 x 8 adds the tiles k, k + 8, ... of
+// column c (128-byte coalesced reads, the eight chains of a column run side by side instead of one chain of
+// `ntiles` dependent loads), then the eight group sums are added in group order.  The order is fixed by the
+// tile index alone, so the result is reproducible and independent of the launch.  Returns the sum to the
+// threads of group 0; `valid` = the column exists.
+__device__ __forceinline__ float sum_tiles_32x8(const float *__restrict__ partials, int64_t n_pad, int ntiles, int l,
+                                                bool valid, float (*part)[32]) {
+    const int c = threadIdx.x & 31, k0 = threadIdx.x >> 5;
+    float acc = 0.f;
+    if (valid) {
+#pragma unroll 8
+        for (int t = k0; t < ntiles; t += 8) acc += partials[(int64_t)t * n_pad + l];
+    }
+    part[k0][c] = acc;
+    __syncthreads();
+    float r = part[0][c];
+#pragma unroll
+    for (int k = 1; k < 8; ++k) r += part[k][c];
+    return r;
+}
+
+// Column pass stage 2: r_l = sum over tiles (fixed order, see above); residual; divide.  32 columns per CTA.
 __global__ void __launch_bounds__(kThreads)
 col_finish_kernel(int n, int64_t n_pad, int ntiles, const float *__restrict__ partials, const float *__restrict__ b,
                   float *__restrict__ v, float *__restrict__ coldiff, int update, float eta, FsDeviceStatus *status) {
-    const int l = blockIdx.x * kThreads + threadIdx.x;
-    if (l >= n) return;
-    float r = 0.f;
-    // same left-to-right order as a plain loop; unrolled so that eight loads are in flight at a time
-#pragma unroll 8
-    for (int t = 0; t < ntiles; ++t) r += partials[(int64_t)t * n_pad + l];
+    __shared__ float part[8][32];
+    const int l = blockIdx.x * 32 + (threadIdx.x & 31);
+    const float r = sum_tiles_32x8(partials, n_pad, ntiles, l, l < n, part);
+    if (threadIdx.x >= 32 || l >= n) return;
     const float bl = b[l], vo = v[l];
     coldiff[l] = fmaf(vo, r, -bl);
     if (update) {
@@ -359,15 +378,13 @@ col_finish_kernel(int n, int64_t n_pad, int ntiles, const float *__restrict__ pa
     }
 }
 
-// Sum of the tile partials alone, in tile order.
+// Sum of the tile partials alone, in the same order.
 __global__ void __launch_bounds__(kThreads)
 sum_partials_kernel(int n, int64_t n_pad, int ntiles, const float *__restrict__ partials, float *__restrict__ r_out) {
-    const int l = blockIdx.x * kThreads + threadIdx.x;
-    if (l >= n) return;
-    float r = 0.f;
-#pragma unroll 8
-    for (int t = 0; t < ntiles; ++t) r += partials[(int64_t)t * n_pad + l];
-    r_out[l] = r;
+    __shared__ float part[8][32];
+    const int l = blockIdx.x * 32 + (threadIdx.x & 31);
+    const float r = sum_tiles_32x8(partials, n_pad, ntiles, l, l < n, part);
+    if (threadIdx.x < 32 && l < n) r_out[l] = r;
 }
 
 // Log-domain column pass stage 1: per (tile, column) running (max, sum) pair.
@@ -526,7 +543,7 @@ void fsk_col_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, in
                   int ntiles, const float *u, const float *b, float *v, float *partials, float *coldiff,
                   int update, float eta, FsDeviceStatus *status, cudaStream_t st) {
     FS_COL_DISPATCH(col_partial_kernel, K, ld, (int)n, n_pad, tiles, nstrips, u, partials);
-    col_finish_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>(
+    col_finish_kernel<<<(unsigned)((n + 31) / 32), kThreads, 0, st>>>(
         (int)n, n_pad, ntiles, partials, b, v, coldiff, update, eta, status);
 }
 
@@ -553,12 +570,12 @@ void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n
 void fsk_col_partial_sum(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
                          int ntiles, const float *u, float *partials, float *r_out, cudaStream_t st) {
     FS_COL_DISPATCH(col_partial_kernel, K, ld, (int)n, n_pad, tiles, nstrips, u, partials);
-    sum_partials_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>((int)n, n_pad, ntiles, partials, r_out);
+    sum_partials_kernel<<<(unsigned)((n + 31) / 32), kThreads, 0, st>>>((int)n, n_pad, ntiles, partials, r_out);
 }
 
 void fsk_col_finish(int64_t n, int64_t n_pad, int ntiles, const float *partials, const float *b, float *v,
                     float *coldiff, int update, float eta, FsDeviceStatus *status, cudaStream_t st) {
-    col_finish_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>((int)n, n_pad, ntiles, partials, b, v,
+    col_finish_kernel<<<(unsigned)((n + 31) / 32), kThreads, 0, st>>>((int)n, n_pad, ntiles, partials, b, v,
                                                                                    coldiff, update, eta, status);
 }
 
