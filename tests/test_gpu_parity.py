@@ -226,10 +226,12 @@ def test_fused_log_is_reproducible_and_traces():
         assert l1[k] == pytest.approx(e["row_l1"], rel=2e-3, abs=1e-6)
 
 
-def test_fused_log_falls_back_after_a_jump_of_the_duals():
+@pytest.mark.parametrize("n", [2048, 4100, 8192, 12288])
+def test_fused_log_falls_back_after_a_jump_of_the_duals(n):
     """A jump of the duals by hundreds of eps between two iterations takes the marginals out of the fast
-    path's fp32 range: the rows and columns concerned must be redone with a maximum, transparently."""
-    w = workloads.make(3, n=2048)
+    path's fp32 range: the rows and columns concerned must be redone with a maximum, transparently.  The sizes
+    cover 4, 2 and 1 rows per stage and a ragged last column group."""
+    w = workloads.make(3, n=n)
     with GpuSolver(w.C, KC, w.eps, w.a, w.b, w.offsets, LG) as g:
         fs.fs_set_option(g.h, fs.FS_OPT_FUSED, 2)
         g.iterate(6)
