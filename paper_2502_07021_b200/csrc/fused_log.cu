@@ -321,8 +321,17 @@ fused_log_finish_kernel(int n, int nclusters, double eps, float s2, const float 
     const int l = blockIdx.x * 32 + c;
     float acc = 0.f;
     if (l < n) {
-#pragma unroll 10
-        for (int k = k0; k < nclusters; k += kFinishGroups) acc += __ldcg(partials + (int64_t)k * n + l);
+        // ten loads issued before the first add; ten at a time if there are more than 160 partial rows
+        for (int kb = k0; kb < nclusters; kb += 10 * kFinishGroups) {
+            float x[10];
+#pragma unroll
+            for (int i = 0; i < 10; ++i) {
+                const int k = kb + i * kFinishGroups;
+                x[i] = k < nclusters ? __ldcg(partials + (int64_t)k * n + l) : 0.f;
+            }
+#pragma unroll
+            for (int i = 0; i < 10; ++i) acc += x[i];
+        }
     }
     part[k0][c] = acc;
     __syncthreads();
