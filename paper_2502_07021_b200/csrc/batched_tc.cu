@@ -30,7 +30,10 @@
 // shared memory (each rank receives the columns of its 128 / KS problems from every rank into an idle
 // ring stage), add them in rank order and apply the divide, the marginal residual and the bf16 re-split
 // of the new scalings; the re-split operand is collected in shared memory and written with 16-byte
-// stores.  One launch per pass; nothing but K, the operand and the result vectors touches HBM.  Every
+// stores.  One launch per pass; nothing but K, the operand and the result vectors touches HBM.  The passes
+// are launched with programmatic stream serialisation: a pass lets its successor start at once, and the
+// successor sets itself up and requests its first K tiles (K never changes) on every SM its predecessor has
+// left, then waits for the predecessor's completion before it touches anything that pass produced.  Every
 // mbarrier wait is bounded: on expiry the kernel raises a status flag, stops issuing work, drains what it
 // had in flight and still takes part in the cluster barriers before it exits.
 #include <cuda.h>
@@ -163,6 +166,11 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
+// Programmatic dependent launch: the pass that follows this one in the stream may begin (set-up, first K tiles)
+// as soon as every CTA of this grid has run launch_dependents; griddep_wait returns when the preceding grid has
+// completed and its writes are visible.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -222,10 +230,29 @@ batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_const
     tc_fence_after();
     const uint32_t tmem = *tmem_slot_ptr;
     bool ok = true;
+    // The next pass may start its set-up and its first K tiles while this one is still running; everything that
+    // reads or writes what the preceding pass produced (the operand tiles, the scalings, the residual) comes
+    // after griddep_wait.  K itself is constant, so its first tiles are requested before the wait.
+    griddep_launch_dependents();
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int it = 0; it < nkb; ++it) {
+            const int pre = nkb < STAGES ? nkb : STAGES; // first fill of the ring: slots are free
+            for (int it = 0; it < pre; ++it) {
+                const uint32_t full = bars + 8 * it, dst = base + it * STAGE_BYTES;
+                mbar_expect_tx(full, STAGE_BYTES);
+                const int ya = (mtile * kblocks + kb0 + it) * BM;
+                tma_load_2d(&tmA_hi, dst, full, 0, ya);
+                tma_load_2d(&tmA_lo, dst + TILE_BYTES, full, 0, ya);
+            }
+            griddep_wait();
+            for (int it = 0; it < pre; ++it) {
+                const uint32_t full = bars + 8 * it, dst = base + it * STAGE_BYTES;
+                const int yb = (ntile * kblocks + kb0 + it) * BN;
+                tma_load_2d(&tmB_hi, dst + 2 * TILE_BYTES, full, 0, yb);
+                tma_load_2d(&tmB_lo, dst + 3 * TILE_BYTES, full, 0, yb);
+            }
+            for (int it = pre; it < nkb; ++it) {
                 const int s = it % STAGES;
                 const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
                 if (!mbar_wait(bars + 8 * (STAGES + s), ph ^ 1u)) { ok = false; break; }
@@ -277,6 +304,7 @@ batched_tc_kernel(const __grid_constant__ CUtensorMap tmA_hi, const __grid_const
         // each thread keeps the running sums of one output row x 64 problems in registers
         const int quarter = warp & 3, half = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;
+        griddep_wait(); // these warps read the old scalings and write this pass's results
         constexpr int HN = BN / 2;
         float sum[HN];
 #pragma unroll
@@ -491,7 +519,9 @@ void fill_launch(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int ks, int
     cfg.stream = st;
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 1, attr[0].val.clusterDim.y = (unsigned)ks, attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr, cfg.numAttrs = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr, cfg.numAttrs = 2;
 }
 
 const void *kernel_for(int ks) {
@@ -514,7 +544,7 @@ bool cluster_fits(int ks, int mtiles, int ntiles) {
         return false;
     }
     cudaLaunchConfig_t cfg{};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     fill_launch(cfg, attr, ks, mtiles, ntiles, nullptr);
     int nclusters = 0;
     if (cudaOccupancyMaxActiveClusters(&nclusters, kernel_for(ks), &cfg) != cudaSuccess) {
@@ -593,7 +623,7 @@ void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float 
     const CUtensorMap &b_hi = transposed ? t->tmU_hi : t->tmV_hi, &b_lo = transposed ? t->tmU_lo : t->tmV_lo;
     __nv_bfloat16 *op_hi = transposed ? t->V_hi : t->U_hi, *op_lo = transposed ? t->V_lo : t->U_lo;
     cudaLaunchConfig_t cfg{};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     fill_launch(cfg, attr, t->ksplit, t->mtiles, t->ntiles, st);
     switch (t->ksplit) {
     case 1: cudaLaunchKernelEx(&cfg, batched_tc_kernel<1>, a_hi, a_lo, b_hi, b_lo, t->kblocks, (int)t->n, t->nbatch, marg, out, diff, op_hi, op_lo, update, eta, status); break;
