@@ -70,6 +70,10 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
     }
     __syncthreads();
     cluster_sync_all(); // every CTA's barriers exist before anyone arrives on them remotely
+    // The kernel after this one (stage 2) may be scheduled at once; this kernel itself is launched with programmatic
+    // stream serialisation: its producer streams K, which never changes, while the preceding stage-2 kernel is still
+    // running, and the compute groups wait for that kernel before they read v or write anything.
+    griddep_launch_dependents();
 
     bool ok = true;
     if (warp == 2 * kWarpsPerGroup) {
@@ -110,11 +114,13 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
     } else if (warp < kWarpsPerGroup) {
         // ---------------- dot group ----------------
         const int t = threadIdx.x; // 0..255
+        griddep_wait();
         float4 v4[F];
 #pragma unroll
         for (int j = 0; j < F; ++j) {
             const int c4 = j * kGroup + t;
-            v4[j] = c4 < seg4 ? __ldg(reinterpret_cast<const float4 *>(v + col0) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            // v was written by the preceding stage-2 kernel, during which this kernel may already be resident: a coherent load
+            v4[j] = c4 < seg4 ? __ldcg(reinterpret_cast<const float4 *>(v + col0) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         int k = 0;
         for (int tl = cluster; tl < ntiles && ok; tl += nclusters) {
@@ -162,6 +168,7 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
     } else {
         // ---------------- accumulate group ----------------
         const int t = threadIdx.x - kGroup; // 0..255
+        griddep_wait();
         float4 r4[F];
 #pragma unroll
         for (int j = 0; j < F; ++j) r4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -253,8 +260,10 @@ void fill_cluster_launch(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int
     attr[0].val.clusterDim.x = (unsigned)S;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
 }
 
 template <int F, int R>
@@ -262,7 +271,7 @@ cudaError_t launch_fused(const FsFusedPlan &p, cudaStream_t st, const float *K, 
                          int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials, float eta,
                          FsDeviceStatus *status) {
     cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     fill_cluster_launch(cfg, attr, p.S, p.nclusters, fused_smem_bytes(F, R, p.nstages), st);
     return cudaLaunchKernelEx(&cfg, fused_iteration_kernel<F, R>, K, ld, n, p.S, p.nclusters, p.nstages, tiles, ntiles, v, a,
                               u, rowdiff, partials, eta, status);
@@ -276,7 +285,7 @@ int query_clusters(int S, int nstages) {
         return 0;
     }
     cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     fill_cluster_launch(cfg, attr, S, 148, smem, nullptr);
     int nc = 0;
     if (cudaOccupancyMaxActiveClusters(&nc, fused_iteration_kernel<F, R>, &cfg) != cudaSuccess) {

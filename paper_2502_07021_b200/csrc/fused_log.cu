@@ -113,12 +113,17 @@ fused_log_iteration_kernel(const float *__restrict__ C, int64_t ld, int n, int n
         }
         for (int s = 0; s < nstages; ++s) producer_issue();
     }
+    // C never changes: the first stages were requested above, possibly while the preceding stage-2 kernel is
+    // still running (programmatic stream serialisation); everything below depends on that kernel's duals.
+    griddep_launch_dependents();
+    griddep_wait();
 
     float4 g4[FT], r4[FT];
 #pragma unroll
     for (int j = 0; j < FT; ++j) {
         const int c4 = j * kThreadsLog + t;
-        g4[j] = c4 < n4 ? __ldg(reinterpret_cast<const float4 *>(ys) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        // written by the preceding stage-2 kernel, during which this kernel may already be resident: a coherent load
+        g4[j] = c4 < n4 ? __ldcg(reinterpret_cast<const float4 *>(ys) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
         r4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     bool out_of_range = false, ok = true;
@@ -317,6 +322,7 @@ fused_log_finish_kernel(int n, int nclusters, double eps, float s2, const float 
                         float *ys, float *__restrict__ g_out, float *__restrict__ coldiff, FsDeviceStatus *status,
                         int *done_blocks) {
     __shared__ float part[kFinishGroups][32], pmax[kFinishGroups][32];
+    griddep_launch_dependents(); // the next iteration's fused kernel may start requesting C
     const int c = threadIdx.x & 31, k0 = threadIdx.x >> 5;
     const int l = blockIdx.x * 32 + c;
     float acc = 0.f;
@@ -401,9 +407,15 @@ template <int FT, int R>
 cudaError_t launch_fused_log(const FsFusedPlan &p, cudaStream_t st, const float *C, int64_t ld, int n, float s2, double eps,
                              const FsRowTile *tiles, int ntiles, float *xs, const float *ys, const float *a,
                              float *f_out, float *rowdiff, float *partials, FsDeviceStatus *status) {
-    fused_log_iteration_kernel<FT, R><<<(unsigned)p.nclusters, kThreadsLog, fused_log_smem_bytes(n, R, p.nstages), st>>>(
-        C, ld, n, p.nclusters, p.nstages, s2, eps, tiles, ntiles, xs, ys, a, f_out, rowdiff, partials, status);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    cfg.gridDim = dim3((unsigned)p.nclusters), cfg.blockDim = dim3(kThreadsLog);
+    cfg.dynamicSmemBytes = fused_log_smem_bytes(n, R, p.nstages), cfg.stream = st;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr, cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fused_log_iteration_kernel<FT, R>, C, ld, n, p.nclusters, p.nstages, s2, eps, tiles, ntiles,
+                              xs, ys, a, f_out, rowdiff, partials, status);
 }
 
 template <int FT, int R>

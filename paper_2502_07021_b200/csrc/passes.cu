@@ -366,6 +366,9 @@ __global__ void __launch_bounds__(kThreads)
 col_finish_kernel(int n, int64_t n_pad, int ntiles, const float *__restrict__ partials, const float *__restrict__ b,
                   float *__restrict__ v, float *__restrict__ coldiff, int update, float eta, FsDeviceStatus *status) {
     __shared__ float part[8][32];
+    // a fused iteration kernel launched behind this one may start streaming K now (it waits for this grid's
+    // completion before it reads v)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int l = blockIdx.x * 32 + (threadIdx.x & 31);
     const float r = sum_tiles_32x8(partials, n_pad, ntiles, l, l < n, part);
     if (threadIdx.x >= 32 || l >= n) return;
