@@ -131,9 +131,9 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
                 const int slot = k % (2 * nstages);
                 if (!mbar_wait(bars + 8 * s, (uint32_t)(k / nstages) & 1u)) { ok = false; break; }
                 const uint32_t st = base + (uint32_t)s * stage_bytes + (uint32_t)t * 16u;
-                float acc[R];
+                float acc[R], acc2[R]; // two chains per row: half the dependent multiply-adds
 #pragma unroll
-                for (int r = 0; r < R; ++r) acc[r] = 0.f;
+                for (int r = 0; r < R; ++r) acc[r] = acc2[r] = 0.f;
 #pragma unroll
                 for (int j = 0; j < F; ++j) {
                     if (j * kGroup + t < seg4) {
@@ -142,13 +142,15 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
                             if (r < cnt) {
                                 const float4 kv = lds4(st + (uint32_t)r * row_bytes + (uint32_t)j * (kGroup * 16u));
                                 acc[r] = fmaf(kv.x, v4[j].x, acc[r]);
-                                acc[r] = fmaf(kv.y, v4[j].y, acc[r]);
+                                acc2[r] = fmaf(kv.y, v4[j].y, acc2[r]);
                                 acc[r] = fmaf(kv.z, v4[j].z, acc[r]);
-                                acc[r] = fmaf(kv.w, v4[j].w, acc[r]);
+                                acc2[r] = fmaf(kv.w, v4[j].w, acc2[r]);
                             }
                         }
                     }
                 }
+#pragma unroll
+                for (int r = 0; r < R; ++r) acc[r] += acc2[r];
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) {
 #pragma unroll
