@@ -251,6 +251,27 @@ def test_fused_log_falls_back_after_a_jump_of_the_duals(n):
 
 
 @pytest.mark.slow
+@pytest.mark.parametrize("cfg", [3, 4])
+def test_large_fused_iterations_are_reproducible(cfg):
+    """The fused iteration kernels start while the stage-2 kernel before them is still running (dependent
+    launch) and wait for it before they read its output; a read that came too early, or through a stale
+    cache line, would show as run-to-run differences at sizes where every SM is busy: two runs of the same
+    problem at n = 16384 must agree bit for bit, and with the two-pass path within its tolerance."""
+    w = workloads.make(cfg, n=16384, want_cost=None if cfg == 3 else False)
+    runs = []
+    for mode in (1, 1, 0):
+        with GpuSolver(w.matrix, w.kind, w.eps, w.a, w.b, w.offsets, w.domain) as g:
+            fs.fs_set_option(g.h, fs.FS_OPT_FUSED, mode)
+            g.iterate(25)
+            runs.append(g.scalings())
+    assert np.array_equal(runs[0][0], runs[1][0]) and np.array_equal(runs[0][1], runs[1][1])
+    if cfg == 3:
+        assert np.max(np.abs(runs[0][0] - runs[2][0])) / w.eps < 3e-5 and np.max(np.abs(runs[0][1] - runs[2][1])) / w.eps < 3e-5
+    else:
+        assert rel_err(runs[0][0], runs[2][0]) < 1e-5 and rel_err(runs[0][1], runs[2][1]) < 1e-5
+
+
+@pytest.mark.slow
 def test_fused_clusters_of_four_beyond_n_32768():
     """Rows longer than 32768 columns are split over clusters of four CTAs (S = 4); this is the only
     size class that takes that path, so it gets a (slow) case of its own: n = 36864, three iterations."""
