@@ -335,6 +335,18 @@ def test_batched_tensor_core_cluster_sizes(n, nb):
     batched_sample(w, U, V, 10, sorted({0, 1, 63, 64, nb // 2, nb - 2, nb - 1}))
 
 
+def test_batched_tensor_core_passes_are_reproducible():
+    """Consecutive tensor-core passes overlap (a pass requests its first K tiles while its predecessor is
+    finishing and waits for it before reading the operand it wrote): two runs must agree bit for bit."""
+    w = workloads.make(5, n=4096, nbatch=128)
+    runs = []
+    for _ in range(2):
+        with GpuSolver(w.K, KK, w.eps, w.a, w.b, w.offsets, SC) as g:
+            g.iterate(30)
+            runs.append(g.scalings())
+    assert np.array_equal(runs[0][0], runs[1][0]) and np.array_equal(runs[0][1], runs[1][1])
+
+
 def test_batched_tensor_core_engine_converges():
     w = workloads.make(5, n=1024, nbatch=64)
     check_converged(w, w.iters, w.C, problems=(0, 33, 63))
