@@ -45,11 +45,11 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (kernel name, n) -> bytes; a capture at n = 16384 is scaled by 4 for n = 32768 (traffic is proportional to n*n).
 TRAFFIC_BYTES_PER_LAUNCH = {
-    ("fused_iteration_kernel", 16384): 1.073989e9 + 4.5e6,
-    ("fused_iteration_kernel", 32768): 4 * (1.073989e9 + 4.5e6),
+    ("fused_iteration_kernel", 16384): 1.074000e9 + 3.67e6,
+    ("fused_iteration_kernel", 32768): 4 * (1.074000e9 + 3.67e6),
     ("log_row_pass_kernel", 16384): 1.074043e9 + 3.39e6,
-    ("fused_log_iteration_kernel", 16384): 1.073987e9 + 4.47e6,
-    ("batched_tc_kernel", 8192): 281.14e6 + 3.94e6,
+    ("fused_log_iteration_kernel", 16384): 1.073997e9 + 4.36e6,
+    ("batched_tc_kernel", 8192): 281.10e6 + 3.51e6,
     # captured on a 200-iteration launch; K is read from DRAM once per launch whatever the iteration count
     ("persistent_iterations_kernel", 4096): 67.26e6 + 1.4e6,
 }
