@@ -283,14 +283,20 @@ def marginals(M, kind, eps, domain, x, y):
     return row, col
 
 
-def marginal_errors(M, kind, eps, domain, x, y, a, b):
-    """dict(row_l1, row_l2, col_l1, col_l2) of the plan's marginals against a and b."""
-    row, col = marginals(M, kind, eps, domain, x, y)
-    n = row.size
+def marginal_error_norms(row, col, a, b):
+    """dict(row_l1, row_l2, col_l1, col_l2): 1-norm and 2-norm of row - a and of col - b for given marginals."""
+    n = np.asarray(row).size
+    row, col = _f64(row, n), _f64(col, n)
     a, b = _f32(a, n), _f32(b, n)
     err = np.empty(4)
     _load().or_marginal_errors(n, _p64(row), _p64(col), _p32(a), _p32(b), _p64(err))
     return dict(row_l1=err[0], row_l2=err[1], col_l1=err[2], col_l2=err[3])
+
+
+def marginal_errors(M, kind, eps, domain, x, y, a, b):
+    """dict(row_l1, row_l2, col_l1, col_l2) of the plan's marginals against a and b."""
+    row, col = marginals(M, kind, eps, domain, x, y)
+    return marginal_error_norms(row, col, a, b)
 
 
 def plan(M, kind, eps, domain, x, y):

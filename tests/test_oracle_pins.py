@@ -425,6 +425,68 @@ def test_against_newton_on_the_dual(n, eps, seed):
     np.testing.assert_allclose(gl + shift, g, atol=1e-7)
 
 
+# ------------------------------------------------------------------ error norms and log-domain marginals
+
+def test_marginal_error_norms_on_hand_made_differences():
+    """Section 5.3's err_a is a 2-norm; the acceptance bound uses the 1-norm.  Differences chosen as Pythagorean
+    triples on a dyadic grid fix both exactly: rows (3, -4, 0)/1024 -> 7/1024 and 5/1024, columns
+    (5, 0, -12)/1024 -> 17/1024 and 13/1024.  A dropped root, a swapped row/column slot or a swapped norm fails."""
+    a = np.array([0.25, 0.5, 0.25], dtype=np.float32)
+    b = np.array([0.5, 0.125, 0.375], dtype=np.float32)
+    row = a.astype(np.float64) + np.array([3.0, -4.0, 0.0]) / 1024
+    col = b.astype(np.float64) + np.array([5.0, 0.0, -12.0]) / 1024
+    e = oracle.marginal_error_norms(row, col, a, b)
+    assert e["row_l1"] == 7 / 1024 and e["row_l2"] == 5 / 1024
+    assert e["col_l1"] == 17 / 1024 and e["col_l2"] == 13 / 1024
+
+
+@pytest.mark.parametrize("domain", [SC, LG])
+def test_marginal_errors_against_plan_sums_and_norm_inequalities(domain):
+    """On a real (unconverged) state: the errors equal numpy's norms of the dense plan's row and column sums
+    minus a, b, and satisfy ||d||_2 <= ||d||_1 <= sqrt(n) ||d||_2."""
+    n, eps = 23, 0.2
+    C = random_cost(n, 91)
+    a, b = dirichlet_pair(n, 92)
+    if domain == SC:
+        x, y = oracle.sinkhorn_scaling(C, C_, eps, a, b, 2)
+        rng = np.random.default_rng(93)
+        x, y = x * (1 + 0.2 * (rng.random(n) - 0.5)), y * (1 + 0.1 * (rng.random(n) - 0.3))      # off both marginals
+    else:
+        x, y = oracle.sinkhorn_log(C, eps, a, b, 2)
+        rng = np.random.default_rng(94)
+        x, y = x + 0.04 * (rng.random(n) - 0.5), y - 0.02 * (rng.random(n) - 0.3)
+    P = oracle.plan(C, C_, eps, domain, x, y)
+    e = oracle.marginal_errors(C, C_, eps, domain, x, y, a, b)
+    dr, dc = P.sum(1) - a.astype(np.float64), P.sum(0) - b.astype(np.float64)
+    assert e["row_l1"] == pytest.approx(np.abs(dr).sum(), rel=1e-11)
+    assert e["row_l2"] == pytest.approx(np.linalg.norm(dr), rel=1e-11)
+    assert e["col_l1"] == pytest.approx(np.abs(dc).sum(), rel=1e-11)
+    assert e["col_l2"] == pytest.approx(np.linalg.norm(dc), rel=1e-11)
+    assert e["row_l1"] > 1e-3 and e["col_l1"] > 1e-3 and abs(e["row_l1"] - e["col_l1"]) > 1e-6
+    for k in ("row", "col"):
+        assert e[k + "_l2"] <= e[k + "_l1"] <= np.sqrt(n) * e[k + "_l2"]
+
+
+def test_log_domain_marginals_rank1_closed_form_both_sides():
+    """Additive cost C_il = x_i + y_l (x != y): at f = g = 0 the plan is exp(-x_i/eps) exp(-y_l/eps), so
+    row_i = exp(-x_i/eps) sum_l exp(-y_l/eps) and col_l = exp(-y_l/eps) sum_i exp(-x_i/eps); after one log row
+    half-step from g = 0 the row marginal is a, and after the column half-step the column marginal is b."""
+    n, eps = 29, 0.13
+    C, x, y = dyadic_additive(n, 77)
+    a, b = dirichlet_pair(n, 78)
+    z = np.zeros(n)
+    row, col = oracle.marginals(C, C_, eps, LG, z, z)
+    np.testing.assert_allclose(row, np.exp(-x / eps) * np.exp(-y / eps).sum(), rtol=1e-13)
+    np.testing.assert_allclose(col, np.exp(-y / eps) * np.exp(-x / eps).sum(), rtol=1e-13)
+    f = oracle.log_row_pass(C, eps, a, z)
+    row, col = oracle.marginals(C, C_, eps, LG, f, z)
+    np.testing.assert_allclose(row, a.astype(np.float64), rtol=1e-13)
+    assert np.abs(col - b).max() > 1e-4                       # the other side is not yet matched
+    g = oracle.log_col_pass(C, eps, b, f)
+    row, col = oracle.marginals(C, C_, eps, LG, f, g)
+    np.testing.assert_allclose(col, b.astype(np.float64), rtol=1e-13)
+
+
 # ------------------------------------------------------------------ library-routine special case
 
 def test_lse_against_scipy():
