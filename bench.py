@@ -8,13 +8,19 @@ column pass each) through fs_iterate, on seeded synthetic inputs that are reside
 the timed region starts.  Rank 0 prints ONE JSON line.  Keys beyond the basic contract:
 
   roofline      dominant kernel (config 4: the single-read fused iteration kernel): algorithmic bytes
-                per launch over its average launch duration, timed with CUDA events on the launching
-                stream, against the measured HBM copy rate of this machine
-  cpu_baseline  the fp64 CPU checker timed on this machine's host cores on a few iterations
+                per launch over its average launch interval against the measured HBM copy rate of this
+                pool.  `frac` is SUSTAINED (the timed region itself); `burst` holds the same for a short
+                loop of single launches from an idle GPU; both carry the SM clock sampled meanwhile and
+                time x clock (SM cycles per launch)
+  other_paths   config 4 on the two-pass path (K streamed twice per iteration): the row pass and the
+                column pass each timed alone, and whole iterations
+  cpu_baseline  the fp64 CPU checker timed on this machine's host cores on a few iterations, with all
+                cores (OpenMP) and on one thread
   e2e           the same metric through fs_solve_host: host buffers in, host buffers out, all
                 host<->device copies inside the timed region
   clocks        SM clock and throttle reasons sampled with nvidia-smi during the timed region
-  other_configs it/s of configurations 1, 2, 3 and 5 from short runs of the same kind (N = 1 only)
+  other_configs it/s of configurations 1, 2, 3 and 5 from short runs of the same kind, each with the kernel
+                path the library chose and the SM clock sampled during it (N = 1 only)
 
 With --impl reference the CPU checker is what gets timed (same config, metric and unit); under a
 multi-process launch only rank 0 runs it.
@@ -115,6 +121,69 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+class NvmlSampler:
+    """SM clock and throttle reasons read through NVML from a thread of this process, every few milliseconds:
+    for timed loops too short for the nvidia-smi child process to see (reading only, nothing is set)."""
+
+    def __init__(self, index: int, period_s: float = 0.004):
+        self.index, self.period, self.samples, self.reasons = index, period_s, [], 0
+        self.thread = None
+        self.stop_flag = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+                self.reasons |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.nv is None:
+            return
+        import threading
+        self.samples, self.reasons, self.stop_flag = [], 0, False
+        self.thread = threading.Thread(target=self._loop, daemon=True)
+        self.thread.start()
+
+    def stop(self):
+        if self.nv is None or self.thread is None:
+            return None
+        self.stop_flag = True
+        self.thread.join(timeout=2)
+        self.thread = None
+        if not self.samples:
+            return None
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        try:
+            smmax = nv.nvmlDeviceGetMaxClockInfo(self.handle, nv.NVML_CLOCK_SM)
+        except Exception:
+            smmax = None
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": smmax,
+                "reasons": sorted(k for k, bit in names.items() if self.reasons & bit), "samples": len(self.samples)}
+
+
+def with_clock(entry, seconds_per_unit, clocks, key):
+    """Adds the sampled median SM clock and time x clock (SM cycles per unit of work) to a result entry."""
+    entry["clocks"] = clocks
+    if clocks and clocks.get("sm_mhz"):
+        entry[key] = seconds_per_unit * clocks["sm_mhz"] * 1e6
+    return entry
+
+
 def visible_device_index(local_rank: int) -> int:
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -166,8 +235,23 @@ def cpu_baseline(w, budget_s=12.0):
         iters += 1
     value = iters * frac / total
     sample = f"{iters} full iteration(s) of the same workload" + (" for 1 of the batch's problems" if w.nbatch > 1 else "")
-    return {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample,
-            "seconds": total}
+    out = {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample,
+           "seconds": total}
+    # the same checker on ONE thread (its OpenMP loops keep every sum's order, so only the time changes)
+    try:
+        import ctypes
+        omp = ctypes.CDLL("libgomp.so.1")
+        omp.omp_get_max_threads.restype = ctypes.c_int
+        before = omp.omp_get_max_threads()
+        omp.omp_set_num_threads(1)
+        try:
+            d1, f1 = oracle_iterate(w, 1)
+        finally:
+            omp.omp_set_num_threads(before)
+        out["single_thread"] = {"value": f1 / d1, "unit": UNIT, "cores": 1, "sample": "1 full iteration", "seconds": d1}
+    except OSError:
+        out["single_thread"] = None
+    return out
 
 
 def run_reference(args, w, world):
@@ -196,7 +280,7 @@ def run_reference(args, w, world):
 
 # ------------------------------------------------------------------------------------------ GPU arm
 
-def time_config(fs, torch, dev, stream, w, steps=3):
+def time_config(fs, torch, dev, stream, w, steps=3, device_index=0):
     """it/s of one configuration through fs_iterate (device-resident inputs, CUDA events)."""
     M = torch.from_numpy(w.matrix).to(dev)
     a = torch.from_numpy(w.a).to(dev)
@@ -211,9 +295,12 @@ def time_config(fs, torch, dev, stream, w, steps=3):
             fs.fs_reset(h, stream)
             fs.fs_iterate(h, w.iters, stream)
 
+        path = fs.fs_iteration_path(h)
         for _ in range(3):
             step()
         stream.synchronize()
+        sampler = NvmlSampler(device_index)
+        sampler.start()
         e0 = torch.cuda.Event(enable_timing=True)
         e1 = torch.cuda.Event(enable_timing=True)
         e0.record(stream)
@@ -221,16 +308,18 @@ def time_config(fs, torch, dev, stream, w, steps=3):
             step()
         e1.record(stream)
         stream.synchronize()
+        clocks = sampler.stop()
         ms = e0.elapsed_time(e1)
         row, col = fs.fs_marginal_error(h, 1, w.nbatch, stream)
     finally:
         fs.fs_destroy(h)
     its = steps * w.iters
-    return {"workload": f"n={w.n}" + (f" N={w.nbatch}" if w.nbatch > 1 else "") + (" log" if w.domain else " scaling"),
+    return with_clock({"path": path, "workload": f"n={w.n}" + (f" N={w.nbatch}" if w.nbatch > 1 else "") + (" log" if w.domain else " scaling"),
             "value": its / (ms * 1e-3), "unit": UNIT, "us_per_iteration": ms * 1e3 / its, "steps": steps,
             "iterations_per_step": w.iters,
             "effective_gbs_2n2": 2 * w.n * w.n * 4 * its / (ms * 1e-3) / 1e9,
-            "final_row_marginal_l1_max": float(row.max()), "final_col_marginal_l1_max": float(col.max())}
+            "final_row_marginal_l1_max": float(row.max()), "final_col_marginal_l1_max": float(col.max())},
+                      ms * 1e-3 / its, clocks, "sm_cycles_per_iteration")
 
 
 def run_sharded(args, rank, local_rank, world):
@@ -351,14 +440,22 @@ def run_ours(args, w, rank, local_rank, world):
     row_err, col_err = fs.fs_marginal_error(h, 1, w.nbatch, stream)
     t_ms, total_iters = fsdist.aggregate(elapsed_ms, args.steps * w.iters, dev)
 
-    # dominant kernel: timed with CUDA events on the launching stream, right after the timed region
+    # dominant kernel.  Two regimes are reported and named: "sustained" = the timed region itself (seconds of
+    # back-to-back iterations, SM clock settled under the power cap), which is what `frac` describes, and
+    # "burst" = a short loop of single launches from an idle GPU, timed with CUDA events on the launching stream
+    # right after the timed region (SM clock near its maximum).
     peaks, peak_kind = measured_peaks()
-    fused = w.nbatch == 1 and w.domain == workloads.DOMAIN_SCALING and w.n >= 6144 and w.n % 4 == 0
-    reps = 20
+    devidx = visible_device_index(local_rank)
+    path = fs.fs_iteration_path(h)
+    n2 = w.n * w.n * 4
+    its_region = args.steps * w.iters
 
-    def timed(fn):
+    def timed(fn, reps):
         fn()
         stream.synchronize()
+        time.sleep(0.5)                       # from an idle GPU
+        smp = NvmlSampler(devidx, period_s=0.001)
+        smp.start()
         k0 = torch.cuda.Event(enable_timing=True)
         k1 = torch.cuda.Event(enable_timing=True)
         k0.record(stream)
@@ -366,53 +463,85 @@ def run_ours(args, w, rank, local_rank, world):
             fn()
         k1.record(stream)
         stream.synchronize()
-        return k0.elapsed_time(k1) * 1e-3 / reps
+        return k0.elapsed_time(k1) * 1e-3 / reps, smp.stop()
 
-    fused_log = w.nbatch == 1 and w.domain == workloads.DOMAIN_LOG and 4096 <= w.n <= 16384 and w.n % 4 == 0
-    n2 = w.n * w.n * 4
-    if fused_log:
-        # one launch of the fused log kernel per iteration; the interval also holds its stage-2 kernel
-        per_launch_s = timed(lambda: fs.fs_iterate(h, 1, stream))
-        kernel, bytes_launch = "fused_log_iteration_kernel", n2
+    # (kernel, algorithmic bytes per launch, launches of it per iteration, burst callable, repeats, note)
+    if path == "fused_log":
+        kernel, bytes_launch, per_iter = "fused_log_iteration_kernel", n2, 1
+        burst_fn, reps = (lambda: fs.fs_iterate(h, 1, stream)), 20
         note = ("one launch per iteration reads C once (n*n*4 bytes), one ex2 per element; the timed interval "
                 "includes the stage-2 kernel that follows it")
-    elif fused:
-        # one launch of the fused kernel per iteration; the interval also holds the stage-2 kernel
-        # that follows it (a few microseconds), so the kernel's own rate is slightly understated
-        per_launch_s = timed(lambda: fs.fs_iterate(h, 1, stream))
-        kernel, bytes_launch = "fused_iteration_kernel", n2
+    elif path == "fused":
+        kernel, bytes_launch, per_iter = "fused_iteration_kernel", n2, 1
+        burst_fn, reps = (lambda: fs.fs_iterate(h, 1, stream)), 20
         note = ("one launch per iteration reads K once (n*n*4 bytes); the timed interval includes the "
                 "col_finish_kernel that follows it")
-    elif w.nbatch == 1 and w.domain == workloads.DOMAIN_SCALING and w.n <= 5120 and w.n % 4 == 0 and w.n >= 8:
+    elif path in ("resident", "persistent"):
         # all iterations of a step in one launch of a persistent kernel; K is read from HBM once per launch
-        # and then served from shared memory (n <= ~720) or from L2 and shared memory
-        reps = 5
-        per_launch_s = timed(lambda: fs.fs_iterate(h, w.iters, stream))
-        kernel = "resident_iterations_kernel" if w.n <= 720 else "persistent_iterations_kernel"
-        bytes_launch = n2 * w.iters
+        # and then served from shared memory or from L2 and shared memory
+        kernel, bytes_launch, per_iter = path + "_iterations_kernel", n2 * w.iters, 1.0 / w.iters
+        burst_fn, reps = (lambda: fs.fs_iterate(h, w.iters, stream)), 5
         note = ("one launch runs all %d iterations of a step; bytes = one read of K per iteration (n*n*4 each), served "
                 "from on-chip memory and L2, not HBM: the kernel is latency-bound and this fraction is not an HBM "
                 "utilisation" % w.iters)
-    elif w.nbatch > 1:
-        per_launch_s = timed(lambda: fs.fs_row_pass(h, stream))
-        kernel, bytes_launch = "batched_tc_kernel", n2 + 4 * w.n * w.nbatch * 4
+    elif path == "batched_tc":
+        kernel, bytes_launch, per_iter = "batched_tc_kernel", n2 + 4 * w.n * w.nbatch * 4, 2
+        burst_fn, reps = (lambda: fs.fs_row_pass(h, stream)), 20
         note = ("one batched pass, one launch: K as two bf16 terms (n*n*4 bytes) + operand and result vectors; the "
                 "split-K partial tiles are exchanged inside the cluster and the update is applied in the same "
                 "kernel; tensor work is 3 bf16 products per useful one")
     else:
-        per_launch_s = timed(lambda: fs.fs_row_pass(h, stream))
-        kernel, bytes_launch = ("log_row_pass_kernel" if w.domain else "row_pass_kernel"), n2
-        note = "one row pass streams the matrix once (n*n*4 bytes)"
-    achieved = bytes_launch / per_launch_s / 1e9
+        kernel = {"two_pass": "row_pass_kernel", "two_pass_log": "log_row_pass_kernel"}.get(path, "batched_fma_kernel")
+        bytes_launch, per_iter = n2, 2
+        burst_fn, reps = (lambda: fs.fs_row_pass(h, stream)), 20
+        note = "one pass streams the matrix once (n*n*4 bytes); an iteration is a row pass and a column pass"
+    per_launch_sustained_s = elapsed_ms * 1e-3 / (its_region * per_iter)
+    achieved = bytes_launch / per_launch_sustained_s / 1e9
+    per_launch_burst_s, burst_clocks = timed(burst_fn, reps)
+    burst_gbs = bytes_launch / per_launch_burst_s / 1e9
     traffic = TRAFFIC_BYTES_PER_LAUNCH.get((kernel, w.n)) if args.traffic_bytes is None else args.traffic_bytes
-    roof = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": achieved / peaks["hbm_gbs"],
-            "peak_source": "of measured (MEASURED_PEAKS.json hbm_gbs, burst copy rate)" if peak_kind == "measured"
-            else "of fallback",
-            "algorithmic_bytes_per_launch": bytes_launch, "us_per_launch": per_launch_s * 1e6, "traffic": traffic,
-            "note": note,
+    peak_src = ("of measured (MEASURED_PEAKS.json hbm_gbs, copy rate)" if peak_kind == "measured" else "of fallback")
+    roof = {"bound": "hbm", "kernel": kernel, "path": path, "achieved": achieved, "peak": peaks["hbm_gbs"],
+            "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src,
+            "regime": "sustained: the timed region itself, elapsed / launches of this kernel in it "
+                      "(the interval also holds the small kernels that run between its launches)",
+            "frac_of_nominal_8000_gbs": achieved / 8000.0,
+            "algorithmic_bytes_per_launch": bytes_launch, "us_per_launch": per_launch_sustained_s * 1e6,
+            "traffic": traffic, "note": note,
+            "burst": with_clock({"regime": "%d single launches from an idle GPU, CUDA events on the launching stream" % reps,
+                                 "achieved": burst_gbs, "frac": burst_gbs / peaks["hbm_gbs"],
+                                 "us_per_launch": per_launch_burst_s * 1e6}, per_launch_burst_s, burst_clocks,
+                                "sm_cycles_per_launch"),
             # BASELINE's accounting (every iteration streams 2 n^2 elements) applied to the timed region
-            "iteration_effective_gbs_2n2": 2 * n2 * (args.steps * w.iters) / (elapsed_ms * 1e-3) / 1e9}
+            "iteration_effective_gbs_2n2": 2 * n2 * its_region / (elapsed_ms * 1e-3) / 1e9}
+    with_clock(roof, per_launch_sustained_s, clocks, "sm_cycles_per_launch")
+
+    # the literal dense-K passes of the same configuration: row pass and two-stage column pass, K streamed twice
+    # per iteration (FS_OPT_FUSED = 0), each pass timed alone with CUDA events and as whole iterations
+    other_paths = None
+    if world == 1 and path == "fused" and not args.headline_only:
+        def gbs(sec):
+            return {"us": sec * 1e6, "gbs": n2 / sec / 1e9, "frac_of_measured": n2 / sec / 1e9 / peaks["hbm_gbs"],
+                    "frac_of_nominal_8000_gbs": n2 / sec / 1e9 / 8000.0}
+        fs.fs_set_option(h, fs.FS_OPT_FUSED, 0)
+        assert fs.fs_iteration_path(h) == "two_pass"
+        fs.fs_reset(h, stream)
+        fs.fs_iterate(h, 10, stream)
+        row_s, row_clk = timed(lambda: fs.fs_row_pass(h, stream), 100)
+        col_s, col_clk = timed(lambda: fs.fs_col_pass(h, stream), 100)
+        fs.fs_reset(h, stream)
+        it_s, it_clk = timed(lambda: fs.fs_iterate(h, w.iters, stream), 2)
+        fs.fs_set_option(h, fs.FS_OPT_FUSED, 1)
+        other_paths = {"two_pass": {
+            "what": "row_pass_kernel, then col_partial_kernel + col_finish_kernel: K is read from HBM twice per iteration",
+            "row_pass": with_clock(dict(gbs(row_s), launches_timed=100), row_s, row_clk, "sm_cycles_per_launch"),
+            "col_pass": with_clock(dict(gbs(col_s), launches_timed=100), col_s, col_clk, "sm_cycles_per_launch"),
+            "iterations": with_clock({"value": w.iters / it_s, "unit": UNIT, "us_per_iteration": it_s / w.iters * 1e6,
+                                      "iterations_timed": 2 * w.iters,
+                                      "gbs_2n2": 2 * n2 * w.iters / it_s / 1e9,
+                                      "frac_of_measured": 2 * n2 * w.iters / it_s / 1e9 / peaks["hbm_gbs"],
+                                      "frac_of_nominal_8000_gbs": 2 * n2 * w.iters / it_s / 1e9 / 8000.0},
+                                     it_s / w.iters, it_clk, "sm_cycles_per_iteration")}}
 
     # the other four configurations, briefly (single GPU runs only): same step definition, fewer steps
     others = None
@@ -421,7 +550,8 @@ def run_ours(args, w, rank, local_rank, world):
         for cfg in (1, 2, 3, 5):
             try:
                 time.sleep(1.0)  # each short run starts from an idle GPU, not from the headline run's power state
-                others[f"config{cfg}"] = time_config(fs, torch, dev, stream, workloads.make(cfg, want_cost=None if cfg == 3 else False))
+                others[f"config{cfg}"] = time_config(fs, torch, dev, stream, workloads.make(cfg, want_cost=None if cfg == 3 else False),
+                                                     device_index=devidx)
             except Exception as exc:  # a failure here must not lose the headline line
                 others[f"config{cfg}"] = {"error": repr(exc)}
         # the one table the paper prints for this path (Table 1: 15 iterations, n = 5000; 1 problem 0.32 s,
@@ -431,7 +561,7 @@ def run_ours(args, w, rank, local_rank, world):
             for label, nb in (("one_problem", 1), ("vectorized_500", 500)):
                 wt = workloads.make(5, n=5000, nbatch=nb, want_cost=False)
                 wt.iters = 15
-                r = time_config(fs, torch, dev, stream, wt, steps=5)
+                r = time_config(fs, torch, dev, stream, wt, steps=5, device_index=devidx)
                 t1[label] = {"seconds_for_15_iterations": 15 * r["us_per_iteration"] * 1e-6,
                              "paper_seconds": 0.32 if nb == 1 else 0.31,
                              "final_row_marginal_l1_max": r["final_row_marginal_l1_max"]}
@@ -484,7 +614,7 @@ def run_ours(args, w, rank, local_rank, world):
             "warmup": max(3, args.warmup), "ms_per_step": t_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": config_dict(w, args, world), "gpu_launches": int(launches), "clocks": clocks,
-            "e2e": e2e, "roofline": roof, "cpu_baseline": base, "other_configs": others,
+            "e2e": e2e, "roofline": roof, "cpu_baseline": base, "other_paths": other_paths, "other_configs": others,
             "final_row_marginal_l1": float(row_err[0]), "final_col_marginal_l1": float(col_err[0])}
     print(json.dumps(line), flush=True)
 

@@ -132,12 +132,16 @@ int fs_col_pass(fs_solver *s, void *stream);
  */
 int fs_marginal_error(fs_solver *s, int norm, double *row_err, double *col_err, void *stream);
 
-/* Copy the current scalings (scaling domain: u, v; log domain: f, g) into caller DEVICE buffers of
+/* fs_scalings -- the outputs of Algorithm 1: the scaling vectors u, v of P* = diag(u) K diag(v) (Section 1)
+ * as they stand after the iterations run so far.  Copies the current scalings (scaling domain: u, v; log
+ * domain: the duals f = eps log u, g = eps log v) into caller DEVICE buffers of
  * [nbatch][n] floats each; either may be NULL.  Synchronises `stream`; reports FS_ERR_NONFINITE
  * like fs_marginal_error (the copy is still made). */
 int fs_scalings(fs_solver *s, float *u_dev_out, float *v_dev_out, void *stream);
 
-/* Overwrite the current scalings (resume from a checkpoint).  DEVICE [nbatch][n]; either may be
+/* fs_set_scalings -- replace Algorithm 1's start state u = v = 1 (its first line) by given vectors, or
+ * resume from a checkpoint: (u, v) is the whole state of the iteration (fixed-point map T of the convergence
+ * appendix), so fs_scalings + fs_set_scalings is a complete checkpoint.  DEVICE [nbatch][n]; either may be
  * NULL (left as is).  Asynchronous on `stream`. */
 int fs_set_scalings(fs_solver *s, const float *u_dev, const float *v_dev, void *stream);
 
@@ -169,7 +173,8 @@ int fs_set_damping(fs_solver *s, double eta);
  * extra non-updating row pass is run for it.  0 switches the trace off.  Clears the trace. */
 int fs_set_error_trace(fs_solver *s, int32_t check_every);
 
-/* Read the trace: up to `cap` entries are written to the HOST arrays (either may be NULL);
+/* fs_error_trace -- the curve err_a(t) = ||P^t 1 - a|| that Section 5.3 plots against the iteration count
+ * (2-norm there; the 1-norm is recorded beside it).  Up to `cap` entries are written to the HOST arrays (either may be NULL);
  * *count receives the number recorded so far; iteration numbers are m, 2m, 3m, ...
  * Synchronises `stream`. */
 int fs_error_trace(fs_solver *s, double *l1_out, double *l2_out, int32_t cap, int32_t *count, void *stream);
@@ -179,6 +184,18 @@ int fs_error_trace(fs_solver *s, double *l1_out, double *l2_out, int32_t cap, in
 int fs_block_errors(fs_solver *s, double *block_l1_out);
 
 int fs_set_option(fs_solver *s, int option, int64_t value);
+
+/* fs_iteration_path -- which kernels fs_iterate runs for this handle as it is configured now (size, domain,
+ * batch, options, error trace).  All of them compute the loop body of Algorithm 1; they differ in how often K
+ * crosses HBM.  Returns a static string:
+ *   "two_pass"      row pass + two-stage column pass, K read twice per iteration
+ *   "two_pass_log"  the same in the log domain
+ *   "fused"         single-read fused iteration (scaling domain)      "fused_log"  its log-domain form
+ *   "resident"      all iterations in one launch, K in one cluster's shared memory
+ *   "persistent"    all iterations in one cooperative launch, K in L2 and shared memory
+ *   "batched_tc"    shared-K batch on tensor cores                     "batched_fma"  its fp32 FMA engine
+ * (A diagnostic of this implementation; the paper has no counterpart.) */
+const char *fs_iteration_path(const fs_solver *s);
 
 /* Number of iterations enqueued since creation / fs_reset. */
 int64_t fs_iterations_done(const fs_solver *s);
@@ -196,7 +213,8 @@ int fs_fused_log_fallbacks(fs_solver *s, int64_t *count_out, void *stream);
 int fs_destroy(fs_solver *s);
 
 /*
- * fs_solve_host -- the whole path from HOST buffers: allocates device memory, copies the matrix and
+ * fs_solve_host -- Algorithm 1 from its inputs (a, b, the matrix, eps, IterMax) to its outputs (u, v) in one
+ * call, with every buffer on the HOST: allocates device memory, copies the matrix and
  * the marginals to the device, runs `iters` iterations, copies the scalings back and frees everything.
  * All pointers are HOST pointers; M_host is n x n with leading dimension ld; a, b, u_out, v_out are
  * [nbatch][n]; row_err_l1_out is [nbatch] or NULL (1-norm row marginal error of the final state).

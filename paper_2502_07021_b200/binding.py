@@ -43,6 +43,7 @@ _SIGNATURES = {
     "fs_error_trace": (_int, [_vp, _vp, _vp, _i32, ctypes.POINTER(_i32), _vp]),
     "fs_block_errors": (_int, [_vp, _vp]),
     "fs_set_option": (_int, [_vp, _int, _i64]),
+    "fs_iteration_path": (ctypes.c_char_p, [_vp]),
     "fs_iterations_done": (_i64, [_vp]),
     "fs_launch_count": (_i64, [_vp]),
     "fs_fused_log_fallbacks": (_int, [_vp, ctypes.POINTER(_i64), _vp]),
@@ -201,6 +202,10 @@ def fs_block_errors(s, c):
 
 def fs_set_option(s, option, value):
     _check(lib().fs_set_option(s, option, value), "fs_set_option")
+
+
+def fs_iteration_path(s):
+    return lib().fs_iteration_path(s).decode()
 
 
 def fs_iterations_done(s):

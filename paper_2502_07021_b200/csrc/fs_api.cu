@@ -1,6 +1,6 @@
 // C ABI of libfs_b200.so: handle, argument validation, the iteration driver (plain launches or
 // captured CUDA graphs) and the result calls.  See include/fs.h for the contract of every
-// entry point; the kernels are in passes.cu, batched.cu and setup.cu.
+// entry point; fs_internal.cuh lists the translation units that hold the kernels.
 #include <math.h>
 #include <stdio.h>
 #include <string.h>
@@ -91,6 +91,7 @@ void destroy_solver(fs_solver *s) {
     free_dev(s->tiles_dev);
     free_dev(s->fused_tiles_dev);
     free_dev(s->fused_partials);
+    free_dev(s->fused_u_prev);
     free_dev(s->fused_log_tmp);
     free_dev(s->persistent_scratch);
     free_dev(s->offsets_dev);
@@ -168,8 +169,30 @@ bool use_fused(const fs_solver *s) {
     return s->n >= kFusedAutoMinN;
 }
 
+// Which kernels fs_iterate runs for this handle as it is configured now.
+enum IterPath { PATH_TWO_PASS, PATH_TWO_PASS_LOG, PATH_FUSED, PATH_FUSED_LOG, PATH_RESIDENT, PATH_PERSISTENT, PATH_BATCHED_TC,
+                PATH_BATCHED_FMA };
+
+IterPath iteration_path(const fs_solver *s) {
+    const bool traced = s->check_every != 0;
+    if (s->nbatch > 1) return use_tc(s) ? PATH_BATCHED_TC : PATH_BATCHED_FMA;
+    if (s->resident.enabled && s->resident_mode != 0 && !traced) return PATH_RESIDENT;
+    if (s->persistent.enabled && !traced &&
+        (s->persistent_mode == 2 || (s->persistent_mode == 1 && s->n <= kPersistentAutoMaxN && s->fused_mode != 2)))
+        return PATH_PERSISTENT;
+    if (use_fused(s)) return s->domain == FS_DOMAIN_LOG ? PATH_FUSED_LOG : PATH_FUSED;
+    return s->domain == FS_DOMAIN_LOG ? PATH_TWO_PASS_LOG : PATH_TWO_PASS;
+}
+
 void enqueue_fused_rows(fs_solver *s, cudaStream_t st, int64_t &launches) {
-    fsk_fused_iteration(s->fused, s->mat, s->mat_ld, s->n, s->fused_tiles_dev, s->fused_ntiles, s->y, s->a, s->x,
+    const float *u_prev = s->x;
+    if (s->eta != 1.f) {
+        // relaxed update: the kernel reads the old u in many threads while it overwrites u, so it gets a copy
+        fsk_scale(s->x, s->n, 1.0, s->fused_u_prev, st);
+        launches += 1;
+        u_prev = s->fused_u_prev;
+    }
+    fsk_fused_iteration(s->fused, s->mat, s->mat_ld, s->n, s->fused_tiles_dev, s->fused_ntiles, s->y, s->a, s->x, u_prev,
                         s->rowdiff, s->fused_partials, s->eta, s->status, st);
     launches += 1;
 }
@@ -382,6 +405,7 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
             const size_t pbytes = sizeof(float) * planes * (size_t)s->fused.nclusters * (size_t)n;
             FS_CU(cudaMalloc(&s->fused_partials, pbytes));
             FS_CU(cudaMemsetAsync(s->fused_partials, 0, pbytes, st));
+            if (domain == FS_DOMAIN_SCALING) FS_CU(cudaMalloc(&s->fused_u_prev, sizeof(float) * (size_t)n));
             if (domain == FS_DOMAIN_LOG) {
                 const size_t tbytes = 64; // stage 2's count of finished CTAs
                 FS_CU(cudaMalloc(&s->fused_log_tmp, tbytes));
@@ -497,8 +521,9 @@ int fs_iterate(fs_solver *s, int32_t k, void *stream) {
     const int ce = s->check_every;
     int chunk = kGraphChunk;
     if (ce > 0 && ce <= kGraphChunk) chunk = ce * (kGraphChunk / ce);
+    const IterPath path = iteration_path(s);
     // small problems without an error trace: all k iterations in one launch of the K-resident kernel
-    if (k > 0 && s->resident.enabled && s->resident_mode != 0 && ce == 0) {
+    if (k > 0 && path == PATH_RESIDENT) {
         FS_CU(fsk_resident_iterate(s->resident, s->mat, s->mat_ld, s->n, k, s->a, s->b, s->x, s->y, s->rowdiff, s->coldiff,
                                    s->eta, s->status, st));
         s->launches += 1;
@@ -507,8 +532,7 @@ int fs_iterate(fs_solver *s, int32_t k, void *stream) {
     }
     // mid-size problems without an error trace: all k iterations in one cooperative launch that reads K once
     // per iteration (automatic while K fits the L2 cache, unless the fused path was asked for explicitly)
-    if (k > 0 && s->persistent.enabled && ce == 0 &&
-        (s->persistent_mode == 2 || (s->persistent_mode == 1 && s->n <= kPersistentAutoMaxN && s->fused_mode != 2))) {
+    if (k > 0 && path == PATH_PERSISTENT) {
         // at most 2^20 iterations per launch: the grid barrier's 32-bit arrival counter must not wrap
         for (int32_t done = 0; done < k;) {
             const int32_t len = std::min<int32_t>(k - done, 1 << 20);
@@ -684,6 +708,20 @@ int fs_error_trace(fs_solver *s, double *l1_out, double *l2_out, int32_t cap, in
         }
     }
     return FS_OK;
+}
+
+const char *fs_iteration_path(const fs_solver *s) {
+    if (!s) return "";
+    switch (iteration_path(s)) {
+    case PATH_TWO_PASS: return "two_pass";
+    case PATH_TWO_PASS_LOG: return "two_pass_log";
+    case PATH_FUSED: return "fused";
+    case PATH_FUSED_LOG: return "fused_log";
+    case PATH_RESIDENT: return "resident";
+    case PATH_PERSISTENT: return "persistent";
+    case PATH_BATCHED_TC: return "batched_tc";
+    default: return "batched_fma";
+    }
 }
 
 int64_t fs_iterations_done(const fs_solver *s) { return s ? s->iter_done : -1; }

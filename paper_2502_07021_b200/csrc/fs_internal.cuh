@@ -2,7 +2,7 @@
 //   fs_api.cu          handle, validation, iteration driver (graphs), result calls: the C ABI
 //   passes.cu          single-problem row / column passes, scaling and log domain (two-pass path)
 //   fused.cu           single-read fused iteration, scaling domain (clusters, bulk copies, DSMEM)
-//   fused_log.cu       the same for the log domain (opt-in)
+//   fused_log.cu       the same for the log domain (automatic for 4096 <= n <= 16384)
 //   resident.cu        K-resident persistent kernel for small n
 //   persistent.cu      grid-persistent single-read iterations for mid-size n (cooperative launch)
 //   batched_tc.cu      shared-K batched passes on tcgen05 tensor cores;  batched.cu  fp32 FMA engine
@@ -110,6 +110,7 @@ struct fs_solver {
     FsRowTile *fused_tiles_dev = nullptr;
     int fused_ntiles = 0;
     float *fused_partials = nullptr;
+    float *fused_u_prev = nullptr;          // scaling-domain fused iteration with eta != 1: u before the iteration
     float *fused_log_tmp = nullptr;         // fused log iteration: stage 2's count of finished CTAs (one int)
     int64_t iter_done = 0;
     int64_t launches = 0;
@@ -170,8 +171,8 @@ int fsk_pass_launches_col();
 // ---- fused.cu ----------------------------------------------------------------------------
 FsFusedPlan fsk_fused_plan(int64_t n, bool vec);
 cudaError_t fsk_fused_iteration(const FsFusedPlan &p, const float *K, int64_t ld, int64_t n, const FsRowTile *tiles,
-                                int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials,
-                                float eta, FsDeviceStatus *status, cudaStream_t st);
+                                int ntiles, const float *v, const float *a, float *u, const float *u_prev, float *rowdiff,
+                                float *partials, float eta, FsDeviceStatus *status, cudaStream_t st);
 
 // ---- resident.cu -------------------------------------------------------------------------
 FsResidentPlan fsk_resident_plan(int64_t n);

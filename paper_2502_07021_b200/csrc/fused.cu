@@ -43,7 +43,7 @@ template <int F, int R>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, int nclusters, int nstages,
                        const FsRowTile *__restrict__ tiles, int ntiles, const float *__restrict__ v,
-                       const float *__restrict__ a, float *__restrict__ u, float *__restrict__ rowdiff,
+                       const float *__restrict__ a, float *u, const float *u_prev, float *__restrict__ rowdiff,
                        float *__restrict__ partials, float eta, FsDeviceStatus *status) {
     extern __shared__ uint8_t smem_raw[];
     constexpr int W = F * 1024;
@@ -177,11 +177,15 @@ fused_iteration_kernel(const float *__restrict__ K, int64_t ld, int n, int S, in
         int k = 0;
         for (int tl = cluster; tl < ntiles && ok; tl += nclusters) {
             const FsRowTile tile = tiles[tl];
-            // the tile's marginal entries and old scalings (at most 32 rows): one load per tile, lane i keeps row i
+            // the tile's marginal entries and old scalings (at most 32 rows): one load per tile, lane i keeps row i.
+            // Every accumulate warp of every CTA of the cluster needs the OLD u_i of a row for the relaxed update,
+            // while one thread overwrites u as rows complete and the warps are coupled only through the ring: with
+            // eta != 1 the old values therefore come from u_prev, a copy made before the launch that nobody writes.
+            // With eta == 1 the old value only feeds the residual, in the thread that also does the write (u_prev == u).
             float a_lane = 1.f, uo_lane = 0.f;
             if (tile.begin + lane < tile.end) {
                 a_lane = a[tile.begin + lane];
-                uo_lane = u[tile.begin + lane];
+                uo_lane = __ldcg(u_prev + tile.begin + lane);
             }
             for (int row = tile.begin; row < tile.end; row += R, ++k) {
                 const int cnt = min(R, tile.end - row);
@@ -270,13 +274,13 @@ void fill_cluster_launch(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int
 
 template <int F, int R>
 cudaError_t launch_fused(const FsFusedPlan &p, cudaStream_t st, const float *K, int64_t ld, int n, const FsRowTile *tiles,
-                         int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials, float eta,
-                         FsDeviceStatus *status) {
+                         int ntiles, const float *v, const float *a, float *u, const float *u_prev, float *rowdiff,
+                         float *partials, float eta, FsDeviceStatus *status) {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[2];
     fill_cluster_launch(cfg, attr, p.S, p.nclusters, fused_smem_bytes(F, R, p.nstages), st);
     return cudaLaunchKernelEx(&cfg, fused_iteration_kernel<F, R>, K, ld, n, p.S, p.nclusters, p.nstages, tiles, ntiles, v, a,
-                              u, rowdiff, partials, eta, status);
+                              u, u_prev, rowdiff, partials, eta, status);
 }
 
 template <int F, int R>
@@ -338,14 +342,16 @@ FsFusedPlan fsk_fused_plan(int64_t n, bool vec) {
 }
 
 // One fused iteration minus the final divide: writes u, rowdiff and the per-cluster column partials
-// [nclusters][n]; the caller runs the stage-2 kernel over them.
+// [nclusters][n]; the caller runs the stage-2 kernel over them.  u_prev holds the scalings before this
+// iteration: a separate copy of u when eta != 1 (the relaxed update of Section 3.3 reads the old u_i in
+// many threads while u is overwritten), u itself when eta == 1.
 cudaError_t fsk_fused_iteration(const FsFusedPlan &p, const float *K, int64_t ld, int64_t n, const FsRowTile *tiles,
-                                int ntiles, const float *v, const float *a, float *u, float *rowdiff, float *partials,
-                                float eta, FsDeviceStatus *status, cudaStream_t st) {
+                                int ntiles, const float *v, const float *a, float *u, const float *u_prev, float *rowdiff,
+                                float *partials, float eta, FsDeviceStatus *status, cudaStream_t st) {
     switch (p.F) {
-    case 2: return launch_fused<2, 8>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
-    case 4: return launch_fused<4, 4>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
-    case 8: return launch_fused<8, 2>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
-    default: return launch_fused<16, 1>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, rowdiff, partials, eta, status);
+    case 2: return launch_fused<2, 8>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, u_prev, rowdiff, partials, eta, status);
+    case 4: return launch_fused<4, 4>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, u_prev, rowdiff, partials, eta, status);
+    case 8: return launch_fused<8, 2>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, u_prev, rowdiff, partials, eta, status);
+    default: return launch_fused<16, 1>(p, st, K, ld, (int)n, tiles, ntiles, v, a, u, u_prev, rowdiff, partials, eta, status);
     }
 }

@@ -175,25 +175,32 @@ void fill_launch(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int S, size
     cfg.numAttrs = 1;
 }
 
-// One-off function attributes: the largest dynamic shared memory any configuration uses, and clusters
-// of 16 CTAs (beyond the portable size of 8).
-bool set_attributes_once() {
-    static int state = 0; // 0 = not tried, 1 = ok, -1 = failed
-    if (state == 0) {
-        const bool ok = cudaFuncSetAttribute(resident_iterations_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             227 * 1024) == cudaSuccess &&
-                        cudaFuncSetAttribute(resident_iterations_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed,
-                                             1) == cudaSuccess;
-        if (!ok) cudaGetLastError();
-        state = ok ? 1 : -1;
+// Function attributes: the largest dynamic shared memory any configuration uses, and clusters of 16 CTAs
+// (beyond the portable size of 8).  Function attributes belong to a device's context, so the outcome is
+// remembered per device: a process that builds solvers on a second GPU sets them there too.
+bool set_attributes_for_current_device() {
+    constexpr int kMaxDevices = 64;
+    static int state[kMaxDevices] = {}; // per device: 0 = not tried, 1 = ok, -1 = failed
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
     }
-    return state == 1;
+    const bool cached = dev >= 0 && dev < kMaxDevices;
+    if (cached && state[dev] != 0) return state[dev] == 1;
+    const bool ok = cudaFuncSetAttribute(resident_iterations_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         227 * 1024) == cudaSuccess &&
+                    cudaFuncSetAttribute(resident_iterations_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed,
+                                         1) == cudaSuccess;
+    if (!ok) cudaGetLastError();
+    if (cached) state[dev] = ok ? 1 : -1;
+    return ok;
 }
 
 bool configure(int n, int S, size_t *smem_out, int *m_out) {
     const int m = (n + S - 1) / S;
     const size_t smem = resident_smem_bytes(n, S, m);
-    if (smem > 227 * 1024 || !set_attributes_once()) return false;
+    if (smem > 227 * 1024 || !set_attributes_for_current_device()) return false;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     fill_launch(cfg, attr, S, smem, nullptr);

@@ -35,11 +35,11 @@ def test_every_declared_symbol_is_exported_and_bound(lib):
 
 def test_strerror_covers_all_codes(lib):
     seen = set()
-    for code in range(0, -11, -1):
+    for code in range(0, -13, -1):
         msg = lib.fs_strerror(code).decode()
         assert msg and msg != "unknown error code"
         seen.add(msg)
-    assert len(seen) == 11
+    assert len(seen) == 13
     assert lib.fs_strerror(-99).decode() == "unknown error code"
 
 

@@ -3,13 +3,16 @@
 allocation may cause, a plug-in that only receives input and output buffers).  Its partial sums
 live in a fixed array inside the library, so every call shares that array and finds the previous
 call's data in it.  The test therefore makes TWO calls in a row, the second on a different,
-smaller problem, and checks each against the regular column pass (fs_create + fs_col_pass).
+smaller problem, and checks each against the regular column pass (fs_create + fs_col_pass) and
+against the fp64 CPU checker's column half-step, so that an error common to both GPU paths cannot
+pass.  A third case runs the largest size the fixed array admits.
 
 Collected last on purpose: a failure here cannot hide the result of any other test.
 """
 import numpy as np
 import pytest
 
+import oracle
 from paper_2502_07021_b200 import binding as fs
 from paper_2502_07021_b200 import workloads
 
@@ -50,6 +53,27 @@ def test_static_column_pass_matches_regular_on_two_calls_in_a_row():
         got, ref = v.cpu().numpy().astype(np.float64), v_ref.cpu().numpy().astype(np.float64)
         assert np.all(np.isfinite(got))
         assert np.max(np.abs(got - ref) / ref) < 2e-6, n
+        v_or, _ = oracle.col_pass(w.K, oracle.KIND_KERNEL, w.eps, bn.cpu().numpy(), u.cpu().numpy())
+        assert np.max(np.abs(got - v_or) / v_or) < 2e-6, n
+
+
+def test_static_column_pass_at_its_largest_size_against_the_checker():
+    import torch
+    n = fs.FS_STATIC_MAX_N
+    w = workloads.make(4, n=n, want_cost=False)
+    stream = torch.cuda.Stream()
+    K = torch.from_numpy(w.K).cuda()
+    rng = np.random.default_rng(3)
+    u_host = (rng.random(n) + 0.5).astype(np.float32)
+    u = torch.from_numpy(u_host).cuda()
+    b = torch.from_numpy(w.b).cuda()
+    v = torch.full_like(u, float("nan"))
+    torch.cuda.synchronize()
+    fs.fs_col_pass_static(K, n, n, u, b, v, stream)
+    stream.synchronize()
+    v_or, _ = oracle.col_pass(w.K, oracle.KIND_KERNEL, w.eps, w.b, u_host)
+    got = v.cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(got)) and np.max(np.abs(got - v_or) / v_or) < 2e-6
 
 
 def test_static_column_pass_rejects_oversize_and_bad_arguments():
