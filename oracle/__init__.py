@@ -74,6 +74,9 @@ def _load():
                 "or_marginals_scaling": [_i64, _f32p, _i64, _int, _dbl, _f64p, _f64p, _f64p, _f64p],
                 "or_marginals_log": [_i64, _f32p, _i64, _dbl, _f64p, _f64p, _f64p, _f64p],
                 "or_marginal_errors": [_i64, _f64p, _f64p, _f32p, _f32p, _f64p],
+                "or_cost_from_points": [_i64, _i64, _f32p, _f32p, _dbl, _f64p],
+                "or_sinkhorn_points": [_i64, _i64, _f32p, _f32p, _dbl, _dbl, _f32p, _f32p, _i64, _f64p, _f64p],
+                "or_marginals_points": [_i64, _i64, _f32p, _f32p, _dbl, _dbl, _f64p, _f64p, _f64p, _f64p],
                 "or_plan": [_i64, _f32p, _i64, _int, _dbl, _int, _f64p, _f64p, _f64p],
                 "or_objectives": [_i64, _f32p, _i64, _int, _dbl, _int, _f64p, _f64p, _f32p, _i64, _f64p],
             }
@@ -265,6 +268,45 @@ def sinkhorn_log(C, eps, a, b, iters, f0=None, g0=None):
     g = _f64(np.zeros(n) if g0 is None else g0, n)
     _load().or_sinkhorn_log(n, _p32(C), ld, float(eps), _p32(a), _p32(b), int(iters), _p64(f), _p64(g))
     return f, g
+
+
+# ----------------------------------------------------------------------------- implicit kernel from points
+
+def _points(X, Y):
+    X = np.ascontiguousarray(X, dtype=np.float32)
+    Y = np.ascontiguousarray(Y, dtype=np.float32)
+    if X.ndim != 2 or X.shape != Y.shape:
+        raise ValueError("X and Y must be float32 arrays of the same shape [n][d]")
+    return X, Y, X.shape[0], X.shape[1]
+
+
+def cost_from_points(X, Y, scale=1.0):
+    """C_il = scale * |x_i - y_l|^2 as an n x n float64 array (X, Y: [n][d] float32)."""
+    X, Y, n, d = _points(X, Y)
+    C = np.empty((n, n))
+    _load().or_cost_from_points(n, d, _p32(X), _p32(Y), float(scale), _p64(C))
+    return C
+
+
+def sinkhorn_points(X, Y, scale, eps, a, b, iters, u0=None, v0=None):
+    """Sinkhorn-Knopp with K_il = exp(-scale |x_i - y_l|^2 / eps) evaluated on the fly; `iters` full
+    iterations from u0, v0 (default ones)."""
+    X, Y, n, d = _points(X, Y)
+    a, b = _f32(a, n), _f32(b, n)
+    u = _f64(np.ones(n) if u0 is None else u0, n)
+    v = _f64(np.ones(n) if v0 is None else v0, n)
+    _load().or_sinkhorn_points(n, d, _p32(X), _p32(Y), float(scale), float(eps), _p32(a), _p32(b), int(iters),
+                               _p64(u), _p64(v))
+    return u, v
+
+
+def marginal_errors_points(X, Y, scale, eps, u, v, a, b):
+    """dict(row_l1, row_l2, col_l1, col_l2) of the implicit-kernel plan's marginals against a and b."""
+    X, Y, n, d = _points(X, Y)
+    u, v = _f64(u, n), _f64(v, n)
+    row, col = np.empty(n), np.empty(n)
+    _load().or_marginals_points(n, d, _p32(X), _p32(Y), float(scale), float(eps), _p64(u), _p64(v), _p64(row), _p64(col))
+    return marginal_error_norms(row, col, a, b)
 
 
 # ----------------------------------------------------------------------------- errors, objectives

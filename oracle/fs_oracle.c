@@ -29,6 +29,8 @@
  *     l_u = log u; the formula is the standard one:
  *        f_i = eps log a_i - eps LSE_l((g_l - C_il)/eps),
  *        g_l = eps log b_l - eps LSE_i((f_i - C_il)/eps))
+ *   - the same iteration with K applied implicitly from two point clouds,
+ *     K_il = exp(-scale |x_i - y_l|^2 / eps)        (Section 3.1, Section 4.1 remark, Section 5.4)
  *   - marginal error err = || P 1 - a ||                 (Section 5.3, DP appendix)
  *   - transport cost <P,C>, dual and primal objective values      (Eq. 1)
  *
@@ -36,7 +38,9 @@
  * scaling/log equivalence, protocol == centralized bit for bit (Prop. 1),
  * fixed-point marginals and strong duality, half-step invariants, the 2x2
  * quadratic closed form, an independent Newton solve of the dual for n <= 8,
- * brute force over all block compositions.  The paper's printed 3x3 toy plan
+ * brute force over all block compositions; for the implicit kernel: hand-placed
+ * points with integer squared distances, symmetry and zero diagonal for one cloud,
+ * translation invariance, agreement with the stored-cost iteration.  The paper's printed 3x3 toy plan
  * is internally inconsistent (its row sums are not the stated a) and pins
  * nothing; it is used only for "column sums equal b".
  */
@@ -282,6 +286,65 @@ void or_sinkhorn_log(int64_t n, const float *C, int64_t ld, double eps, const fl
     for (int64_t t = 0; t < iters; ++t) {
         or_log_row_pass(n, C, ld, eps, a, g, f);
         or_log_col_pass(n, C, ld, eps, b, f, g);
+    }
+}
+
+/* ---------------------------------------------------------------- implicit (on-the-fly) kernel from points */
+
+/* Embedding cost between point i of cloud X and point l of cloud Y (both n x d, fp32, row-major):
+ * C_il = scale * sum_k (x_ik - y_lk)^2 -- the squared Euclidean cost of the embedding experiment (Section 5.4),
+ * optionally rescaled (the workloads divide by the largest entry).  Plain differences, k ascending. */
+static inline double sqdist_cost(const float *X, const float *Y, int64_t d, double scale, int64_t i, int64_t l) {
+    double s = 0.0;
+    for (int64_t k = 0; k < d; ++k) {
+        double t = (double)X[i * d + k] - (double)Y[l * d + k];
+        s += t * t;
+    }
+    return scale * s;
+}
+
+/* C (n x n doubles, row-major) from the two clouds. */
+void or_cost_from_points(int64_t n, int64_t d, const float *X, const float *Y, double scale, double *C) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i)
+        for (int64_t l = 0; l < n; ++l) C[i * n + l] = sqdist_cost(X, Y, d, scale, i, l);
+}
+
+/* Sinkhorn-Knopp with the kernel applied implicitly: K_il = exp(-C_il/eps) is evaluated from the points every
+ * time it is needed and never stored (Section 3.1 "do not assume it is explicitly materialized"; Section 4.1,
+ * remark on on-the-fly kernels).  Same iteration, order and start convention as or_sinkhorn_scaling. */
+void or_sinkhorn_points(int64_t n, int64_t d, const float *X, const float *Y, double scale, double eps,
+                        const float *a, const float *b, int64_t iters, double *u, double *v) {
+    for (int64_t t = 0; t < iters; ++t) {
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < n; ++i) {
+            double q = 0.0;
+            for (int64_t l = 0; l < n; ++l) q += exp(-sqdist_cost(X, Y, d, scale, i, l) / eps) * v[l];
+            u[i] = (double)a[i] / q;
+        }
+#pragma omp parallel for schedule(static)
+        for (int64_t l = 0; l < n; ++l) {
+            double r = 0.0;
+            for (int64_t i = 0; i < n; ++i) r += exp(-sqdist_cost(X, Y, d, scale, i, l) / eps) * u[i];
+            v[l] = (double)b[l] / r;
+        }
+    }
+}
+
+/* Marginals of P = diag(u) K diag(v) with the implicit kernel: row_i = u_i (K v)_i, col_l = v_l (K^T u)_l. */
+void or_marginals_points(int64_t n, int64_t d, const float *X, const float *Y, double scale, double eps,
+                         const double *u, const double *v, double *row, double *col) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) {
+        double q = 0.0;
+        for (int64_t l = 0; l < n; ++l) q += exp(-sqdist_cost(X, Y, d, scale, i, l) / eps) * v[l];
+        row[i] = u[i] * q;
+    }
+#pragma omp parallel for schedule(static)
+    for (int64_t l = 0; l < n; ++l) {
+        double r = 0.0;
+        for (int64_t i = 0; i < n; ++i) r += exp(-sqdist_cost(X, Y, d, scale, i, l) / eps) * u[i];
+        col[l] = v[l] * r;
     }
 }
 

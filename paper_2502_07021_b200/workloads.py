@@ -62,6 +62,9 @@ class Workload:
     b: np.ndarray
     K: np.ndarray | None = None  # float32 [n][n] Gibbs kernel (scaling-domain configs)
     C: np.ndarray | None = None  # float32 [n][n] cost
+    X: np.ndarray | None = None  # float32 [n][dim] points of the first cloud (only with fp32_points)
+    Y: np.ndarray | None = None  # float32 [n][dim] points of the second cloud (X itself for one cloud)
+    cost_scale: float = 1.0      # C_il = cost_scale * |x_i - y_l|^2 (1 / largest squared distance, or 1)
     meta: dict = field(default_factory=dict)
 
     @property
@@ -129,10 +132,14 @@ def cost_and_kernel(X, Y, eps, normalize, want_cost=True, want_kernel=True, chun
 
 
 def make(cfg: int, n: int | None = None, nbatch: int | None = None, c: int | None = None,
-         offsets=None, want_cost: bool | None = None, want_kernel: bool | None = None, rows=None) -> Workload:
+         offsets=None, want_cost: bool | None = None, want_kernel: bool | None = None, rows=None,
+         fp32_points: bool = False) -> Workload:
     """Build configuration `cfg` (1..5).  `n`, `nbatch`, `c`/`offsets` override the stated sizes
     to get a smaller or differently partitioned copy of the same recipe.  `rows = (lo, hi)` materialises
-    only that row block of the matrices (a, b stay whole): what one shard of a row partition holds."""
+    only that row block of the matrices (a, b stay whole): what one shard of a row partition holds.
+    With `fp32_points` the clouds are rounded to fp32 BEFORE the cost is formed and are returned as X, Y
+    together with cost_scale: the inputs of the implicit-kernel path (the matrices, if asked for, are then
+    those of the rounded points, so that both paths describe the same problem)."""
     s = dict(_SPECS[cfg])
     n = int(s["n"] if n is None else n)
     nb = int(s["nbatch"] if nbatch is None else nbatch)
@@ -145,6 +152,11 @@ def make(cfg: int, n: int | None = None, nbatch: int | None = None, c: int | Non
         off = equal_offsets(n, cc)
     X = _points(s["cloud"], np.random.default_rng(1000 + cfg), n, s["dim"], shifted=False)
     Y = _points(s["cloud"], np.random.default_rng(2000 + cfg), n, s["dim"], shifted=True) if s["two_clouds"] else X
+    if fp32_points:
+        X32 = X.astype(np.float32)
+        Y32 = X32 if Y is X else Y.astype(np.float32)
+        X = X32.astype(np.float64)
+        Y = X if Y32 is X32 else Y32.astype(np.float64)
     log = s["domain"] == DOMAIN_LOG
     if want_cost is None:
         want_cost = True if log else n <= 8192
@@ -166,7 +178,8 @@ def make(cfg: int, n: int | None = None, nbatch: int | None = None, c: int | Non
     name = f"cfg{cfg}_n{n}" + (f"_N{nb}" if nb > 1 else "") + ("_log" if log else "_scaling") + f"_c{cc}"
     return Workload(cfg=cfg, name=name, n=n, c=cc, offsets=off, eps=float(s["eps"]), domain=s["domain"],
                     iters=int(s["iters"]), nbatch=nb, check_every=int(s["check_every"]), a=a, b=b,
-                    K=K32, C=C32, meta=meta)
+                    K=K32, C=C32, meta=meta, X=X32 if fp32_points else None, Y=Y32 if fp32_points else None,
+                    cost_scale=float(meta["cost_scale"]))
 
 
 def additive_cost(n: int, seed: int = 7):

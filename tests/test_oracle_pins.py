@@ -487,6 +487,59 @@ def test_log_domain_marginals_rank1_closed_form_both_sides():
     np.testing.assert_allclose(col, b.astype(np.float64), rtol=1e-13)
 
 
+# ------------------------------------------------------------------ implicit kernel from points
+
+def test_cost_from_points_hand_placed_integer_distances():
+    """3-4-5 and 6-8-10 triangles: every squared distance is an integer fixed by hand; X != Y catches a
+    transposed result, the scale factor is applied once."""
+    X = np.array([[0, 0], [3, 4], [1, 1]], dtype=np.float32)
+    Y = np.array([[0, 0], [6, 8], [1, 2]], dtype=np.float32)
+    ref = np.array([[0, 100, 5], [25, 25, 8], [2, 74, 1]], dtype=np.float64)
+    assert np.array_equal(oracle.cost_from_points(X, Y), ref)
+    assert np.array_equal(oracle.cost_from_points(X, Y, 0.25), ref / 4)
+    assert np.array_equal(oracle.cost_from_points(Y, X), ref.T)
+
+
+def test_cost_from_points_symmetry_translation_and_generator():
+    rng = np.random.default_rng(5)
+    n, d = 40, 7
+    X = (rng.integers(-512, 512, (n, d)) / 256.0).astype(np.float32)          # dyadic grid: shifts stay exact
+    Y = (rng.integers(-512, 512, (n, d)) / 256.0).astype(np.float32)
+    C1 = oracle.cost_from_points(X, X)
+    assert np.array_equal(C1, C1.T) and np.all(np.diag(C1) == 0) and np.all(C1[~np.eye(n, dtype=bool)] > 0)
+    shift = (rng.integers(-64, 64, d) / 16.0).astype(np.float32)
+    assert np.array_equal(oracle.cost_from_points(X + shift, Y + shift), oracle.cost_from_points(X, Y))
+    # the workload generator forms the same cost by the expanded square in fp64 and rounds it to fp32
+    w = workloads.make(2, n=300, fp32_points=True, want_cost=True)
+    C = oracle.cost_from_points(w.X, w.Y, w.cost_scale)
+    assert np.max(np.abs(C - w.C.astype(np.float64))) <= 2.0 ** -24 * C.max() * 1.01
+    assert C.max() == pytest.approx(1.0, rel=1e-12)                            # config 2 divides by the largest entry
+
+
+def test_sinkhorn_points_equals_stored_cost_iteration():
+    """On integer grid points every C_il is an integer, exact in fp32: the implicit iteration must reproduce the
+    stored-cost iteration (pinned above by closed forms and the Newton solve) to rounding, two clouds, and
+    its marginal errors those of the stored-cost state."""
+    rng = np.random.default_rng(9)
+    n, d, eps, scale = 31, 3, 6.0, 0.5
+    X = rng.integers(0, 5, (n, d)).astype(np.float32)
+    Y = rng.integers(0, 5, (n, d)).astype(np.float32)
+    C = oracle.cost_from_points(X, Y, scale)
+    C32 = C.astype(np.float32)
+    assert np.array_equal(C32.astype(np.float64), C)
+    a, b = dirichlet_pair(n, 10)
+    for iters in (1, 7):
+        u, v = oracle.sinkhorn_points(X, Y, scale, eps, a, b, iters)
+        ur, vr = oracle.sinkhorn_scaling(C32, C_, eps, a, b, iters)
+        np.testing.assert_allclose(u, ur, rtol=1e-13)
+        np.testing.assert_allclose(v, vr, rtol=1e-13)
+    e = oracle.marginal_errors_points(X, Y, scale, eps, u, v * 1.01, a, b)
+    er = oracle.marginal_errors(C32, C_, eps, SC, ur, vr * 1.01, a, b)
+    for k in e:
+        assert e[k] == pytest.approx(er[k], rel=1e-11)
+    assert e["row_l1"] > 1e-3
+
+
 # ------------------------------------------------------------------ library-routine special case
 
 def test_lse_against_scipy():
