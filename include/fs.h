@@ -194,6 +194,7 @@ int fs_set_option(fs_solver *s, int option, int64_t value);
  *   "resident"      all iterations in one launch, K in one cluster's shared memory
  *   "persistent"    all iterations in one cooperative launch, K in L2 and shared memory
  *   "batched_tc"    shared-K batch on tensor cores                     "batched_fma"  its fp32 FMA engine
+ *   "implicit"      kernel formed on the fly from point clouds (fs_create_points)
  * (A diagnostic of this implementation; the paper has no counterpart.) */
 const char *fs_iteration_path(const fs_solver *s);
 
@@ -223,6 +224,38 @@ int fs_destroy(fs_solver *s);
 int fs_solve_host(int64_t n, int32_t c, const int64_t *row_offsets, const float *M_host, int64_t ld,
                   int matrix_kind, double eps, const float *a_host, const float *b_host, int32_t nbatch,
                   int domain, int32_t iters, float *u_out, float *v_out, double *row_err_l1_out);
+
+/*
+ * fs_create_points -- a solver whose kernel is applied IMPLICITLY from two point clouds and never stored
+ * (Section 3.1: K is not assumed materialised, a client only needs x -> K_{I,:} x and the transpose action;
+ * Section 4.1, remark on on-the-fly kernels: the matvec time then includes the kernel evaluation; cost of
+ * Section 5.4):
+ *
+ *      K_il = exp(-cost_scale * |x_i - y_l|^2 / eps),     i, l = 0 .. n-1.
+ *
+ *   X_dev, Y_dev  DEVICE [n][d] fp32 row-major point clouds (Y_dev may equal X_dev: one cloud, symmetric cost).
+ *                 Copied into the library's own operand layout; not needed after the call.
+ *   d             coordinates per point, 1 <= d <= 58 (FS_ERR_UNSUPPORTED beyond).
+ *   cost_scale    factor on the squared distance (e.g. 1 / largest squared distance), > 0.
+ *   n, c, row_offsets, eps, a_dev, b_dev, stream   as for fs_create; one problem, scaling domain.
+ *
+ * The handle works with fs_iterate, fs_row_pass, fs_col_pass, fs_marginal_error, fs_scalings, fs_set_scalings,
+ * fs_reset, fs_set_damping, the error trace and fs_block_errors; fs_transport_cost returns FS_ERR_UNSUPPORTED.
+ * Memory is O(n d): nothing of size n^2 exists.  The squared distance is formed as a tensor-core contraction of
+ * the translated, scaled points split into two bf16 terms each; the exponent -c|x - y|^2 log2(e)/eps then carries
+ * an absolute error of at most about 2^-16 * max|z_x| * max|z_y| (z = sqrt(2 cost_scale log2(e) / eps) times the
+ * centred point).  The call computes that bound and returns FS_ERR_UNSUPPORTED when it exceeds 1e-3 (very small
+ * eps on wide clouds): such problems need a stored cost and the log domain.
+ */
+int fs_create_points(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets, const float *X_dev,
+                     const float *Y_dev, int32_t d, double cost_scale, double eps, const float *a_dev, const float *b_dev,
+                     void *stream);
+
+/* fs_solve_host_points -- fs_solve_host for the implicit kernel: HOST point clouds in ([n][d] each), HOST scalings
+ * out; O(n d) bytes cross the bus instead of the n x n matrix.  Synchronous. */
+int fs_solve_host_points(int64_t n, int32_t c, const int64_t *row_offsets, const float *X_host, const float *Y_host,
+                         int32_t d, double cost_scale, double eps, const float *a_host, const float *b_host, int32_t iters,
+                         float *u_out, float *v_out, double *row_err_l1_out);
 
 /*
  * fs_col_pass_static -- v = b ./ (K^T u) for one problem, WITHOUT allocating anything.

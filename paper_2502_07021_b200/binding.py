@@ -49,6 +49,8 @@ _SIGNATURES = {
     "fs_fused_log_fallbacks": (_int, [_vp, ctypes.POINTER(_i64), _vp]),
     "fs_destroy": (_int, [_vp]),
     "fs_solve_host": (_int, [_i64, _i32, _vp, _vp, _i64, _int, _dbl, _vp, _vp, _i32, _int, _i32, _vp, _vp, _vp]),
+    "fs_create_points": (_int, [ctypes.POINTER(_vp), _i64, _i32, _vp, _vp, _vp, _i32, _dbl, _dbl, _vp, _vp, _vp]),
+    "fs_solve_host_points": (_int, [_i64, _i32, _vp, _vp, _vp, _i32, _dbl, _dbl, _vp, _vp, _i32, _vp, _vp, _vp]),
     "fs_col_pass_static": (_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp]),
     "fs_shard_create": (_int, [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp, _i64, _int, _dbl, _vp, _vp, _vp]),
     "fs_shard_row_pass": (_int, [_vp, _vp]),
@@ -133,6 +135,16 @@ def fs_create(n, c, row_offsets, M_dev, ld, matrix_kind, eps, a_dev, b_dev, nbat
     out = _vp()
     _check(lib().fs_create(ctypes.byref(out), n, c, offp, _dev(M_dev), ld, matrix_kind, float(eps), _dev(a_dev),
                            _dev(b_dev), nbatch, domain, _stream(stream)), "fs_create")
+    return out
+
+
+def fs_create_points(n, c, row_offsets, X_dev, Y_dev, d, cost_scale, eps, a_dev, b_dev, stream=None):
+    off, offp = _host(row_offsets, np.int64)
+    if off.shape != (c + 1,):
+        raise FsError(FS_ERR_BAD_OFFSETS, "fs_create_points")
+    out = _vp()
+    _check(lib().fs_create_points(ctypes.byref(out), n, c, offp, _dev(X_dev), _dev(Y_dev), d, float(cost_scale), float(eps),
+                                  _dev(a_dev), _dev(b_dev), _stream(stream)), "fs_create_points")
     return out
 
 
@@ -276,6 +288,30 @@ def fs_selftest_bounded_wait(poll_limit, arrive, stream=None):
     _check(lib().fs_selftest_bounded_wait(poll_limit, 1 if arrive else 0, ctypes.byref(out), _stream(stream)),
            "fs_selftest_bounded_wait")
     return out.value == 1
+
+
+def _host_ptr(x):
+    if x is None:
+        return None
+    if hasattr(x, "data_ptr"):
+        if x.is_cuda:
+            raise ValueError("host buffers expected")
+        return x.data_ptr()
+    if x.dtype != np.float32 or not x.flags["C_CONTIGUOUS"]:
+        raise ValueError("host buffers must be contiguous float32")
+    return x.ctypes.data
+
+
+def fs_solve_host_points(n, c, row_offsets, X_host, Y_host, d, cost_scale, eps, a_host, b_host, iters, u_out, v_out,
+                         want_error=True):
+    """Host point clouds in, host scalings out (numpy float32 or pinned torch CPU tensors); returns the 1-norm
+    row marginal error (array of one) or None."""
+    off, offp = _host(row_offsets, np.int64)
+    err = np.zeros(1) if want_error else None
+    _check(lib().fs_solve_host_points(n, c, offp, _host_ptr(X_host), _host_ptr(Y_host), d, float(cost_scale), float(eps),
+                                      _host_ptr(a_host), _host_ptr(b_host), iters, _host_ptr(u_out), _host_ptr(v_out),
+                                      err.ctypes.data_as(_vp) if want_error else None), "fs_solve_host_points")
+    return err
 
 
 def fs_solve_host(n, c, row_offsets, M_host, ld, matrix_kind, eps, a_host, b_host, nbatch, domain, iters,

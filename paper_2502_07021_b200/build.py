@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfs_b200.so")
 OBJ_DIR = os.path.join(os.path.dirname(HERE), "_build")
-SOURCES = ["fs_api.cu", "passes.cu", "batched.cu", "batched_tc.cu", "fused.cu", "fused_log.cu", "resident.cu", "persistent.cu", "shard.cu", "setup.cu", "col_pass_static.cu"]
+SOURCES = ["fs_api.cu", "passes.cu", "batched.cu", "batched_tc.cu", "fused.cu", "fused_log.cu", "resident.cu", "persistent.cu", "shard.cu", "setup.cu", "col_pass_static.cu", "implicit.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 

@@ -101,6 +101,7 @@ void destroy_solver(fs_solver *s) {
     free_dev(s->status);
     free_dev(s->cost_scratch);
     if (s->tc) fsk_tc_destroy(s->tc);
+    if (s->implicit) fsk_implicit_destroy(s->implicit);
     delete s;
 }
 
@@ -122,8 +123,20 @@ int upload_tiles(fs_solver *s) {
 
 bool use_tc(const fs_solver *s) { return s->tc != nullptr && s->batch_engine != 1; }
 
+// Half-step with the kernel formed on the fly from the point clouds: partial sums per (row, column split), then
+// the ordinary stage-2 kernel (fixed-order sum, residual, divide).
+void enqueue_implicit(fs_solver *s, int transposed, int update, cudaStream_t st, int64_t &launches) {
+    fsk_implicit_pass(s->implicit, transposed, transposed ? s->x : s->y, s->status, st);
+    fsk_col_finish(s->n, s->vec_pad, fsk_implicit_nsplit(s->implicit), fsk_implicit_partials(s->implicit),
+                   transposed ? s->b : s->a, transposed ? s->y : s->x, transposed ? s->coldiff : s->rowdiff, update, s->eta,
+                   s->status, st);
+    launches += 2;
+}
+
 void enqueue_row(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
-    if (s->nbatch > 1 && use_tc(s)) {
+    if (s->implicit) {
+        enqueue_implicit(s, 0, update, st, launches);
+    } else if (s->nbatch > 1 && use_tc(s)) {
         fsk_tc_pass(s->tc, 0, s->a, s->x, s->rowdiff, update, s->eta, s->status, st);
         launches += 1;
     } else if (s->nbatch > 1) {
@@ -141,7 +154,9 @@ void enqueue_row(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
 }
 
 void enqueue_col(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
-    if (s->nbatch > 1 && use_tc(s)) {
+    if (s->implicit) {
+        enqueue_implicit(s, 1, update, st, launches);
+    } else if (s->nbatch > 1 && use_tc(s)) {
         fsk_tc_pass(s->tc, 1, s->b, s->y, s->coldiff, update, s->eta, s->status, st);
         launches += 1;
     } else if (s->nbatch > 1) {
@@ -171,10 +186,11 @@ bool use_fused(const fs_solver *s) {
 
 // Which kernels fs_iterate runs for this handle as it is configured now.
 enum IterPath { PATH_TWO_PASS, PATH_TWO_PASS_LOG, PATH_FUSED, PATH_FUSED_LOG, PATH_RESIDENT, PATH_PERSISTENT, PATH_BATCHED_TC,
-                PATH_BATCHED_FMA };
+                PATH_BATCHED_FMA, PATH_IMPLICIT };
 
 IterPath iteration_path(const fs_solver *s) {
     const bool traced = s->check_every != 0;
+    if (s->implicit) return PATH_IMPLICIT;
     if (s->nbatch > 1) return use_tc(s) ? PATH_BATCHED_TC : PATH_BATCHED_FMA;
     if (s->resident.enabled && s->resident_mode != 0 && !traced) return PATH_RESIDENT;
     if (s->persistent.enabled && !traced &&
@@ -279,6 +295,26 @@ int set_initial_state(fs_solver *s, cudaStream_t st) {
     return FS_OK;
 }
 
+// Assumption A2 checked on the device: strictly positive, finite, equal mass per problem.
+int validate_marginals(const float *a_dev, const float *b_dev, int64_t n, int32_t nbatch, cudaStream_t st) {
+    double *scan = nullptr;
+    FS_CU(cudaMalloc(&scan, sizeof(double) * 4 * (size_t)nbatch));
+    fsk_min_sum(a_dev, n, nbatch, scan, st);
+    fsk_min_sum(b_dev, n, nbatch, scan + 2 * (size_t)nbatch, st);
+    std::vector<double> h(4 * (size_t)nbatch);
+    cudaError_t e = cudaMemcpyAsync(h.data(), scan, sizeof(double) * h.size(), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(scan);
+    if (e != cudaSuccess) return cuda_fail(e, "marginal validation");
+    for (int p = 0; p < nbatch; ++p) {
+        const double amin = h[2 * p], asum = h[2 * p + 1];
+        const double bmin = h[2 * nbatch + 2 * p], bsum = h[2 * nbatch + 2 * p + 1];
+        if (!(amin > 0.0) || !(bmin > 0.0) || !isfinite(asum) || !isfinite(bsum)) return FS_ERR_NONPOSITIVE_MARGINAL;
+        if (fabs(asum - bsum) > 1e-4 * asum) return FS_ERR_MASS_MISMATCH;
+    }
+    return FS_OK;
+}
+
 } // namespace
 
 extern "C" {
@@ -326,21 +362,8 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
 
     // validate the marginals on the device before anything is built (assumption A2)
     {
-        double *scan = nullptr;
-        FS_CU(cudaMalloc(&scan, sizeof(double) * 4 * (size_t)nbatch));
-        fsk_min_sum(a_dev, n, nbatch, scan, st);
-        fsk_min_sum(b_dev, n, nbatch, scan + 2 * (size_t)nbatch, st);
-        std::vector<double> h(4 * (size_t)nbatch);
-        cudaError_t e = cudaMemcpyAsync(h.data(), scan, sizeof(double) * h.size(), cudaMemcpyDeviceToHost, st);
-        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-        cudaFree(scan);
-        if (e != cudaSuccess) return cuda_fail(e, "marginal validation");
-        for (int p = 0; p < nbatch; ++p) {
-            const double amin = h[2 * p], asum = h[2 * p + 1];
-            const double bmin = h[2 * nbatch + 2 * p], bsum = h[2 * nbatch + 2 * p + 1];
-            if (!(amin > 0.0) || !(bmin > 0.0) || !isfinite(asum) || !isfinite(bsum)) return FS_ERR_NONPOSITIVE_MARGINAL;
-            if (fabs(asum - bsum) > 1e-4 * asum) return FS_ERR_MASS_MISMATCH;
-        }
+        const int vrc = validate_marginals(a_dev, b_dev, n, nbatch, st);
+        if (vrc != FS_OK) return vrc;
     }
 
     fs_solver *s = new fs_solver();
@@ -421,6 +444,71 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
     // batched problems: tensor-core engine when the batch is wide enough to fill its 128-problem tiles
     if (nbatch >= kTcMinBatch && n >= kTcMinN) s->tc = fsk_tc_create(s->mat, s->mat_ld, n, nbatch, st);
     rc = set_initial_state(s, st);
+    if (rc != FS_OK) return rc;
+    FS_CU(cudaStreamSynchronize(st));
+    FS_CU(cudaGetLastError());
+    guard.s = nullptr;
+    *out = s;
+    return FS_OK;
+}
+
+int fs_create_points(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets, const float *X_dev,
+                     const float *Y_dev, int32_t d, double cost_scale, double eps, const float *a_dev, const float *b_dev,
+                     void *stream) {
+    if (!out) return FS_ERR_NULL;
+    *out = nullptr;
+    if (!row_offsets || !X_dev || !Y_dev || !a_dev || !b_dev) return FS_ERR_NULL;
+    if (n < 1 || n > (int64_t(1) << 24) || d < 1) return FS_ERR_BAD_N;
+    if (c < 1 || c > n) return FS_ERR_BAD_OFFSETS;
+    if (row_offsets[0] != 0 || row_offsets[c] != n) return FS_ERR_BAD_OFFSETS;
+    for (int32_t j = 0; j < c; ++j)
+        if (row_offsets[j + 1] <= row_offsets[j]) return FS_ERR_BAD_OFFSETS;
+    if (!(eps > 0.0) || !isfinite(eps) || !(cost_scale > 0.0) || !isfinite(cost_scale)) return FS_ERR_BAD_EPS;
+    if (d > fsk_implicit_max_dim()) return FS_ERR_UNSUPPORTED;
+
+    cudaStream_t st = (cudaStream_t)stream;
+    {
+        const int vrc = validate_marginals(a_dev, b_dev, n, 1, st);
+        if (vrc != FS_OK) return vrc;
+    }
+    fs_solver *s = new fs_solver();
+    struct Guard {
+        fs_solver *s;
+        ~Guard() { destroy_solver(s); }
+    } guard{s};
+    s->n = n, s->ld = 0, s->c = c, s->nbatch = 1, s->domain = FS_DOMAIN_SCALING, s->matrix_kind = FS_MATRIX_KERNEL, s->eps = eps;
+    s->offsets.assign(row_offsets, row_offsets + c + 1);
+    s->n_pad = (n + 3) & ~int64_t(3);
+    s->vec_pad = fsk_implicit_padded_n(n);
+    s->block_err_host.assign(2 * (size_t)c, 0.0);
+    s->plan = fsk_choose_plan(n, false, FS_DOMAIN_SCALING);
+
+    int irc = FS_OK;
+    s->implicit = fsk_implicit_create(X_dev, Y_dev, n, d, cost_scale, eps, st, &irc, nullptr);
+    if (!s->implicit) return irc == FS_ERR_CUDA ? cuda_fail(cudaGetLastError(), "implicit operator set-up") : irc;
+
+    const size_t vb = sizeof(float) * (size_t)s->vec_pad;
+    FS_CU(cudaStreamCreateWithFlags(&s->capture_stream, cudaStreamNonBlocking));
+    FS_CU(cudaMalloc(&s->a, sizeof(float) * n));
+    FS_CU(cudaMalloc(&s->b, sizeof(float) * n));
+    FS_CU(cudaMalloc(&s->x, vb)); // zero beyond n: the pass reads whole 128-column tiles of its input vector
+    FS_CU(cudaMalloc(&s->y, vb));
+    FS_CU(cudaMalloc(&s->rowdiff, sizeof(float) * n));
+    FS_CU(cudaMalloc(&s->coldiff, sizeof(float) * n));
+    FS_CU(cudaMalloc(&s->offsets_dev, sizeof(int64_t) * (c + 1)));
+    FS_CU(cudaMalloc(&s->block_err, sizeof(double) * 2 * c));
+    FS_CU(cudaMalloc(&s->err_out, sizeof(double) * 4));
+    FS_CU(cudaMalloc(&s->status, sizeof(FsDeviceStatus)));
+    s->trace_cap = kTraceCap;
+    FS_CU(cudaMalloc(&s->trace, sizeof(double) * 2 * s->trace_cap));
+    FS_CU(cudaMemsetAsync(s->x, 0, vb, st));
+    FS_CU(cudaMemsetAsync(s->y, 0, vb, st));
+    FS_CU(cudaMemcpyAsync(s->a, a_dev, sizeof(float) * n, cudaMemcpyDeviceToDevice, st));
+    FS_CU(cudaMemcpyAsync(s->b, b_dev, sizeof(float) * n, cudaMemcpyDeviceToDevice, st));
+    FS_CU(cudaMemcpyAsync(s->offsets_dev, s->offsets.data(), sizeof(int64_t) * (c + 1), cudaMemcpyHostToDevice, st));
+    FS_CU(cudaMemsetAsync(s->rowdiff, 0, sizeof(float) * n, st));
+    FS_CU(cudaMemsetAsync(s->coldiff, 0, sizeof(float) * n, st));
+    const int rc = set_initial_state(s, st);
     if (rc != FS_OK) return rc;
     FS_CU(cudaStreamSynchronize(st));
     FS_CU(cudaGetLastError());
@@ -667,6 +755,7 @@ int fs_reset(fs_solver *s, void *stream) {
 
 int fs_transport_cost(fs_solver *s, const float *C_dev, int64_t ldc, double *cost_out, void *stream) {
     if (!s || !cost_out) return FS_ERR_NULL;
+    if (s->implicit) return FS_ERR_UNSUPPORTED; // no stored kernel to form P from
     cudaStream_t st = (cudaStream_t)stream;
     const float *C = C_dev;
     int64_t ldC = ldc;
@@ -720,6 +809,7 @@ const char *fs_iteration_path(const fs_solver *s) {
     case PATH_RESIDENT: return "resident";
     case PATH_PERSISTENT: return "persistent";
     case PATH_BATCHED_TC: return "batched_tc";
+    case PATH_IMPLICIT: return "implicit";
     default: return "batched_fma";
     }
 }
@@ -772,6 +862,47 @@ int fs_solve_host(int64_t n, int32_t c, const int64_t *row_offsets, const float 
     FS_CU2(cudaMemcpyAsync(a, a_host, vb, cudaMemcpyHostToDevice, st));
     FS_CU2(cudaMemcpyAsync(b, b_host, vb, cudaMemcpyHostToDevice, st));
     rc = fs_create(&s, n, c, row_offsets, M, n, matrix_kind, eps, a, b, nbatch, domain, st);
+    if (rc == FS_OK) rc = fs_iterate(s, iters, st);
+    if (rc == FS_OK && row_err_l1_out) rc = fs_marginal_error(s, 1, row_err_l1_out, nullptr, st);
+    int rc2 = FS_OK;
+    if (rc == FS_OK || rc == FS_ERR_NONFINITE) rc2 = fs_scalings(s, u, v, st);
+    if (rc == FS_OK) rc = rc2;
+    if (rc == FS_OK || rc == FS_ERR_NONFINITE) {
+        if (u_out) FS_CU2(cudaMemcpyAsync(u_out, u, vb, cudaMemcpyDeviceToHost, st));
+        if (v_out) FS_CU2(cudaMemcpyAsync(v_out, v, vb, cudaMemcpyDeviceToHost, st));
+        FS_CU2(cudaStreamSynchronize(st));
+    }
+    cleanup();
+    return rc;
+}
+
+int fs_solve_host_points(int64_t n, int32_t c, const int64_t *row_offsets, const float *X_host, const float *Y_host,
+                         int32_t d, double cost_scale, double eps, const float *a_host, const float *b_host, int32_t iters,
+                         float *u_out, float *v_out, double *row_err_l1_out) {
+    if (!row_offsets || !X_host || !Y_host || !a_host || !b_host) return FS_ERR_NULL;
+    if (n < 1 || d < 1 || iters < 0) return FS_ERR_BAD_N;
+    cudaStream_t st = nullptr;
+    float *X = nullptr, *Y = nullptr, *a = nullptr, *b = nullptr, *u = nullptr, *v = nullptr;
+    fs_solver *s = nullptr;
+    const size_t vb = sizeof(float) * (size_t)n, pb = vb * (size_t)d;
+    int rc = FS_OK;
+    auto cleanup = [&]() {
+        if (s) fs_destroy(s);
+        free_dev(X), free_dev(Y), free_dev(a), free_dev(b), free_dev(u), free_dev(v);
+        if (st) cudaStreamDestroy(st);
+    };
+    FS_CU2(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
+    FS_CU2(cudaMalloc(&X, pb));
+    FS_CU2(cudaMalloc(&Y, pb));
+    FS_CU2(cudaMalloc(&a, vb));
+    FS_CU2(cudaMalloc(&b, vb));
+    FS_CU2(cudaMalloc(&u, vb));
+    FS_CU2(cudaMalloc(&v, vb));
+    FS_CU2(cudaMemcpyAsync(X, X_host, pb, cudaMemcpyHostToDevice, st));
+    FS_CU2(cudaMemcpyAsync(Y, Y_host, pb, cudaMemcpyHostToDevice, st));
+    FS_CU2(cudaMemcpyAsync(a, a_host, vb, cudaMemcpyHostToDevice, st));
+    FS_CU2(cudaMemcpyAsync(b, b_host, vb, cudaMemcpyHostToDevice, st));
+    rc = fs_create_points(&s, n, c, row_offsets, X, Y, d, cost_scale, eps, a, b, st);
     if (rc == FS_OK) rc = fs_iterate(s, iters, st);
     if (rc == FS_OK && row_err_l1_out) rc = fs_marginal_error(s, 1, row_err_l1_out, nullptr, st);
     int rc2 = FS_OK;

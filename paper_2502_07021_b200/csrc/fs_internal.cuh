@@ -6,6 +6,7 @@
 //   resident.cu        K-resident persistent kernel for small n
 //   persistent.cu      grid-persistent single-read iterations for mid-size n (cooperative launch)
 //   batched_tc.cu      shared-K batched passes on tcgen05 tensor cores;  batched.cu  fp32 FMA engine
+//   implicit.cu        passes with the kernel formed on the fly from point clouds (tcgen05 + ex2); tcgen05_ptx.cuh
 //   shard.cu           row-partitioned shards for several GPUs (fs_shard_*)
 //   col_pass_static.cu column half-step without any allocation
 //   setup.cu           one-off and O(n) helpers;  cluster_ptx.cuh  PTX wrappers of the cluster kernels
@@ -125,6 +126,9 @@ struct fs_solver {
 
     // batched tensor-core path
     void *tc = nullptr;
+    // implicit kernel from point clouds (fs_create_points): no matrix at all; x, y are padded with zeros to vec_pad
+    void *implicit = nullptr;
+    int64_t vec_pad = 0;
 
     cudaStream_t capture_stream = nullptr;
     struct GraphEntry {
@@ -210,6 +214,17 @@ void fsk_tc_destroy(void *tc);
 void fsk_tc_refresh(void *tc, const float *u, const float *v, cudaStream_t st);
 void fsk_tc_pass(void *tc, int transposed, const float *marg, float *out, float *diff, int update, float eta,
                  FsDeviceStatus *status, cudaStream_t st);
+
+// ---- implicit.cu -------------------------------------------------------------------------
+// Kernel applied on the fly from two clouds X, Y ([n][d] fp32): K_il = exp(-cost_scale |x_i - y_l|^2 / eps).
+void *fsk_implicit_create(const float *X, const float *Y, int64_t n, int d, double cost_scale, double eps, cudaStream_t st,
+                          int *err, float *bound_out);
+void fsk_implicit_destroy(void *h);
+int64_t fsk_implicit_padded_n(int64_t n); // length of the zero-padded input vectors the pass reads
+int fsk_implicit_max_dim();
+int fsk_implicit_nsplit(const void *h);
+float *fsk_implicit_partials(void *h);    // [nsplit][padded n] partial sums written by a pass
+cudaError_t fsk_implicit_pass(void *h, int transposed, const float *in, FsDeviceStatus *status, cudaStream_t st);
 
 // ---- setup.cu ----------------------------------------------------------------------------
 // C and K are nrows x n.

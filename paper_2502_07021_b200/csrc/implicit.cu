@@ -1,0 +1,430 @@
+// Implicit (on-the-fly) kernel operator from two point clouds (Section 3.1: K need not be materialised, a client
+// only has to apply x -> K_{I,:} x and its transpose action; Section 4.1, remark on on-the-fly kernels: t_mv then
+// includes the kernel evaluation; Section 5.4: C_il = |x_i - y_l|^2 on embeddings).
+//
+//      K_il = exp(-s |x_i - y_l|^2 / eps) = 2^(t_il),   t_il = -(1/2) |z_i - w_l|^2,
+//      z = sqrt(2 c) (x - mu),  w = sqrt(2 c) (y - mu),  c = (s / eps) log2(e),
+//
+// with mu a common translation (the mean of the two clouds: the cost does not change, the magnitudes that the
+// rounding errors scale with do).  t_il = z_i . w_l - |z_i|^2/2 - |w_l|^2/2 is ONE dense contraction when the two
+// norms ride along as extra columns of the operands: row operand [z, h, 1], column operand [w, 1, g] with
+// h = -|z|^2/2, g = -|w|^2/2.  The contraction runs on the tensor cores (tcgen05.mma, bf16 operands, fp32
+// accumulation in tensor memory): z and w are split into two bf16 terms (hi + lo, 16 significand bits) and the
+// products hi.hi + hi.lo + lo.hi are accumulated; h and g are split into THREE bf16 terms that each meet an exact
+// 1, so the norms enter with fp32 accuracy.  The epilogue reads a 128 x 128 tile of exponents from tensor memory,
+// applies one ex2 per element and accumulates K_il * in_l per row: nothing of size n^2 ever exists in memory.
+//
+// One kernel serves both half-steps of Algorithm 1: the row pass takes X as row operand, Y as column operand and
+// v as input; the column pass takes Y as row operand, X as column operand and u as input (K^T tiles are formed
+// directly, no transposition).  Work item = (128-row tile, range of column tiles); items are dealt round-robin to
+// persistent CTAs; each item writes one partial sum per row, and the ordinary stage-2 kernel adds the partials of a
+// row in a fixed order and applies the divide: deterministic, no atomics.
+//
+// CTA: warp 0 issues TMA loads (row operand tile and the input-vector slice once per item, column operand tiles
+// through a 3-stage ring), warp 1 issues the MMAs into two 128-column accumulators in turn, warps 2..9 are the
+// epilogue (TMEM lane quarter = warp % 4, column half = (warp - 2) / 4).  The bound is the special-function unit:
+// one ex2 per matrix element per pass.  Every wait is bounded; on expiry the kernel raises the status flag, skips
+// the remaining work and still passes every barrier before it frees its tensor memory and exits.
+//
+// Accuracy.  The dot product carries an absolute error of about 2^-16 sum_k |z_ik w_lk| (dropped lo.lo term and the
+// representation error of the split), which is the absolute error of the exponent.  Set-up computes the bound
+// 2^-16 max|z| max|w| and refuses problems where it exceeds 1e-3 (small eps on wide clouds: use a stored cost and
+// the log domain there).
+#include "fs_internal.cuh"
+#include "tcgen05_ptx.cuh"
+
+namespace {
+
+using namespace fstc;
+
+constexpr int BM = 128, BN = 128, BK = 64;
+constexpr int TILE_BYTES = BM * BK * 2;      // one bf16 operand tile (hi or lo): 128 rows of 128 bytes
+constexpr int PAIR_BYTES = 2 * TILE_BYTES;   // hi + lo
+constexpr int B_STAGES = 3;
+constexpr int MAX_T = 32;                    // column tiles per work item (input slice of at most 16 KB)
+constexpr int VSLOT_BYTES = MAX_T * BN * 4;
+constexpr int kImpThreads = 320;             // TMA warp, MMA warp, eight epilogue warps
+constexpr int TMEM_COLS = 256;               // two 128-column fp32 accumulators
+constexpr int kMaxDim = BK - 6;              // coordinates + 3 norm terms + 3 ones fit one 64-column k-block
+// shared memory: A slots, B ring, input slots, combine buffers, barriers, TMEM slot
+constexpr int OFF_A = 0;
+constexpr int OFF_B = OFF_A + 2 * PAIR_BYTES;
+constexpr int OFF_V = OFF_B + B_STAGES * PAIR_BYTES;
+constexpr int OFF_COMB = OFF_V + 2 * VSLOT_BYTES;
+constexpr int OFF_BARS = OFF_COMB + 2 * BM * 4;
+constexpr int NUM_BARS = 6 + 2 * B_STAGES + 4; // item_full[2], item_free_mma[2], item_free_epi[2], b_full, b_empty, acc_full[2], acc_empty[2]
+constexpr int SMEM_BYTES = OFF_BARS + 8 * NUM_BARS + 16 + 1024;
+
+struct ImplicitState {
+    int64_t n = 0, n_pad = 0;
+    int d = 0, kd = 0;            // coordinates per point; 16-wide k-steps of the contraction
+    int tiles = 0;                // 128-point tiles per cloud
+    int T = 0, nsplit = 0;        // column tiles per item, items per row tile
+    int grid = 0;
+    float bound = 0.f;            // bound on the absolute error of the exponent
+    __nv_bfloat16 *buf[8] = {};   // X row-side hi, lo; X column-side hi, lo; Y row-side hi, lo; Y column-side hi, lo
+    CUtensorMap map[8];
+    float *partials = nullptr;    // [nsplit][n_pad]
+};
+
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
+    hi = __float2bfloat16_rn(x);
+    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+// mu_k = mean over both clouds of coordinate k, in double, fixed order (one block per coordinate).
+__global__ void __launch_bounds__(256)
+cloud_mean_kernel(const float *__restrict__ X, const float *__restrict__ Y, int n, int d, double *__restrict__ mu) {
+    __shared__ double red[256];
+    const int k = blockIdx.x;
+    double s = 0.0;
+    for (int i = threadIdx.x; i < n; i += 256) s += (double)X[(int64_t)i * d + k] + (double)Y[(int64_t)i * d + k];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int off = 128; off > 0; off >>= 1) {
+        if (threadIdx.x < off) red[threadIdx.x] += red[threadIdx.x + off];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) mu[k] = red[0] / (2.0 * n);
+}
+
+// One thread per point: z = sqrt(2c) (p - mu) rounded to fp32 and split into bf16 hi + lo; h = -|z|^2/2 (from the
+// rounded z, in double) split into three bf16 terms.  Row-side layout: [z | h1 h2 h3 | 1 1 1], column-side layout:
+// [z | 1 1 1 | h1 h2 h3]; rows of 64 bf16, the rest zero (the buffers are cleared before).  maxsq receives the
+// largest |z|^2 as the bit pattern of a non-negative float.
+__global__ void __launch_bounds__(256)
+prepare_points_kernel(const float *__restrict__ P, int n, int d, const double *__restrict__ mu, double sqrt2c,
+                      __nv_bfloat16 *__restrict__ row_hi, __nv_bfloat16 *__restrict__ row_lo,
+                      __nv_bfloat16 *__restrict__ col_hi, __nv_bfloat16 *__restrict__ col_lo, unsigned int *maxsq) {
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= n) return;
+    double sq = 0.0;
+    const int64_t o = (int64_t)i * BK;
+    for (int k = 0; k < d; ++k) {
+        const float z = (float)(sqrt2c * ((double)P[(int64_t)i * d + k] - mu[k]));
+        __nv_bfloat16 hi, lo;
+        split_bf16(z, hi, lo);
+        row_hi[o + k] = hi, row_lo[o + k] = lo;
+        col_hi[o + k] = hi, col_lo[o + k] = lo;
+        sq += (double)z * (double)z;
+    }
+    const double h = -0.5 * sq;
+    const __nv_bfloat16 h1 = __float2bfloat16_rn((float)h);
+    const double r1 = h - (double)__bfloat162float(h1);
+    const __nv_bfloat16 h2 = __float2bfloat16_rn((float)r1);
+    const __nv_bfloat16 h3 = __float2bfloat16_rn((float)(r1 - (double)__bfloat162float(h2)));
+    const __nv_bfloat16 one = __float2bfloat16_rn(1.f);
+    row_hi[o + d] = h1, row_hi[o + d + 1] = h2, row_hi[o + d + 2] = h3;
+    row_hi[o + d + 3] = one, row_hi[o + d + 4] = one, row_hi[o + d + 5] = one;
+    col_hi[o + d] = one, col_hi[o + d + 1] = one, col_hi[o + d + 2] = one;
+    col_hi[o + d + 3] = h1, col_hi[o + d + 4] = h2, col_hi[o + d + 5] = h3;
+    atomicMax(maxsq, __float_as_uint((float)sq));
+}
+
+// ---- the pass kernel ----------------------------------------------------------------------
+// partial[cs * pitch + i] = sum over the columns l of item (row tile of i, column split cs) of 2^(t_il) * vin[l].
+// vin is padded with zeros up to tiles * 128 entries, so the padding columns of the last tile contribute nothing.
+__global__ void __launch_bounds__(kImpThreads, 1)
+implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_constant__ CUtensorMap tmR_lo,
+                     const __grid_constant__ CUtensorMap tmC_hi, const __grid_constant__ CUtensorMap tmC_lo,
+                     const float *__restrict__ vin, float *__restrict__ partial, int64_t pitch, int nrows, int tiles,
+                     int T, int nsplit, int kd, FsDeviceStatus *status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bars = base + OFF_BARS;
+    const uint32_t item_full = bars, item_free_mma = bars + 16, item_free_epi = bars + 32;
+    const uint32_t b_full = bars + 48, b_empty = b_full + 8 * B_STAGES;
+    const uint32_t acc_full = b_empty + 8 * B_STAGES, acc_empty = acc_full + 16;
+    const uint32_t tmem_slot = bars + 8 * NUM_BARS;
+    uint32_t *tmem_slot_ptr = reinterpret_cast<uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nitems = tiles * nsplit;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(item_full + 8 * s, 1);
+            mbar_init(item_free_mma + 8 * s, 1);
+            mbar_init(item_free_epi + 8 * s, 8);
+            mbar_init(acc_full + 8 * s, 1);
+            mbar_init(acc_empty + 8 * s, 8);
+        }
+        for (int s = 0; s < B_STAGES; ++s) {
+            mbar_init(b_full + 8 * s, 1);
+            mbar_init(b_empty + 8 * s, 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem = *tmem_slot_ptr;
+    bool ok = true;
+
+    if (warp == 0) {
+        // ---------------- producer ----------------
+        if (lane == 0) {
+            int k = 0, bt = 0, ki = 0; // items begun, column tiles issued, items whose loads were issued
+            for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x, ++k) {
+                const int slot = k & 1;
+                const uint32_t ph = (uint32_t)(k >> 1) & 1u;
+                if (!mbar_wait(item_free_mma + 8 * slot, ph ^ 1u) || !mbar_wait(item_free_epi + 8 * slot, ph ^ 1u)) { ok = false; break; }
+                const int rt = w / nsplit, cs = w % nsplit;
+                const int t0 = cs * T, t1 = min(t0 + T, tiles);
+                const uint32_t full = item_full + 8 * slot;
+                mbar_expect_tx(full, (uint32_t)PAIR_BYTES + (uint32_t)(t1 - t0) * BN * 4u);
+                tma_load_2d(&tmR_hi, base + OFF_A + slot * PAIR_BYTES, full, 0, rt * BM);
+                tma_load_2d(&tmR_lo, base + OFF_A + slot * PAIR_BYTES + TILE_BYTES, full, 0, rt * BM);
+                bulk_load(base + OFF_V + slot * VSLOT_BYTES, vin + (int64_t)t0 * BN, (uint32_t)(t1 - t0) * BN * 4u, full);
+                ki = k + 1;
+                for (int j = t0; j < t1; ++j, ++bt) {
+                    const int s = bt % B_STAGES;
+                    if (!mbar_wait(b_empty + 8 * s, ((uint32_t)(bt / B_STAGES) & 1u) ^ 1u)) { ok = false; break; }
+                    const uint32_t bf = b_full + 8 * s, dst = base + OFF_B + s * PAIR_BYTES;
+                    mbar_expect_tx(bf, PAIR_BYTES);
+                    tma_load_2d(&tmC_hi, dst, bf, 0, j * BN);
+                    tma_load_2d(&tmC_lo, dst + TILE_BYTES, bf, 0, j * BN);
+                }
+            }
+            if (!ok) {
+                // drain: copies already issued must land before this CTA's shared memory goes away
+                for (int j = max(0, bt - B_STAGES); j < bt; ++j) (void)mbar_wait(b_full + 8 * (j % B_STAGES), (uint32_t)(j / B_STAGES) & 1u);
+                for (int j = max(0, ki - 2); j < ki; ++j) (void)mbar_wait(item_full + 8 * (j & 1), (uint32_t)(j >> 1) & 1u);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issue ----------------
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16_m128(BN);
+            int k = 0, bt = 0;
+            for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x, ++k) {
+                const int slot = k & 1;
+                if (!mbar_wait(item_full + 8 * slot, (uint32_t)(k >> 1) & 1u)) { ok = false; break; }
+                fence_after();
+                const int cs = w % nsplit;
+                const int t0 = cs * T, t1 = min(t0 + T, tiles);
+                const uint64_t a_hi = make_desc(base + OFF_A + slot * PAIR_BYTES), a_lo = make_desc(base + OFF_A + slot * PAIR_BYTES + TILE_BYTES);
+                for (int j = t0; j < t1; ++j, ++bt) {
+                    const int s = bt % B_STAGES, buf = bt & 1;
+                    if (!mbar_wait(acc_empty + 8 * buf, ((uint32_t)(bt >> 1) & 1u) ^ 1u)) { ok = false; break; }
+                    if (!mbar_wait(b_full + 8 * s, (uint32_t)(bt / B_STAGES) & 1u)) { ok = false; break; }
+                    fence_after();
+                    const uint32_t st = base + OFF_B + s * PAIR_BYTES;
+                    const uint64_t b_hi = make_desc(st), b_lo = make_desc(st + TILE_BYTES);
+                    const uint32_t acc = tmem + (uint32_t)(buf * BN);
+                    for (int kk = 0; kk < kd; ++kk) {
+                        const uint64_t adv = (uint64_t)(kk * 32 >> 4); // 16 bf16 = 32 bytes along the contraction
+                        mma_bf16(acc, a_lo + adv, b_hi + adv, idesc, kk > 0 ? 1u : 0u);
+                        mma_bf16(acc, a_hi + adv, b_lo + adv, idesc, 1u);
+                        mma_bf16(acc, a_hi + adv, b_hi + adv, idesc, 1u);
+                    }
+                    commit(b_empty + 8 * s);      // ring slot free once these MMAs have read it
+                    commit(acc_full + 8 * buf);   // exponent tile complete
+                }
+                if (ok) commit(item_free_mma + 8 * slot); // row operand slot free once every MMA of the item has read it
+            }
+        }
+    } else {
+        // ---------------- epilogue ----------------
+        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        const int row = quarter * 32 + lane;
+        int k = 0, bt = 0;
+        for (int w = blockIdx.x; w < nitems; w += gridDim.x, ++k) {
+            const int slot = k & 1;
+            const int rt = w / nsplit, cs = w % nsplit;
+            const int t0 = cs * T, t1 = min(t0 + T, tiles);
+            float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+            if (ok) ok = mbar_wait(item_full + 8 * slot, (uint32_t)(k >> 1) & 1u);
+            ok = __all_sync(0xffffffffu, ok);
+            for (int j = t0; j < t1 && ok; ++j, ++bt) {
+                const int buf = bt & 1;
+                ok = mbar_wait(acc_full + 8 * buf, (uint32_t)(bt >> 1) & 1u);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                fence_after();
+                const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2));
+                const uint32_t vaddr = base + OFF_V + slot * VSLOT_BYTES + (uint32_t)((j - t0) * BN + half * (BN / 2)) * 4u;
+                uint32_t ta[32], tb[32];
+                tmem_ld32_issue(taddr, ta);
+                tmem_ld32_issue(taddr + 32, tb);
+                tmem_ld_wait();
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float4 v4 = lds4(vaddr + (uint32_t)q * 16u);
+                    acc0 = fmaf(ex2(__uint_as_float(ta[4 * q + 0])), v4.x, acc0);
+                    acc1 = fmaf(ex2(__uint_as_float(ta[4 * q + 1])), v4.y, acc1);
+                    acc2 = fmaf(ex2(__uint_as_float(ta[4 * q + 2])), v4.z, acc2);
+                    acc3 = fmaf(ex2(__uint_as_float(ta[4 * q + 3])), v4.w, acc3);
+                }
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float4 v4 = lds4(vaddr + 128u + (uint32_t)q * 16u);
+                    acc0 = fmaf(ex2(__uint_as_float(tb[4 * q + 0])), v4.x, acc0);
+                    acc1 = fmaf(ex2(__uint_as_float(tb[4 * q + 1])), v4.y, acc1);
+                    acc2 = fmaf(ex2(__uint_as_float(tb[4 * q + 2])), v4.z, acc2);
+                    acc3 = fmaf(ex2(__uint_as_float(tb[4 * q + 3])), v4.w, acc3);
+                }
+                fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_empty + 8 * buf);
+            }
+            // the two column halves of a row are added in a fixed order; every epilogue warp reaches this barrier
+            // for every item, whatever happened before, so that nobody is left waiting
+            const float sum = (acc0 + acc1) + (acc2 + acc3);
+            const uint32_t comb = base + OFF_COMB + (uint32_t)(slot * BM + row) * 4u;
+            if (half == 1) asm volatile("st.shared.f32 [%0], %1;" ::"r"(comb), "f"(sum) : "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (half == 0 && ok) {
+                float other;
+                asm volatile("ld.shared.f32 %0, [%1];" : "=f"(other) : "r"(comb) : "memory");
+                const int gi = rt * BM + row;
+                if (gi < nrows) partial[(int64_t)cs * pitch + gi] = sum + other;
+            }
+            __syncwarp();
+            if (lane == 0 && ok) mbar_arrive(item_free_epi + 8 * slot);
+        }
+    }
+    if (!ok) status->timeout = 1;
+    fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// operand array of `rows` points x 64 bf16 (rows of 128 bytes); box = one 128-point tile, 128-byte swizzle
+bool make_map(CUtensorMap *map, const __nv_bfloat16 *ptr, int64_t rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)BK, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)BK * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16 *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+void implicit_free(ImplicitState *t) {
+    if (!t) return;
+    for (auto p : t->buf) cudaFree(p);
+    cudaFree(t->partials);
+    delete t;
+}
+
+// Column tiles per item: the smallest number of splits of a row tile's columns that keeps the persistent CTAs
+// evenly loaded (items are dealt round-robin, every item costs about the same).
+void choose_split(int tiles, int sms, int *T_out, int *nsplit_out) {
+    int bestT = tiles < MAX_T ? tiles : MAX_T;
+    double best_eff = -1.0;
+    for (int ns = (tiles + MAX_T - 1) / MAX_T; ns <= tiles && ns <= 64; ++ns) {
+        const int T = (tiles + ns - 1) / ns;
+        const int ns_eff = (tiles + T - 1) / T;
+        const int64_t items = (int64_t)tiles * ns_eff;
+        const int64_t rounds = (items + sms - 1) / sms;
+        // per-item overhead (row operand reload, pipeline fill) counted as one extra column tile
+        const double eff = (double)tiles * tiles / ((double)rounds * sms * (T + 1));
+        if (eff > best_eff * 1.02) best_eff = eff, bestT = T;
+    }
+    *T_out = bestT;
+    *nsplit_out = (tiles + bestT - 1) / bestT;
+}
+
+} // namespace
+
+void fsk_implicit_destroy(void *h) { implicit_free(static_cast<ImplicitState *>(h)); }
+
+int64_t fsk_implicit_padded_n(int64_t n) { return (n + BM - 1) / BM * BM; }
+int fsk_implicit_max_dim() { return kMaxDim; }
+
+// Builds the operand arrays of both clouds.  *err receives FS_OK, FS_ERR_UNSUPPORTED (d too large, no tensor-map
+// entry point, exponent error bound above the limit) or FS_ERR_CUDA.  Synchronises st.
+void *fsk_implicit_create(const float *X, const float *Y, int64_t n, int d, double cost_scale, double eps, cudaStream_t st,
+                          int *err, float *bound_out) {
+    *err = FS_ERR_UNSUPPORTED;
+    if (d < 1 || d > kMaxDim || !encode_fn()) return nullptr;
+    ImplicitState *t = new ImplicitState();
+    t->n = n, t->d = d;
+    t->n_pad = fsk_implicit_padded_n(n);
+    t->tiles = (int)(t->n_pad / BM);
+    t->kd = (d + 6 + 15) / 16;
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    choose_split(t->tiles, sms, &t->T, &t->nsplit);
+    const int64_t items = (int64_t)t->tiles * t->nsplit;
+    t->grid = (int)(items < sms ? items : sms);
+    const size_t bytes = (size_t)t->n_pad * BK * 2;
+    bool ok = true;
+    for (auto &p : t->buf) ok = ok && cudaMalloc(&p, bytes) == cudaSuccess && cudaMemsetAsync(p, 0, bytes, st) == cudaSuccess;
+    ok = ok && cudaMalloc(&t->partials, sizeof(float) * (size_t)t->nsplit * t->n_pad) == cudaSuccess;
+    double *mu = nullptr;
+    unsigned int *maxsq = nullptr;
+    ok = ok && cudaMalloc(&mu, sizeof(double) * d) == cudaSuccess && cudaMalloc(&maxsq, 2 * sizeof(unsigned int)) == cudaSuccess &&
+         cudaMemsetAsync(maxsq, 0, 2 * sizeof(unsigned int), st) == cudaSuccess;
+    float hmax[2] = {0.f, 0.f};
+    if (ok) {
+        const double sqrt2c = sqrt(2.0 * cost_scale / eps * 1.4426950408889634);
+        const unsigned grid = (unsigned)((n + 255) / 256);
+        cloud_mean_kernel<<<d, 256, 0, st>>>(X, Y, (int)n, d, mu);
+        prepare_points_kernel<<<grid, 256, 0, st>>>(X, (int)n, d, mu, sqrt2c, t->buf[0], t->buf[1], t->buf[2], t->buf[3], maxsq);
+        prepare_points_kernel<<<grid, 256, 0, st>>>(Y, (int)n, d, mu, sqrt2c, t->buf[4], t->buf[5], t->buf[6], t->buf[7], maxsq + 1);
+        ok = cudaGetLastError() == cudaSuccess &&
+             cudaMemcpyAsync(hmax, maxsq, 2 * sizeof(float), cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+             cudaStreamSynchronize(st) == cudaSuccess;
+    }
+    cudaFree(mu), cudaFree(maxsq);
+    for (int i = 0; i < 8 && ok; ++i) ok = make_map(&t->map[i], t->buf[i], t->n_pad);
+    ok = ok && cudaFuncSetAttribute(implicit_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        implicit_free(t);
+        *err = FS_ERR_CUDA;
+        return nullptr;
+    }
+    t->bound = (float)(ldexp(1.0, -16) * sqrt((double)hmax[0]) * sqrt((double)hmax[1]));
+    if (bound_out) *bound_out = t->bound;
+    if (!(t->bound <= 1e-3f)) {
+        implicit_free(t);
+        *err = FS_ERR_UNSUPPORTED;
+        return nullptr;
+    }
+    *err = FS_OK;
+    return t;
+}
+
+int fsk_implicit_nsplit(const void *h) { return static_cast<const ImplicitState *>(h)->nsplit; }
+float *fsk_implicit_partials(void *h) { return static_cast<ImplicitState *>(h)->partials; }
+
+// Stage 1 of one half-step: transposed = 0: partial sums of K in (rows = X, columns = Y); 1: of K^T in.
+// `in` holds n_pad floats, zero beyond n.  The caller runs the stage-2 kernel over [nsplit][n_pad].
+cudaError_t fsk_implicit_pass(void *h, int transposed, const float *in, FsDeviceStatus *status, cudaStream_t st) {
+    ImplicitState *t = static_cast<ImplicitState *>(h);
+    const int r = transposed ? 4 : 0, c = transposed ? 2 : 6; // row-side arrays of one cloud, column-side of the other
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)t->grid);
+    cfg.blockDim = dim3(kImpThreads);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = st;
+    return cudaLaunchKernelEx(&cfg, implicit_pass_kernel, t->map[r], t->map[r + 1], t->map[c], t->map[c + 1], in, t->partials,
+                              t->n_pad, (int)t->n, t->tiles, t->T, t->nsplit, t->kd, status);
+}

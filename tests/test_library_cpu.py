@@ -71,6 +71,19 @@ def test_host_side_validation_needs_no_device(lib):
     assert create(domain=1, kind=0) == fs.FS_ERR_DOMAIN
     assert create(domain=1, kind=1, nbatch=2) == fs.FS_ERR_UNSUPPORTED
     assert out.value is None
+
+    def create_points(n=8, c=2, offsets=offp, X=fake, Y=fake, d=3, scale=1.0, eps=0.1, a=fake, b=fake):
+        return lib.fs_create_points(ctypes.byref(out), n, c, offsets, X, Y, d, scale, eps, a, b, None)
+
+    assert create_points(X=None) == fs.FS_ERR_NULL
+    assert create_points(b=None) == fs.FS_ERR_NULL
+    assert create_points(n=0) == fs.FS_ERR_BAD_N
+    assert create_points(d=0) == fs.FS_ERR_BAD_N
+    assert create_points(d=59) == fs.FS_ERR_UNSUPPORTED
+    assert create_points(c=9) == fs.FS_ERR_BAD_OFFSETS
+    assert create_points(eps=0.0) == fs.FS_ERR_BAD_EPS
+    assert create_points(scale=-1.0) == fs.FS_ERR_BAD_EPS
+    assert out.value is None
     # NULL handles
     assert lib.fs_iterate(None, 1, None) == fs.FS_ERR_NULL
     assert lib.fs_destroy(None) == fs.FS_ERR_NULL
