@@ -14,6 +14,7 @@ the timed region starts.  Rank 0 prints ONE JSON line.  Keys beyond the basic co
                 time x clock (SM cycles per launch)
   other_paths   config 4 on the two-pass path (K streamed twice per iteration): the row pass and the
                 column pass each timed alone, and whole iterations
+                and through the implicit-kernel path (fs_create_points) with its ex2-rate ("alu") roofline
   cpu_baseline  the fp64 CPU checker timed on this machine's host cores on a few iterations, with all
                 cores (OpenMP) and on one thread
   e2e           the same metric through fs_solve_host: host buffers in, host buffers out, all
@@ -322,6 +323,112 @@ def time_config(fs, torch, dev, stream, w, steps=3, device_index=0):
                       ms * 1e-3 / its, clocks, "sm_cycles_per_iteration")
 
 
+def run_implicit_only(args, rank, local_rank, world):
+    """--path implicit: one JSON line for the implicit-kernel path alone (profiling runs, scaled-down sizes)."""
+    import torch
+    from paper_2502_07021_b200 import binding as fs
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.Stream(device=dev)
+    wp = workloads.make(args.config, n=args.n, nbatch=1, fp32_points=True, want_cost=False, want_kernel=False)
+    if args.iters is not None:
+        wp.iters = args.iters
+    r = time_implicit(fs, torch, dev, stream, wp, visible_device_index(local_rank), args, wp=wp)
+    if rank != 0:
+        return
+    line = {"metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world, "steps": r["steps"], "warmup": 3,
+            "ms_per_step": r["us_per_iteration"] * wp.iters * 1e-3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"config {wp.cfg} from its point clouds: n={wp.n} d={wp.X.shape[1]} eps={wp.eps}, "
+                                   f"{wp.iters} iterations per step, kernel applied implicitly"},
+            "gpu_launches": 4 * wp.iters * r["steps"], "clocks": r.get("clocks"), "e2e": r.get("e2e"),
+            "roofline": r["roofline"], "cpu_baseline": None}
+    print(json.dumps(line), flush=True)
+
+
+def time_implicit(fs, torch, dev, stream, w, devidx, args, wp=None):
+    """Config `w` from its fp32 point clouds through fs_create_points: device-timed it/s, the ex2 roofline of its
+    pass kernel and the end-to-end rate through fs_solve_host_points."""
+    if wp is None:
+        wp = workloads.make(w.cfg, fp32_points=True, want_cost=False, want_kernel=False)
+    d = wp.X.shape[1]
+    X = torch.from_numpy(wp.X).to(dev)
+    Y = torch.from_numpy(wp.Y).to(dev)
+    a = torch.from_numpy(wp.a).to(dev)
+    b = torch.from_numpy(wp.b).to(dev)
+    torch.cuda.synchronize()
+    h = fs.fs_create_points(wp.n, wp.c, wp.offsets, X, Y, d, wp.cost_scale, wp.eps, a, b, stream)
+    try:
+        def step():
+            fs.fs_reset(h, stream)
+            fs.fs_iterate(h, wp.iters, stream)
+        for _ in range(3):
+            step()
+        stream.synchronize()
+        steps = max(1, min(args.steps, 5))
+        smp = NvmlSampler(devidx)
+        smp.start()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            step()
+        e1.record(stream)
+        stream.synchronize()
+        clocks = smp.stop()
+        ms = e0.elapsed_time(e1)
+        row, col = fs.fs_marginal_error(h, 1, 1, stream)
+        # the special-function rate right after, at the clock the board holds under this kind of load
+        smp2 = NvmlSampler(devidx)
+        smp2.start()
+        ex2_rate = fs.fs_selftest_ex2_rate(1 << 15, stream)
+        ex2_clocks = smp2.stop()
+    finally:
+        fs.fs_destroy(h)
+    its = steps * wp.iters
+    pass_s = ms * 1e-3 / (2 * its)
+    n2 = float(wp.n) * float(wp.n)
+    achieved = n2 / pass_s
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    nominal = 16.0 * sms * (clocks["sm_mhz"] * 1e6 if clocks and clocks.get("sm_mhz") else 1.965e9)
+    out = {"what": "fs_create_points: K_il = exp(-s|x_i - y_l|^2/eps) formed on the fly (tcgen05 contraction + one ex2 per "
+                   "element per pass), two implicit_pass_kernel launches and two stage-2 launches per iteration",
+           "value": its / (ms * 1e-3), "unit": UNIT, "us_per_iteration": ms * 1e3 / its, "steps": steps,
+           "iterations_per_step": wp.iters, "points_bytes": int(2 * wp.n * d * 4),
+           "final_row_marginal_l1": float(row[0]), "final_col_marginal_l1": float(col[0]),
+           "roofline": {"bound": "alu", "kernel": "implicit_pass_kernel", "unit": "Gex2/s",
+                        "achieved": achieved / 1e9, "peak": ex2_rate / 1e9, "frac": achieved / ex2_rate,
+                        "peak_source": "measured: fs_selftest_ex2_rate (every thread issues independent ex2.approx) right "
+                                       "after the timed region",
+                        "peak_clocks": ex2_clocks,
+                        "nominal_peak": nominal / 1e9,
+                        "nominal_peak_source": "16 ex2 per clock per SM x SM count x the median SM clock sampled in the "
+                                               "timed region",
+                        "frac_of_nominal": achieved / nominal,
+                        "algorithmic_ex2_per_launch": n2, "us_per_launch": pass_s * 1e6, "traffic": None}}
+    with_clock(out, ms * 1e-3 / its, clocks, "sm_cycles_per_iteration")
+    if not args.no_e2e:
+        pin = [torch.from_numpy(x).pin_memory() for x in (wp.X, wp.Y, wp.a, wp.b)]
+        uo = torch.empty(wp.n, dtype=torch.float32).pin_memory()
+        vo = torch.empty(wp.n, dtype=torch.float32).pin_memory()
+        call = lambda: fs.fs_solve_host_points(wp.n, wp.c, wp.offsets, pin[0], pin[1], d, wp.cost_scale, wp.eps, pin[2],
+                                               pin[3], wp.iters, uo, vo)
+        call()
+        ts = []
+        for _ in range(3):
+            t0 = time.perf_counter()
+            call()
+            ts.append(time.perf_counter() - t0)
+        med = statistics.median(ts)
+        out["e2e"] = {"value": wp.iters / med, "unit": UNIT, "ms_per_step": med * 1e3,
+                      "h2d_bytes_per_step": int(2 * wp.n * d * 4 + 2 * wp.n * 4), "d2h_bytes_per_step": int(2 * wp.n * 4 + 8),
+                      "note": "fs_solve_host_points: allocation, H2D of the two clouds and the marginals, operand set-up, all "
+                              "iterations, marginal error, D2H of the scalings, free -- every step"}
+    return out
+
+
 def run_sharded(args, rank, local_rank, world):
     """Row-partitioned run (opt-in, --multi sharded): one shard of the SAME problem per GPU, one all-reduce
     of n floats per iteration over NCCL; total work is fixed, so scaling is strong."""
@@ -543,6 +650,16 @@ def run_ours(args, w, rank, local_rank, world):
                                       "frac_of_nominal_8000_gbs": 2 * n2 * w.iters / it_s / 1e9 / 8000.0},
                                      it_s / w.iters, it_clk, "sm_cycles_per_iteration")}}
 
+    # the same configuration with the kernel applied implicitly from the point clouds (fs_create_points): no matrix in
+    # memory, one ex2 per matrix element per pass; bound by the special-function units ("alu" roofline)
+    if world == 1 and not args.headline_only and args.n is None and w.cfg in (2, 4) and w.nbatch == 1:
+        try:
+            if other_paths is None:
+                other_paths = {}
+            other_paths["implicit"] = time_implicit(fs, torch, dev, stream, w, devidx, args)
+        except Exception as exc:  # must not lose the headline line
+            other_paths = dict(other_paths or {}, implicit={"error": repr(exc)})
+
     # the other four configurations, briefly (single GPU runs only): same step definition, fewer steps
     others = None
     if world == 1 and not args.headline_only and args.config == 4 and args.n is None and args.iters is None:
@@ -633,6 +750,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--multi", default="replicas", choices=["replicas", "sharded"],
                     help="N > 1: independent replicas (default, weak scaling) or row shards of one problem")
+    ap.add_argument("--path", default="auto", choices=["auto", "implicit"],
+                    help="implicit: time only the implicit-kernel path (fs_create_points) of the configuration")
     ap.add_argument("--headline-only", action="store_true", help="skip the short runs of configurations 1, 2, 3, 5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic-bytes", type=float, default=None,
@@ -655,6 +774,10 @@ def main():
             run_sharded(args, rank, local_rank, world)
         finally:
             fsdist.finalize()
+        return 0
+    if args.path == "implicit":
+        run_implicit_only(args, rank, local_rank, world)
+        fsdist.finalize()
         return 0
     w = workloads.make(args.config, n=args.n, want_cost=None if args.config == 3 else False)
     if args.iters is not None:

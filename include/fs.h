@@ -322,6 +322,16 @@ int fs_shard_destroy(fs_shard *s);
  */
 int fs_selftest_bounded_wait(int32_t poll_limit, int32_t arrive, int32_t *timed_out, void *stream);
 
+/*
+ * fs_selftest_ex2_rate -- measures what the GPU's special-function units sustain on ex2.approx, the instruction
+ * that bounds the implicit-kernel passes (one per matrix element) and the log-domain passes: a kernel in which
+ * every thread runs `iters` rounds of eight independent ex2 (1 <= iters <= 2^24; 2048 threads per SM), timed with
+ * CUDA events on `stream`.  *ex2_per_second (HOST) receives the rate.  It is the denominator of the "alu" roofline
+ * the benchmark reports for those passes (nominally 16 per clock per SM).  Synchronises `stream`.  (Measurement
+ * aid; no counterpart in the paper.)
+ */
+int fs_selftest_ex2_rate(int32_t iters, double *ex2_per_second, void *stream);
+
 const char *fs_strerror(int code);
 
 /* Text of the last CUDA error seen by this thread's calls ("" if none). */

@@ -61,6 +61,7 @@ _SIGNATURES = {
     "fs_shard_row_error": (_int, [_vp, _vp, _vp, _vp]),
     "fs_shard_destroy": (_int, [_vp]),
     "fs_selftest_bounded_wait": (_int, [_i32, _i32, ctypes.POINTER(_i32), _vp]),
+    "fs_selftest_ex2_rate": (_int, [_i32, ctypes.POINTER(_dbl), _vp]),
     "fs_strerror": (ctypes.c_char_p, [_int]),
     "fs_last_cuda_error": (ctypes.c_char_p, []),
 }
@@ -312,6 +313,13 @@ def fs_solve_host_points(n, c, row_offsets, X_host, Y_host, d, cost_scale, eps, 
                                       _host_ptr(a_host), _host_ptr(b_host), iters, _host_ptr(u_out), _host_ptr(v_out),
                                       err.ctypes.data_as(_vp) if want_error else None), "fs_solve_host_points")
     return err
+
+
+def fs_selftest_ex2_rate(iters=4096, stream=None):
+    """ex2.approx per second sustained by the special-function units (microbenchmark)."""
+    out = _dbl(0.0)
+    _check(lib().fs_selftest_ex2_rate(iters, ctypes.byref(out), _stream(stream)), "fs_selftest_ex2_rate")
+    return out.value
 
 
 def fs_solve_host(n, c, row_offsets, M_host, ld, matrix_kind, eps, a_host, b_host, nbatch, domain, iters,

@@ -222,8 +222,8 @@ void *fsk_implicit_create(const float *X, const float *Y, int64_t n, int d, doub
 void fsk_implicit_destroy(void *h);
 int64_t fsk_implicit_padded_n(int64_t n); // length of the zero-padded input vectors the pass reads
 int fsk_implicit_max_dim();
-int fsk_implicit_nsplit(const void *h);
-float *fsk_implicit_partials(void *h);    // [nsplit][padded n] partial sums written by a pass
+int fsk_implicit_nsplit(const void *h);   // number of partial rows a pass writes
+float *fsk_implicit_partials(void *h);    // [partial rows][padded n] partial sums written by a pass
 cudaError_t fsk_implicit_pass(void *h, int transposed, const float *in, FsDeviceStatus *status, cudaStream_t st);
 
 // ---- setup.cu ----------------------------------------------------------------------------

@@ -17,12 +17,12 @@
 // One kernel serves both half-steps of Algorithm 1: the row pass takes X as row operand, Y as column operand and
 // v as input; the column pass takes Y as row operand, X as column operand and u as input (K^T tiles are formed
 // directly, no transposition).  Work item = (128-row tile, range of column tiles); items are dealt round-robin to
-// persistent CTAs; each item writes one partial sum per row, and the ordinary stage-2 kernel adds the partials of a
+// persistent CTAs; each item writes four partial sums per row (one per epilogue warpgroup), and the ordinary stage-2 kernel adds the partials of a
 // row in a fixed order and applies the divide: deterministic, no atomics.
 //
 // CTA: warp 0 issues TMA loads (row operand tile and the input-vector slice once per item, column operand tiles
-// through a 3-stage ring), warp 1 issues the MMAs into two 128-column accumulators in turn, warps 2..9 are the
-// epilogue (TMEM lane quarter = warp % 4, column half = (warp - 2) / 4).  The bound is the special-function unit:
+// through a 3-stage ring), warp 1 issues the MMAs into four 128-column accumulators in turn, warps 2..17 are the
+// epilogue (TMEM lane quarter = warp % 4, warpgroup = (warp - 2) / 4 owns one accumulator).  The bound is the special-function unit:
 // one ex2 per matrix element per pass.  Every wait is bounded; on expiry the kernel raises the status flag, skips
 // the remaining work and still passes every barrier before it frees its tensor memory and exits.
 //
@@ -43,16 +43,17 @@ constexpr int PAIR_BYTES = 2 * TILE_BYTES;   // hi + lo
 constexpr int B_STAGES = 3;
 constexpr int MAX_T = 32;                    // column tiles per work item (input slice of at most 16 KB)
 constexpr int VSLOT_BYTES = MAX_T * BN * 4;
-constexpr int kImpThreads = 320;             // TMA warp, MMA warp, eight epilogue warps
-constexpr int TMEM_COLS = 256;               // two 128-column fp32 accumulators
+constexpr int EPI_WARPS = 16;                // four per scheduler: enough independent ex2 in flight to keep the unit busy
+constexpr int kImpThreads = 64 + 32 * EPI_WARPS; // TMA warp, MMA warp, sixteen epilogue warps
+constexpr int NACC = 4;                      // exponent tiles in flight between the tensor core and the epilogue
+constexpr int TMEM_COLS = NACC * BN;         // four 128-column fp32 accumulators: all of tensor memory
 constexpr int kMaxDim = BK - 6;              // coordinates + 3 norm terms + 3 ones fit one 64-column k-block
-// shared memory: A slots, B ring, input slots, combine buffers, barriers, TMEM slot
+// shared memory: A slots, B ring, input slots, barriers, TMEM slot
 constexpr int OFF_A = 0;
 constexpr int OFF_B = OFF_A + 2 * PAIR_BYTES;
 constexpr int OFF_V = OFF_B + B_STAGES * PAIR_BYTES;
-constexpr int OFF_COMB = OFF_V + 2 * VSLOT_BYTES;
-constexpr int OFF_BARS = OFF_COMB + 2 * BM * 4;
-constexpr int NUM_BARS = 6 + 2 * B_STAGES + 4; // item_full[2], item_free_mma[2], item_free_epi[2], b_full, b_empty, acc_full[2], acc_empty[2]
+constexpr int OFF_BARS = OFF_V + 2 * VSLOT_BYTES;
+constexpr int NUM_BARS = 6 + 2 * B_STAGES + 2 * NACC; // item_full[2], item_free_mma[2], item_free_epi[2], b_full, b_empty, acc_full, acc_empty
 constexpr int SMEM_BYTES = OFF_BARS + 8 * NUM_BARS + 16 + 1024;
 
 struct ImplicitState {
@@ -64,7 +65,7 @@ struct ImplicitState {
     float bound = 0.f;            // bound on the absolute error of the exponent
     __nv_bfloat16 *buf[8] = {};   // X row-side hi, lo; X column-side hi, lo; Y row-side hi, lo; Y column-side hi, lo
     CUtensorMap map[8];
-    float *partials = nullptr;    // [nsplit][n_pad]
+    float *partials = nullptr;    // [nsplit * NACC][n_pad]: one partial sum per row, column split and warpgroup
 };
 
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
@@ -121,8 +122,27 @@ prepare_points_kernel(const float *__restrict__ P, int n, int d, const double *_
     atomicMax(maxsq, __float_as_uint((float)sq));
 }
 
+// 32 exponents of one row -> 32 kernel entries -> four running sums of K_il * in_l.  All 32 ex2 are issued before
+// the first multiply-add that needs one: with few epilogue warps per scheduler the special-function unit is only
+// kept busy if every warp has many independent ex2 in flight.
+__device__ __forceinline__ void consume_chunk(const uint32_t *r, uint32_t vaddr, float &acc0, float &acc1, float &acc2,
+                                              float &acc3) {
+    float e[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) e[j] = ex2(__uint_as_float(r[j]));
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const float4 v4 = lds4(vaddr + (uint32_t)q * 16u);
+        acc0 = fmaf(e[4 * q + 0], v4.x, acc0);
+        acc1 = fmaf(e[4 * q + 1], v4.y, acc1);
+        acc2 = fmaf(e[4 * q + 2], v4.z, acc2);
+        acc3 = fmaf(e[4 * q + 3], v4.w, acc3);
+    }
+}
+
 // ---- the pass kernel ----------------------------------------------------------------------
-// partial[cs * pitch + i] = sum over the columns l of item (row tile of i, column split cs) of 2^(t_il) * vin[l].
+// partial[(cs * 4 + g) * pitch + i] = sum over the columns l of the tiles that warpgroup g consumed of item (row tile
+// of i, column split cs) of 2^(t_il) * vin[l]; which tiles those are depends only on the launch geometry.
 // vin is padded with zeros up to tiles * 128 entries, so the padding columns of the last tile contribute nothing.
 __global__ void __launch_bounds__(kImpThreads, 1)
 implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_constant__ CUtensorMap tmR_lo,
@@ -134,7 +154,7 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
     const uint32_t bars = base + OFF_BARS;
     const uint32_t item_full = bars, item_free_mma = bars + 16, item_free_epi = bars + 32;
     const uint32_t b_full = bars + 48, b_empty = b_full + 8 * B_STAGES;
-    const uint32_t acc_full = b_empty + 8 * B_STAGES, acc_empty = acc_full + 16;
+    const uint32_t acc_full = b_empty + 8 * B_STAGES, acc_empty = acc_full + 8 * NACC;
     const uint32_t tmem_slot = bars + 8 * NUM_BARS;
     uint32_t *tmem_slot_ptr = reinterpret_cast<uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -144,9 +164,11 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
         for (int s = 0; s < 2; ++s) {
             mbar_init(item_full + 8 * s, 1);
             mbar_init(item_free_mma + 8 * s, 1);
-            mbar_init(item_free_epi + 8 * s, 8);
+            mbar_init(item_free_epi + 8 * s, EPI_WARPS);
+        }
+        for (int s = 0; s < NACC; ++s) {
             mbar_init(acc_full + 8 * s, 1);
-            mbar_init(acc_empty + 8 * s, 8);
+            mbar_init(acc_empty + 8 * s, EPI_WARPS / NACC);
         }
         for (int s = 0; s < B_STAGES; ++s) {
             mbar_init(b_full + 8 * s, 1);
@@ -208,8 +230,8 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
                 const int t0 = cs * T, t1 = min(t0 + T, tiles);
                 const uint64_t a_hi = make_desc(base + OFF_A + slot * PAIR_BYTES), a_lo = make_desc(base + OFF_A + slot * PAIR_BYTES + TILE_BYTES);
                 for (int j = t0; j < t1; ++j, ++bt) {
-                    const int s = bt % B_STAGES, buf = bt & 1;
-                    if (!mbar_wait(acc_empty + 8 * buf, ((uint32_t)(bt >> 1) & 1u) ^ 1u)) { ok = false; break; }
+                    const int s = bt % B_STAGES, buf = bt % NACC;
+                    if (!mbar_wait(acc_empty + 8 * buf, ((uint32_t)(bt / NACC) & 1u) ^ 1u)) { ok = false; break; }
                     if (!mbar_wait(b_full + 8 * s, (uint32_t)(bt / B_STAGES) & 1u)) { ok = false; break; }
                     fence_after();
                     const uint32_t st = base + OFF_B + s * PAIR_BYTES;
@@ -229,59 +251,53 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
         }
     } else {
         // ---------------- epilogue ----------------
-        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        // Four warpgroups of four warps.  Warpgroup g owns accumulator g and consumes the tiles bt = g, g + 4, ... of
+        // this CTA's tile stream on its own: a thread holds one row (TMEM lane quarter = warp % 4) and walks its
+        // 128 columns in four chunks of 32, the TMEM load of the next chunk in flight while the current one goes
+        // through the special-function unit.  The four warps that share a scheduler belong to different
+        // warpgroups and therefore sit in different phases of their tiles, which keeps the unit fed; the
+        // warpgroups meet nowhere: each writes its own partial sum per row and item.
+        const int quarter = warp & 3, wg = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;
-        int k = 0, bt = 0;
+        const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(wg * BN);
+        int k = 0, bt0 = 0; // items begun; index in the CTA's tile stream of the item's first tile
         for (int w = blockIdx.x; w < nitems; w += gridDim.x, ++k) {
             const int slot = k & 1;
             const int rt = w / nsplit, cs = w % nsplit;
             const int t0 = cs * T, t1 = min(t0 + T, tiles);
+            const uint32_t vslot = base + OFF_V + slot * VSLOT_BYTES;
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
             if (ok) ok = mbar_wait(item_full + 8 * slot, (uint32_t)(k >> 1) & 1u);
             ok = __all_sync(0xffffffffu, ok);
-            for (int j = t0; j < t1 && ok; ++j, ++bt) {
-                const int buf = bt & 1;
-                ok = mbar_wait(acc_full + 8 * buf, (uint32_t)(bt >> 1) & 1u);
+            // first tile of this item that belongs to the warpgroup
+            for (int jj = (wg - bt0) & (NACC - 1); jj < t1 - t0 && ok; jj += NACC) {
+                const int bt = bt0 + jj;
+                ok = mbar_wait(acc_full + 8 * wg, (uint32_t)(bt / NACC) & 1u);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 fence_after();
-                const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2));
-                const uint32_t vaddr = base + OFF_V + slot * VSLOT_BYTES + (uint32_t)((j - t0) * BN + half * (BN / 2)) * 4u;
-                uint32_t ta[32], tb[32];
-                tmem_ld32_issue(taddr, ta);
-                tmem_ld32_issue(taddr + 32, tb);
-                tmem_ld_wait();
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float4 v4 = lds4(vaddr + (uint32_t)q * 16u);
-                    acc0 = fmaf(ex2(__uint_as_float(ta[4 * q + 0])), v4.x, acc0);
-                    acc1 = fmaf(ex2(__uint_as_float(ta[4 * q + 1])), v4.y, acc1);
-                    acc2 = fmaf(ex2(__uint_as_float(ta[4 * q + 2])), v4.z, acc2);
-                    acc3 = fmaf(ex2(__uint_as_float(ta[4 * q + 3])), v4.w, acc3);
-                }
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float4 v4 = lds4(vaddr + 128u + (uint32_t)q * 16u);
-                    acc0 = fmaf(ex2(__uint_as_float(tb[4 * q + 0])), v4.x, acc0);
-                    acc1 = fmaf(ex2(__uint_as_float(tb[4 * q + 1])), v4.y, acc1);
-                    acc2 = fmaf(ex2(__uint_as_float(tb[4 * q + 2])), v4.z, acc2);
-                    acc3 = fmaf(ex2(__uint_as_float(tb[4 * q + 3])), v4.w, acc3);
-                }
+                const uint32_t vaddr = vslot + (uint32_t)(jj * BN) * 4u;
+                uint32_t ra[32], rb[32];
+                tmem_ld32_issue(lane_base, ra);
+                tmem_ld_wait32(ra);
+                tmem_ld32_issue(lane_base + 32, rb);
+                consume_chunk(ra, vaddr, acc0, acc1, acc2, acc3);
+                tmem_ld_wait32(rb);
+                tmem_ld32_issue(lane_base + 64, ra);
+                consume_chunk(rb, vaddr + 128u, acc0, acc1, acc2, acc3);
+                tmem_ld_wait32(ra);
+                tmem_ld32_issue(lane_base + 96, rb);
+                consume_chunk(ra, vaddr + 256u, acc0, acc1, acc2, acc3);
+                tmem_ld_wait32(rb);
                 fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(acc_empty + 8 * buf);
+                if (lane == 0) mbar_arrive(acc_empty + 8 * wg); // the whole tile has left tensor memory
+                consume_chunk(rb, vaddr + 384u, acc0, acc1, acc2, acc3);
             }
-            // the two column halves of a row are added in a fixed order; every epilogue warp reaches this barrier
-            // for every item, whatever happened before, so that nobody is left waiting
-            const float sum = (acc0 + acc1) + (acc2 + acc3);
-            const uint32_t comb = base + OFF_COMB + (uint32_t)(slot * BM + row) * 4u;
-            if (half == 1) asm volatile("st.shared.f32 [%0], %1;" ::"r"(comb), "f"(sum) : "memory");
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (half == 0 && ok) {
-                float other;
-                asm volatile("ld.shared.f32 %0, [%1];" : "=f"(other) : "r"(comb) : "memory");
+            bt0 += t1 - t0;
+            if (ok) {
                 const int gi = rt * BM + row;
-                if (gi < nrows) partial[(int64_t)cs * pitch + gi] = sum + other;
+                if (gi < nrows) partial[(int64_t)(cs * NACC + wg) * pitch + gi] = (acc0 + acc1) + (acc2 + acc3);
             }
             __syncwarp();
             if (lane == 0 && ok) mbar_arrive(item_free_epi + 8 * slot);
@@ -376,7 +392,7 @@ void *fsk_implicit_create(const float *X, const float *Y, int64_t n, int d, doub
     const size_t bytes = (size_t)t->n_pad * BK * 2;
     bool ok = true;
     for (auto &p : t->buf) ok = ok && cudaMalloc(&p, bytes) == cudaSuccess && cudaMemsetAsync(p, 0, bytes, st) == cudaSuccess;
-    ok = ok && cudaMalloc(&t->partials, sizeof(float) * (size_t)t->nsplit * t->n_pad) == cudaSuccess;
+    ok = ok && cudaMalloc(&t->partials, sizeof(float) * (size_t)t->nsplit * NACC * t->n_pad) == cudaSuccess;
     double *mu = nullptr;
     unsigned int *maxsq = nullptr;
     ok = ok && cudaMalloc(&mu, sizeof(double) * d) == cudaSuccess && cudaMalloc(&maxsq, 2 * sizeof(unsigned int)) == cudaSuccess &&
@@ -412,11 +428,11 @@ void *fsk_implicit_create(const float *X, const float *Y, int64_t n, int d, doub
     return t;
 }
 
-int fsk_implicit_nsplit(const void *h) { return static_cast<const ImplicitState *>(h)->nsplit; }
+int fsk_implicit_nsplit(const void *h) { return static_cast<const ImplicitState *>(h)->nsplit * NACC; }
 float *fsk_implicit_partials(void *h) { return static_cast<ImplicitState *>(h)->partials; }
 
 // Stage 1 of one half-step: transposed = 0: partial sums of K in (rows = X, columns = Y); 1: of K^T in.
-// `in` holds n_pad floats, zero beyond n.  The caller runs the stage-2 kernel over [nsplit][n_pad].
+// `in` holds n_pad floats, zero beyond n.  The caller runs the stage-2 kernel over the fsk_implicit_nsplit() partial rows.
 cudaError_t fsk_implicit_pass(void *h, int transposed, const float *in, FsDeviceStatus *status, cudaStream_t st) {
     ImplicitState *t = static_cast<ImplicitState *>(h);
     const int r = transposed ? 4 : 0, c = transposed ? 2 : 6; // row-side arrays of one cloud, column-side of the other

@@ -179,6 +179,22 @@ __global__ void bounded_wait_probe_kernel(uint32_t limit, int arrive, int *timed
     if (threadIdx.x == 32) *timed_out = fsptx::mbar_wait_limited(b, 0, limit) ? 0 : 1;
 }
 
+// Special-function-unit microbenchmark: every thread runs `iters` rounds of eight independent ex2.approx
+// (each followed by one add that keeps the values in [-1, 0]); nothing else competes for the unit.
+__global__ void __launch_bounds__(256) ex2_rate_kernel(int iters, float *__restrict__ out) {
+    float x[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) x[j] = -0.125f * (float)(j + 1) - 1e-3f * (float)(threadIdx.x & 31);
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) x[j] = fsptx::ex2(x[j]) - 1.0f;
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s += x[j];
+    out[(size_t)blockIdx.x * 256 + threadIdx.x] = s;
+}
+
 unsigned grid_for(int64_t count) {
     int64_t g = (count + kThreads - 1) / kThreads;
     return (unsigned)(g < 1 ? 1 : (g > 148 * 16 ? 148 * 16 : g));
@@ -243,5 +259,38 @@ extern "C" int fs_selftest_bounded_wait(int32_t poll_limit, int32_t arrive, int3
         return FS_ERR_CUDA;
     }
     *timed_out = h;
+    return FS_OK;
+}
+
+extern "C" int fs_selftest_ex2_rate(int32_t iters, double *ex2_per_second, void *stream) {
+    if (!ex2_per_second) return FS_ERR_NULL;
+    if (iters < 1 || iters > (1 << 24)) return FS_ERR_BAD_N;
+    cudaStream_t st = (cudaStream_t)stream;
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FS_ERR_CUDA;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int blocks = sms * 8; // 2048 threads per SM: every scheduler has warps to issue from
+    float *out = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    cudaError_t e = cudaMalloc(&out, sizeof(float) * 256 * (size_t)blocks);
+    if (e == cudaSuccess) e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) {
+        ex2_rate_kernel<<<blocks, 256, 0, st>>>(iters / 16 + 1, out); // warm-up
+        cudaEventRecord(e0, st);
+        ex2_rate_kernel<<<blocks, 256, 0, st>>>(iters, out);
+        cudaEventRecord(e1, st);
+        e = cudaEventSynchronize(e1);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(out);
+    if (e != cudaSuccess || !(ms > 0.f)) {
+        cudaGetLastError();
+        return FS_ERR_CUDA;
+    }
+    *ex2_per_second = 8.0 * (double)iters * 256.0 * (double)blocks / ((double)ms * 1e-3);
     return FS_OK;
 }

@@ -68,6 +68,16 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t *r) {
                  : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// The same wait, tied to the 32 registers of an earlier tmem_ld32_issue: the load is asynchronous, so every use of
+// those registers has to stay behind the wait; naming them as read-write operands makes that a data dependency.
+__device__ __forceinline__ void tmem_ld_wait32(uint32_t *r) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :: "memory");
+}
 
 // Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes with the 128-byte
 // swizzle: 8-row groups 1024 bytes apart (stride byte offset), descriptor version 1.
