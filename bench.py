@@ -442,7 +442,7 @@ def run_sharded(args, rank, local_rank, world):
     stream = torch.cuda.Stream(device=dev)
     n_total = args.n or workloads._SPECS[args.config]["n"]
     lo, hi = fsdist.row_range(n_total, rank, world)
-    w = workloads.make(args.config, n=args.n, want_cost=False, rows=(lo, hi))
+    w = workloads.make(args.config, n=args.n, nbatch=1, want_cost=False, rows=(lo, hi))
     if w.domain != workloads.DOMAIN_SCALING or w.nbatch != 1:
         raise RuntimeError("--multi sharded covers the single-problem scaling-domain configurations")
     if args.iters is not None:
@@ -456,9 +456,15 @@ def run_sharded(args, rank, local_rank, world):
     torch.cuda.synchronize()
     sh = fs.fs_shard_create(w.n, lo, hi - lo, Kb, w.n, fs.FS_MATRIX_KERNEL, w.eps, a_loc, b, stream)
 
-    def step():
+    sizes = [fsdist.row_range(n_total, r, world)[1] - fsdist.row_range(n_total, r, world)[0] for r in range(world)]
+    split = {"local_ms": 0.0, "exchange_ms": 0.0}
+
+    def step(timed=False):
         fs.fs_shard_set_scalings(sh, ones_u, ones_v, stream)
-        fsdist.sharded_iterate(fs, sh, r_buf, w.iters, stream)
+        t = fsdist.sharded_iterate(fs, sh, r_buf, w.iters, stream, exchange=args.exchange, sizes=sizes, timed=timed)
+        if t:
+            split["local_ms"] += t["local_ms"]
+            split["exchange_ms"] += t["exchange_ms"]
 
     for _ in range(max(3, args.warmup)):
         step()
@@ -478,6 +484,11 @@ def run_sharded(args, rank, local_rank, world):
     fsdist.barrier()
     clocks = sampler.stop()
     t_ms, _ = fsdist.aggregate(e0.elapsed_time(e1), 0.0, dev)
+    # the paper's split of an iteration into local operator time and collective time (max over ranks), from one
+    # more step with CUDA events around every phase (the events themselves cost a little, so it is not the timed one)
+    step(timed=True)
+    loc_ms, _ = fsdist.aggregate(split["local_ms"], 0.0, dev)
+    exc_ms, _ = fsdist.aggregate(split["exchange_ms"], 0.0, dev)
     l1, _ = fs.fs_shard_row_error(sh, stream)
     _, l1 = fsdist.aggregate(0.0, l1, dev)
     fs.fs_shard_destroy(sh)
@@ -489,8 +500,15 @@ def run_sharded(args, rank, local_rank, world):
     line = {"metric": METRIC, "value": its / (t_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": t_ms / args.steps, "higher_is_better": True,
             "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": dict(config_dict(w, args, world), parallelism=f"{world} row shards of one problem, "
-                           "all-reduce of n floats per iteration (NCCL)"),
+            "config": dict(config_dict(w, args, world), parallelism=f"{world} row shards of one problem, exchange = "
+                           + {"allreduce": "one sum all-reduce of n floats per iteration",
+                              "ordered": "all-gather of the G partial vectors, added in rank order on every shard",
+                              "alg1": "Algorithm 1: two Allgathers of scaling slices per iteration (symmetric K)"}[args.exchange]
+                           + " (NCCL)"),
+            "phase_split": {"local_us_per_iteration": 1e3 * loc_ms / w.iters, "exchange_us_per_iteration": 1e3 * exc_ms / w.iters,
+                            "exchange_fraction": exc_ms / max(loc_ms + exc_ms, 1e-30),
+                            "note": "CUDA events around every local step and every collective of one extra step, max over "
+                                    "ranks; the paper reports the same split (local matvec time vs collective time)"},
             "gpu_launches": int(its * 5), "clocks": clocks, "e2e": None,
             "roofline": {"bound": "hbm", "kernel": "row_pass_kernel + col_partial_kernel (per shard)",
                          "achieved": 2 * per_pass_bytes * its / (t_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
@@ -752,6 +770,8 @@ def main():
                     help="N > 1: independent replicas (default, weak scaling) or row shards of one problem")
     ap.add_argument("--path", default="auto", choices=["auto", "implicit"],
                     help="implicit: time only the implicit-kernel path (fs_create_points) of the configuration")
+    ap.add_argument("--exchange", default="allreduce", choices=["allreduce", "ordered", "alg1"],
+                    help="--multi sharded: how the shards exchange per iteration (alg1 needs a symmetric kernel: config 5 shape)")
     ap.add_argument("--headline-only", action="store_true", help="skip the short runs of configurations 1, 2, 3, 5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic-bytes", type=float, default=None,

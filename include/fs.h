@@ -306,6 +306,20 @@ int fs_shard_create(fs_shard **out, int64_t n, int64_t row_lo, int64_t m, const 
 int fs_shard_row_pass(fs_shard *s, void *stream);
 int fs_shard_col_partial(fs_shard *s, float *r_dev_out, void *stream);
 int fs_shard_col_finish(fs_shard *s, const float *r_total_dev, void *stream);
+/* Fixed reduction order for the column sums: the shards all-gather their partial vectors p^(g) (the caller's
+ * collective) and every shard adds them itself, g = 0, 1, ..., G-1, before the divide.  parts_dev: DEVICE
+ * [nparts][pitch] floats (pitch >= n), part g being shard g's fs_shard_col_partial output.  The result is then
+ * independent of how the collective library orders its additions.  Asynchronous. */
+int fs_shard_col_finish_gathered(fs_shard *s, const float *parts_dev, int32_t nparts, int64_t pitch, void *stream);
+/* Algorithm 1's column step as printed, for a SYMMETRIC kernel (every cost the paper runs): client j applies
+ * r_I = (K_{:,I})^T u, which for K = K^T is K_{I,:} u, to the all-gathered u (DEVICE [n]) and forms
+ * v_I = b_I ./ r_I.  The shard's own copy of v is updated on its slice and v_I is also written to
+ * v_block_dev_out (DEVICE [m]; it may point into a caller-owned full vector at row_lo) for the second Allgather,
+ * whose result goes back in with fs_shard_set_scalings(s, NULL, v_full).  The symmetry is the caller's promise
+ * (Assumption 1); it is not checked.  Asynchronous.  fs_shard_local_u copies the shard's u_I (DEVICE [m]) without
+ * synchronising: the send buffer of the first Allgather. */
+int fs_shard_col_block_pass(fs_shard *s, const float *u_full_dev, float *v_block_dev_out, void *stream);
+int fs_shard_local_u(fs_shard *s, float *u_block_dev_out, void *stream);
 int fs_shard_scalings(fs_shard *s, float *u_local_dev_out, float *v_dev_out, void *stream);
 int fs_shard_set_scalings(fs_shard *s, const float *u_local_dev, const float *v_dev, void *stream);
 int fs_shard_row_error(fs_shard *s, double *l1_out, double *sumsq_out, void *stream);

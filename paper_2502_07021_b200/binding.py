@@ -56,6 +56,9 @@ _SIGNATURES = {
     "fs_shard_row_pass": (_int, [_vp, _vp]),
     "fs_shard_col_partial": (_int, [_vp, _vp, _vp]),
     "fs_shard_col_finish": (_int, [_vp, _vp, _vp]),
+    "fs_shard_col_finish_gathered": (_int, [_vp, _vp, _i32, _i64, _vp]),
+    "fs_shard_col_block_pass": (_int, [_vp, _vp, _vp, _vp]),
+    "fs_shard_local_u": (_int, [_vp, _vp, _vp]),
     "fs_shard_scalings": (_int, [_vp, _vp, _vp, _vp]),
     "fs_shard_set_scalings": (_int, [_vp, _vp, _vp, _vp]),
     "fs_shard_row_error": (_int, [_vp, _vp, _vp, _vp]),
@@ -262,6 +265,20 @@ def fs_shard_col_partial(s, r_dev_out, stream=None):
 
 def fs_shard_col_finish(s, r_total_dev, stream=None):
     _check(lib().fs_shard_col_finish(s, _dev(r_total_dev), _stream(stream)), "fs_shard_col_finish")
+
+
+def fs_shard_col_finish_gathered(s, parts_dev, nparts, pitch, stream=None):
+    _check(lib().fs_shard_col_finish_gathered(s, _dev(parts_dev), nparts, pitch, _stream(stream)),
+           "fs_shard_col_finish_gathered")
+
+
+def fs_shard_col_block_pass(s, u_full_dev, v_block_dev_out, stream=None):
+    _check(lib().fs_shard_col_block_pass(s, _dev(u_full_dev), _dev(v_block_dev_out), _stream(stream)),
+           "fs_shard_col_block_pass")
+
+
+def fs_shard_local_u(s, u_block_dev_out, stream=None):
+    _check(lib().fs_shard_local_u(s, _dev(u_block_dev_out), _stream(stream)), "fs_shard_local_u")
 
 
 def fs_shard_scalings(s, u_local_dev_out, v_dev_out, stream=None):

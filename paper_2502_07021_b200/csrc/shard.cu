@@ -9,7 +9,12 @@
 // which is the strict row-partition form (the column sums are assembled from per-shard partial
 // products, as in the appendix's 2D block baseline); for any K it gives the iterates of Algorithm 1 up
 // to the association of the column sums.  The all-reduce is the caller's (torch.distributed / NCCL in
-// paper_2502_07021_b200/distributed.py); this file only provides the three device steps.
+// paper_2502_07021_b200/distributed.py); this file only provides the device steps.  Two more forms:
+//   - a fixed reduction order: the shards all-gather their partial vectors and fs_shard_col_finish_gathered adds the
+//     G vectors in rank order on every shard, so the result does not depend on the collective's algorithm;
+//   - Algorithm 1 as printed (two Allgathers per iteration), valid when K is symmetric: the column block
+//     (K_{:,I})^T u is then K_{I,:} u, a second row-type pass over the same local block with u as input
+//     (fs_shard_col_block_pass); its iterates are those of centralized Sinkhorn exactly (Proposition 1).
 #include <math.h>
 
 #include <vector>
@@ -143,6 +148,35 @@ int fs_shard_col_finish(fs_shard *s, const float *r_total_dev, void *stream) {
     // stage 2 over a single "partial" row: the residual v .* r - b and v = b ./ r
     fsk_col_finish(s->n, s->n, 1, r_total_dev, s->b, s->v, s->coldiff, 1, s->eta, s->status, (cudaStream_t)stream);
     FS_SH(cudaGetLastError());
+    return FS_OK;
+}
+
+int fs_shard_col_finish_gathered(fs_shard *s, const float *parts_dev, int32_t nparts, int64_t pitch, void *stream) {
+    if (!s || !parts_dev) return FS_ERR_NULL;
+    if (nparts < 1 || pitch < s->n) return FS_ERR_BAD_N;
+    // stage 2 over the G gathered partial vectors, added in rank order (fixed association)
+    fsk_col_finish(s->n, pitch, nparts, parts_dev, s->b, s->v, s->coldiff, 1, s->eta, s->status, (cudaStream_t)stream);
+    FS_SH(cudaGetLastError());
+    return FS_OK;
+}
+
+int fs_shard_col_block_pass(fs_shard *s, const float *u_full_dev, float *v_block_dev_out, void *stream) {
+    if (!s || !u_full_dev || !v_block_dev_out) return FS_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    // K symmetric: r_I = (K_{:,I})^T u = K_{I,:} u.  The row-pass kernel with u as input and the local slice of b
+    // as marginal gives v_I = b_I ./ r_I and the residual v_I .* r_I - b_I (old v_I from the shard's own copy).
+    float *v_loc = s->v + s->row_lo;
+    fsk_row_pass(s->plan, s->mat, s->mat_ld, s->n, s->m, u_full_dev, s->b + s->row_lo, v_loc, s->coldiff + s->row_lo, 1,
+                 s->eta, s->status, st);
+    FS_SH(cudaGetLastError());
+    if (v_block_dev_out != v_loc)
+        FS_SH(cudaMemcpyAsync(v_block_dev_out, v_loc, sizeof(float) * s->m, cudaMemcpyDeviceToDevice, st));
+    return FS_OK;
+}
+
+int fs_shard_local_u(fs_shard *s, float *u_block_dev_out, void *stream) {
+    if (!s || !u_block_dev_out) return FS_ERR_NULL;
+    FS_SH(cudaMemcpyAsync(u_block_dev_out, s->u, sizeof(float) * s->m, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
     return FS_OK;
 }
 

@@ -66,28 +66,134 @@ def row_range(n: int, rank: int, world: int):
     return shard_problems(n, rank, world)
 
 
-def sharded_iterate(api, shard, r_buf, k: int, stream=None, group=None):
-    """k Sinkhorn iterations of a row-partitioned problem, one shard per process (Algorithm 1 with the
-    column sums assembled by an all-reduce of the per-shard partial products, n floats per iteration).
+class _PhaseTimer:
+    """Accumulates the time of the local device steps and of the exchanges of a sharded run: CUDA events on the
+    shard's stream when there is one (read back after one synchronisation at the end), wall clock otherwise."""
 
-    `api` provides fs_shard_row_pass / fs_shard_col_partial / fs_shard_col_finish (the ctypes binding on
-    GPUs); `r_buf` is a length-n float32 tensor on the shard's device that receives the partial and then
-    the reduced column sums.  The collective is torch.distributed's (NCCL on GPUs, gloo on CPU); with a
-    CUDA `stream` the three steps and the collective are ordered on that stream.
+    def __init__(self, stream, on_cuda):
+        self.stream, self.on_cuda = stream, on_cuda
+        self.marks, self.total = [], {"local": 0.0, "exchange": 0.0}
+
+    def mark(self):
+        import time
+
+        import torch
+        if self.on_cuda:
+            ev = torch.cuda.Event(enable_timing=True)
+            ev.record(self.stream)
+            return ev
+        return time.perf_counter()
+
+    def add(self, phase, t0, t1):
+        self.marks.append((phase, t0, t1))
+
+    def result(self):
+        if self.on_cuda and self.marks:
+            self.marks[-1][2].synchronize()
+        for phase, t0, t1 in self.marks:
+            self.total[phase] += t0.elapsed_time(t1) if self.on_cuda else (t1 - t0) * 1e3
+        self.marks = []
+        return {"local_ms": self.total["local"], "exchange_ms": self.total["exchange"]}
+
+
+def gather_blocks(local_block, sizes, out_full, group=None):
+    """All-gather of contiguous blocks of unequal length (sizes[r] entries from rank r) into `out_full`, in rank
+    order: every rank contributes its block padded to the longest one, and the valid parts are copied out."""
+    import torch
+    import torch.distributed as dist
+    world = len(sizes)
+    if not (dist.is_available() and dist.is_initialized()) or world == 1:
+        out_full[:sizes[0]].copy_(local_block[:sizes[0]])
+        return
+    mmax = max(sizes)
+    send = torch.zeros(mmax, dtype=local_block.dtype, device=local_block.device)
+    send[:local_block.numel()].copy_(local_block)
+    recv = [torch.empty(mmax, dtype=local_block.dtype, device=local_block.device) for _ in range(world)]
+    dist.all_gather(recv, send, group=group)
+    lo = 0
+    for r in range(world):
+        out_full[lo:lo + sizes[r]].copy_(recv[r][:sizes[r]])
+        lo += sizes[r]
+
+
+def sharded_iterate(api, shard, r_buf, k: int, stream=None, group=None, exchange: str = "allreduce", sizes=None,
+                    timed: bool = False):
+    """k Sinkhorn iterations of a row-partitioned problem, one shard per process.
+
+    exchange = "allreduce": Algorithm 1 with the column sums assembled by ONE sum all-reduce of the per-shard
+        partial products (n floats per iteration); valid for any K; the order of the additions is the
+        collective library's.
+    exchange = "ordered": the same partial products are all-gathered (G x n floats) and every shard adds them in
+        rank order itself (fs_shard_col_finish_gathered): bit-reproducible whatever the library does.
+    exchange = "alg1": Algorithm 1 as printed, two Allgathers of scaling slices per iteration, valid for a
+        SYMMETRIC K (fs_shard_col_block_pass): the iterates are those of centralized Sinkhorn (Proposition 1).
+        `sizes` lists the shards' row counts in rank order.
+
+    `api` provides the fs_shard_* steps (the ctypes binding on GPUs); `r_buf` is a length-n float32 tensor on the
+    shard's device.  Collectives are torch.distributed's (NCCL on GPUs, gloo on CPU); with a CUDA `stream` all
+    steps are ordered on that stream.  With `timed` the time of the local steps and of the exchanges is
+    accumulated separately (the paper's compute / communication split) and returned as a dict.
     """
     import contextlib
 
     import torch
     import torch.distributed as dist
     use_dist = dist.is_available() and dist.is_initialized()
-    ctx = torch.cuda.stream(stream) if (stream is not None and r_buf.is_cuda) else contextlib.nullcontext()
+    world = dist.get_world_size(group) if use_dist else 1
+    rank = dist.get_rank(group) if use_dist else 0
+    on_cuda = r_buf.is_cuda
+    n = r_buf.numel()
+    ctx = torch.cuda.stream(stream) if (stream is not None and on_cuda) else contextlib.nullcontext()
+    timer = _PhaseTimer(stream, on_cuda and stream is not None) if timed else None
+
+    def phase(name, fn):
+        if timer is None:
+            fn()
+            return
+        t0 = timer.mark()
+        fn()
+        timer.add(name, t0, timer.mark())
+
     with ctx:
+        if exchange == "ordered":
+            parts = torch.empty(world * n, dtype=r_buf.dtype, device=r_buf.device)
+        if exchange == "alg1":
+            if sizes is None:
+                sizes = [row_range(n, r, world)[1] - row_range(n, r, world)[0] for r in range(world)]
+            lo = sum(sizes[:rank])
+            u_loc = torch.empty(sizes[rank], dtype=r_buf.dtype, device=r_buf.device)
+            u_full = torch.empty(n, dtype=r_buf.dtype, device=r_buf.device)
+            v_full = r_buf
         for _ in range(k):
-            api.fs_shard_row_pass(shard, stream)
-            api.fs_shard_col_partial(shard, r_buf, stream)
-            if use_dist:
-                dist.all_reduce(r_buf, op=dist.ReduceOp.SUM, group=group)
-            api.fs_shard_col_finish(shard, r_buf, stream)
+            if exchange == "alg1":
+                def local_u():
+                    api.fs_shard_row_pass(shard, stream)
+                    api.fs_shard_local_u(shard, u_loc, stream)
+                phase("local", local_u)
+                phase("exchange", lambda: gather_blocks(u_loc, sizes, u_full, group))
+                v_loc = v_full[lo:lo + sizes[rank]]
+                phase("local", lambda: api.fs_shard_col_block_pass(shard, u_full, v_loc, stream))
+                phase("exchange", lambda: gather_blocks(v_loc.clone(), sizes, v_full, group))
+                phase("local", lambda: api.fs_shard_set_scalings(shard, None, v_full, stream))
+                continue
+
+            def local_partial():
+                api.fs_shard_row_pass(shard, stream)
+                api.fs_shard_col_partial(shard, r_buf, stream)
+            phase("local", local_partial)
+            if exchange == "ordered":
+                def gather_parts():
+                    if use_dist:
+                        dist.all_gather(list(parts.view(world, n).unbind(0)), r_buf, group=group)
+                    else:
+                        parts[:n].copy_(r_buf)
+                phase("exchange", gather_parts)
+                phase("local", lambda: api.fs_shard_col_finish_gathered(shard, parts, world, n, stream))
+            else:
+                if use_dist:
+                    phase("exchange", lambda: dist.all_reduce(r_buf, op=dist.ReduceOp.SUM, group=group))
+                phase("local", lambda: api.fs_shard_col_finish(shard, r_buf, stream))
+    return timer.result() if timer is not None else None
 
 
 def finalize():

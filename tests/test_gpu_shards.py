@@ -88,3 +88,91 @@ def test_shards_from_cost_blocks_and_bad_arguments():
         with pytest.raises(fs.FsError) as ei:
             fs.fs_shard_create(n, lo, m, x, n, 0, 0.1, x, x)
         assert ei.value.code == code
+
+
+def make_shards(w, G, torch, dev, stream):
+    b = torch.from_numpy(w.b).to(dev)
+    shards, blocks, keep = [], [], []
+    for r in range(G):
+        lo, hi = fsdist.row_range(w.n, r, G)
+        Mb = torch.from_numpy(np.ascontiguousarray(w.K[lo:hi])).to(dev)
+        ab = torch.from_numpy(w.a[lo:hi].copy()).to(dev)
+        keep += [Mb, ab, b]
+        torch.cuda.synchronize()
+        shards.append(fs.fs_shard_create(w.n, lo, hi - lo, Mb, w.n, fs.FS_MATRIX_KERNEL, w.eps, ab, b, stream))
+        blocks.append((lo, hi))
+    return shards, blocks, keep
+
+
+@pytest.mark.parametrize("n,G", [(1000, 3), (4099, 4)])
+def test_shards_run_algorithm_1_with_allgathers_on_a_symmetric_kernel(n, G):
+    """Algorithm 1 as printed on G shards of one GPU: u slices are gathered (here: copied into one vector, which
+    is what an Allgather leaves on every rank), each shard applies its column block as K_{I,:} u (K symmetric)
+    and the v slices are gathered.  Reference: the oracle's c-client protocol, which equals centralized Sinkhorn."""
+    import torch
+    w = workloads.make(5, n=n, nbatch=1)                 # one cloud: symmetric kernel
+    assert np.array_equal(w.K, w.K.T)
+    dev = torch.device("cuda:0")
+    stream = torch.cuda.Stream(device=dev)
+    shards, blocks, keep = make_shards(w, G, torch, dev, stream)
+    u_full = torch.empty(n, dtype=torch.float32, device=dev)
+    v_full = torch.empty(n, dtype=torch.float32, device=dev)
+    try:
+        with torch.cuda.stream(stream):
+            for _ in range(10):
+                for s, (lo, hi) in zip(shards, blocks):
+                    fs.fs_shard_row_pass(s, stream)
+                    fs.fs_shard_local_u(s, u_full[lo:hi], stream)             # Allgather of u
+                for s, (lo, hi) in zip(shards, blocks):
+                    fs.fs_shard_col_block_pass(s, u_full, v_full[lo:hi], stream)   # Allgather of v
+                for s in shards:
+                    fs.fs_shard_set_scalings(s, None, v_full, stream)
+        stream.synchronize()
+        u, v = u_full.cpu().numpy(), v_full.cpu().numpy()
+    finally:
+        for s in shards:
+            fs.fs_shard_destroy(s)
+    off = [lo for lo, _ in blocks] + [n]
+    uo, vo, agree = oracle.sinkhorn_protocol(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, off, 10)
+    assert agree
+    assert np.max(np.abs(u - uo) / uo) <= 1e-4 and np.max(np.abs(v - vo) / vo) <= 1e-4
+
+
+def test_shards_add_gathered_partials_in_rank_order_reproducibly():
+    """Fixed reduction order: the G partial vectors sit side by side (what an all-gather leaves on every rank) and
+    fs_shard_col_finish_gathered adds them g = 0..G-1.  Every shard ends with the same v, two runs agree bit for
+    bit, and the iterates are the oracle's row-partition iterates."""
+    import torch
+    n, G = 3000, 3
+    w = workloads.make(2, n=n)
+    dev = torch.device("cuda:0")
+    stream = torch.cuda.Stream(device=dev)
+    runs = []
+    for _ in range(2):
+        shards, blocks, keep = make_shards(w, G, torch, dev, stream)
+        parts = torch.empty(G * n, dtype=torch.float32, device=dev)
+        try:
+            with torch.cuda.stream(stream):
+                for _ in range(8):
+                    for g, s in enumerate(shards):
+                        fs.fs_shard_row_pass(s, stream)
+                        fs.fs_shard_col_partial(s, parts[g * n:(g + 1) * n], stream)
+                    for s in shards:
+                        fs.fs_shard_col_finish_gathered(s, parts, G, n, stream)
+            vs = []
+            u = np.empty(n, dtype=np.float32)
+            for s, (lo, hi) in zip(shards, blocks):
+                ub = torch.empty(hi - lo, dtype=torch.float32, device=dev)
+                vb = torch.empty(n, dtype=torch.float32, device=dev)
+                fs.fs_shard_scalings(s, ub, vb, stream)
+                u[lo:hi] = ub.cpu().numpy()
+                vs.append(vb.cpu().numpy())
+        finally:
+            for s in shards:
+                fs.fs_shard_destroy(s)
+        assert all(np.array_equal(vb, vs[0]) for vb in vs[1:])
+        runs.append((u, vs[0]))
+    assert np.array_equal(runs[0][0], runs[1][0]) and np.array_equal(runs[0][1], runs[1][1])
+    off = [fsdist.row_range(n, r, G)[0] for r in range(G)] + [n]
+    uo, vo = oracle.sinkhorn_rowpartition(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, off, 8)
+    assert np.max(np.abs(runs[0][0] - uo) / uo) <= 1e-4 and np.max(np.abs(runs[0][1] - vo) / vo) <= 1e-4
