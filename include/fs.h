@@ -59,7 +59,8 @@ enum {
     FS_ERR_NONFINITE = -9,            /* an update produced a non-finite or non-positive scaling */
     FS_ERR_UNSUPPORTED = -10,         /* combination not implemented (batched log domain) */
     FS_ERR_TOO_LARGE = -11,           /* size exceeds a fixed capacity (fs_col_pass_static: n > FS_STATIC_MAX_N) */
-    FS_ERR_TIMEOUT = -12              /* a bounded wait inside a kernel ran out; the handle's results are invalid */
+    FS_ERR_TIMEOUT = -12,             /* a bounded wait inside a kernel ran out; the handle's results are invalid */
+    FS_ERR_INTERNAL = -13             /* checked build only: a kernel computed an index outside its buffer */
 };
 
 /* Options for fs_set_option. */
@@ -345,6 +346,18 @@ int fs_selftest_bounded_wait(int32_t poll_limit, int32_t arrive, int32_t *timed_
  * aid; no counterpart in the paper.)
  */
 int fs_selftest_ex2_rate(int32_t iters, double *ex2_per_second, void *stream);
+
+/*
+ * fs_debug_report -- counters of the CHECKED build of this library (python -m paper_2502_07021_b200.build --debug ->
+ * libfs_b200_debug.so, compiled with -DFS_DEBUG), which stands in for a memory-checking tool: every owned device
+ * buffer is followed by 256 canary bytes verified when it is freed, every launcher verifies its geometry and the
+ * extents of its partial-result buffers on the host, and kernels guard the stores into those buffers (an index
+ * outside the buffer is flagged, reported as FS_ERR_INTERNAL by the next result call, and the access is skipped;
+ * nothing traps).  All outputs are HOST and may be NULL: *checked_build is 1 in that build and 0 in the ordinary one
+ * (where the other counters stay 0); canary and launch-check failures counted so far; buffers allocated so far.
+ * (Development aid; no counterpart in the paper.)
+ */
+int fs_debug_report(int32_t *checked_build, int64_t *canary_failures, int64_t *launch_check_failures, int64_t *allocations);
 
 const char *fs_strerror(int code);
 

@@ -18,10 +18,13 @@ FS_OK = 0
 FS_ERR_NULL, FS_ERR_BAD_N, FS_ERR_BAD_OFFSETS, FS_ERR_BAD_EPS = -1, -2, -3, -4
 FS_ERR_NONPOSITIVE_MARGINAL, FS_ERR_MASS_MISMATCH, FS_ERR_DOMAIN = -5, -6, -7
 FS_ERR_CUDA, FS_ERR_NONFINITE, FS_ERR_UNSUPPORTED, FS_ERR_TOO_LARGE, FS_ERR_TIMEOUT = -8, -9, -10, -11, -12
+FS_ERR_INTERNAL = -13
 FS_STATIC_MAX_N = 16384
 FS_OPT_USE_GRAPH, FS_OPT_BATCH_ENGINE, FS_OPT_ROW_SHAPE, FS_OPT_COL_SHAPE, FS_OPT_FUSED, FS_OPT_RESIDENT, FS_OPT_PERSISTENT = 1, 2, 3, 4, 5, 6, 7
 
-LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libfs_b200.so")
+# FS_B200_DEBUG=1 in the environment selects the checked build (canaries, launch checks, guarded stores)
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)),
+                        "libfs_b200_debug.so" if os.environ.get("FS_B200_DEBUG") == "1" else "libfs_b200.so")
 
 _vp = ctypes.c_void_p
 _i64 = ctypes.c_int64
@@ -65,6 +68,7 @@ _SIGNATURES = {
     "fs_shard_destroy": (_int, [_vp]),
     "fs_selftest_bounded_wait": (_int, [_i32, _i32, ctypes.POINTER(_i32), _vp]),
     "fs_selftest_ex2_rate": (_int, [_i32, ctypes.POINTER(_dbl), _vp]),
+    "fs_debug_report": (_int, [ctypes.POINTER(_i32), ctypes.POINTER(_i64), ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
     "fs_strerror": (ctypes.c_char_p, [_int]),
     "fs_last_cuda_error": (ctypes.c_char_p, []),
 }
@@ -330,6 +334,14 @@ def fs_solve_host_points(n, c, row_offsets, X_host, Y_host, d, cost_scale, eps, 
                                       _host_ptr(a_host), _host_ptr(b_host), iters, _host_ptr(u_out), _host_ptr(v_out),
                                       err.ctypes.data_as(_vp) if want_error else None), "fs_solve_host_points")
     return err
+
+
+def fs_debug_report():
+    """dict(checked_build, canary_failures, launch_check_failures, allocations) of the loaded library."""
+    cb, cf, lf, al = _i32(0), _i64(0), _i64(0), _i64(0)
+    _check(lib().fs_debug_report(ctypes.byref(cb), ctypes.byref(cf), ctypes.byref(lf), ctypes.byref(al)), "fs_debug_report")
+    return dict(checked_build=bool(cb.value), canary_failures=cf.value, launch_check_failures=lf.value,
+                allocations=al.value)
 
 
 def fs_selftest_ex2_rate(iters=4096, stream=None):

@@ -1,6 +1,6 @@
 """Build libfs_b200.so in-tree with nvcc for sm_100a (cross-compiles without a GPU).
 
-    python -m paper_2502_07021_b200.build [--force]
+    python -m paper_2502_07021_b200.build [--force] [--debug]
 """
 from __future__ import annotations
 
@@ -27,27 +27,35 @@ def _newest_header() -> float:
     return t
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+DEBUG_LIB = os.path.join(HERE, "libfs_b200_debug.so")
+
+
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Ordinary library, or with debug=True the checked build (-DFS_DEBUG: canaries behind every owned buffer, launch
+    geometry checks, guarded stores) as libfs_b200_debug.so."""
     nvcc = os.environ.get("NVCC", "nvcc")
-    os.makedirs(OBJ_DIR, exist_ok=True)
+    obj_dir = os.path.join(OBJ_DIR, "debug") if debug else OBJ_DIR
+    lib = DEBUG_LIB if debug else LIB
+    flags = NVCC_FLAGS + (["-DFS_DEBUG"] if debug else [])
+    os.makedirs(obj_dir, exist_ok=True)
     hdr = _newest_header()
     objs, rebuilt = [], False
     for src in SOURCES:
         sp = os.path.join(CSRC, src)
-        op = os.path.join(OBJ_DIR, src.replace(".cu", ".o"))
+        op = os.path.join(obj_dir, src.replace(".cu", ".o"))
         objs.append(op)
         if force or not os.path.exists(op) or os.path.getmtime(op) < max(os.path.getmtime(sp), hdr):
-            cmd = [nvcc, *NVCC_FLAGS, "-c", sp, "-o", op]
+            cmd = [nvcc, *flags, "-c", sp, "-o", op]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             subprocess.run(cmd, check=True)
             rebuilt = True
-    if rebuilt or not os.path.exists(LIB):
-        tmp = LIB + f".tmp{os.getpid()}"
+    if rebuilt or not os.path.exists(lib):
+        tmp = lib + f".tmp{os.getpid()}"
         subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp, *objs], check=True)
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

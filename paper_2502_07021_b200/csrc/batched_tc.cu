@@ -556,8 +556,8 @@ bool cluster_fits(int ks, int mtiles, int ntiles) {
 
 void tc_free(TcState *t) {
     if (!t) return;
-    cudaFree(t->K_hi), cudaFree(t->K_lo), cudaFree(t->Kt_hi), cudaFree(t->Kt_lo);
-    cudaFree(t->U_hi), cudaFree(t->U_lo), cudaFree(t->V_hi), cudaFree(t->V_lo);
+    fsk_free(t->K_hi), fsk_free(t->K_lo), fsk_free(t->Kt_hi), fsk_free(t->Kt_lo);
+    fsk_free(t->U_hi), fsk_free(t->U_lo), fsk_free(t->V_hi), fsk_free(t->V_lo);
     delete t;
 }
 
@@ -587,8 +587,8 @@ void *fsk_tc_create(const float *K, int64_t ld, int64_t n, int nbatch, cudaStrea
     bool ok = true;
     __nv_bfloat16 **mats[4] = {&t->K_hi, &t->K_lo, &t->Kt_hi, &t->Kt_lo};
     __nv_bfloat16 **vecs[4] = {&t->U_hi, &t->U_lo, &t->V_hi, &t->V_lo};
-    for (auto m : mats) ok = ok && cudaMalloc(m, mat_bytes) == cudaSuccess && cudaMemsetAsync(*m, 0, mat_bytes, st) == cudaSuccess;
-    for (auto v : vecs) ok = ok && cudaMalloc(v, vec_bytes) == cudaSuccess && cudaMemsetAsync(*v, 0, vec_bytes, st) == cudaSuccess;
+    for (auto m : mats) ok = ok && fsk_malloc(m, mat_bytes) == cudaSuccess && cudaMemsetAsync(*m, 0, mat_bytes, st) == cudaSuccess;
+    for (auto v : vecs) ok = ok && fsk_malloc(v, vec_bytes) == cudaSuccess && cudaMemsetAsync(*v, 0, vec_bytes, st) == cudaSuccess;
     if (ok) {
         dim3 grid((unsigned)((n + 31) / 32), (unsigned)((n + 31) / 32));
         split_matrix_kernel<<<grid, 256, 0, st>>>(K, ld, (int)n, t->kblocks, t->K_hi, t->K_lo, t->Kt_hi, t->Kt_lo);

@@ -64,7 +64,7 @@ std::vector<FsRowTile> build_tiles(const std::vector<int64_t> &off, int h) {
 }
 
 void free_dev(void *p) {
-    if (p) cudaFree(p);
+    if (p) fsk_free(p);
 }
 
 void destroy_graphs(fs_solver *s) {
@@ -111,11 +111,11 @@ int upload_tiles(fs_solver *s) {
     s->tiles_dev = nullptr;
     free_dev(s->partials);
     s->partials = nullptr;
-    FS_CU(cudaMalloc(&s->tiles_dev, sizeof(FsRowTile) * s->tiles.size()));
+    FS_CU(fsk_malloc(&s->tiles_dev, sizeof(FsRowTile) * s->tiles.size()));
     FS_CU(cudaMemcpy(s->tiles_dev, s->tiles.data(), sizeof(FsRowTile) * s->tiles.size(), cudaMemcpyHostToDevice));
     const int planes = s->domain == FS_DOMAIN_LOG ? 2 : 1;
     s->partials_bytes = sizeof(float) * (size_t)planes * s->tiles.size() * (size_t)s->n_pad;
-    FS_CU(cudaMalloc(&s->partials, s->partials_bytes));
+    FS_CU(fsk_malloc(&s->partials, s->partials_bytes));
     return FS_OK;
 }
 
@@ -165,11 +165,12 @@ void enqueue_col(fs_solver *s, int update, cudaStream_t st, int64_t &launches) {
         launches += 1;
     } else if (s->domain == FS_DOMAIN_SCALING) {
         fsk_col_pass(s->plan, s->mat, s->mat_ld, s->n, s->n_pad, s->tiles_dev, (int)s->tiles.size(), s->x, s->b, s->y,
-                     s->partials, s->coldiff, update, s->eta, s->status, st);
+                     s->partials, s->coldiff, update, s->eta, s->status, st, (int64_t)(s->partials_bytes / sizeof(float)));
         launches += fsk_pass_launches_col();
     } else {
         fsk_log_col_pass(s->plan, s->mat, s->mat_ld, s->n, s->n_pad, s->eps, s->tiles_dev, (int)s->tiles.size(), s->xs,
-                         s->b, s->logb, s->y, s->ys, s->partials, s->coldiff, update, s->status, st);
+                         s->b, s->logb, s->y, s->ys, s->partials, s->coldiff, update, s->status, st,
+                         (int64_t)(s->partials_bytes / sizeof(float)));
         launches += fsk_pass_launches_col();
     }
 }
@@ -270,6 +271,7 @@ int check_status(fs_solver *s, cudaStream_t st) {
         FS_CU(cudaStreamSynchronize(st));
         return FS_ERR_TIMEOUT;
     }
+    if (h.oob) return FS_ERR_INTERNAL; // checked build: a kernel computed an index outside its buffer
     if (h.nonfinite) {
         FS_CU(cudaMemsetAsync(&s->status->nonfinite, 0, sizeof(int), st));
         FS_CU(cudaStreamSynchronize(st));
@@ -298,13 +300,13 @@ int set_initial_state(fs_solver *s, cudaStream_t st) {
 // Assumption A2 checked on the device: strictly positive, finite, equal mass per problem.
 int validate_marginals(const float *a_dev, const float *b_dev, int64_t n, int32_t nbatch, cudaStream_t st) {
     double *scan = nullptr;
-    FS_CU(cudaMalloc(&scan, sizeof(double) * 4 * (size_t)nbatch));
+    FS_CU(fsk_malloc(&scan, sizeof(double) * 4 * (size_t)nbatch));
     fsk_min_sum(a_dev, n, nbatch, scan, st);
     fsk_min_sum(b_dev, n, nbatch, scan + 2 * (size_t)nbatch, st);
     std::vector<double> h(4 * (size_t)nbatch);
     cudaError_t e = cudaMemcpyAsync(h.data(), scan, sizeof(double) * h.size(), cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    cudaFree(scan);
+    fsk_free(scan);
     if (e != cudaSuccess) return cuda_fail(e, "marginal validation");
     for (int p = 0; p < nbatch; ++p) {
         const double amin = h[2 * p], asum = h[2 * p + 1];
@@ -334,6 +336,7 @@ const char *fs_strerror(int code) {
     case FS_ERR_UNSUPPORTED: return "combination not supported";
     case FS_ERR_TOO_LARGE: return "size exceeds the fixed capacity of this entry point";
     case FS_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case FS_ERR_INTERNAL: return "checked build: an index outside its buffer was computed (the access was skipped)";
     default: return "unknown error code";
     }
 }
@@ -379,18 +382,18 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
     s->block_err_host.assign(2 * (size_t)c, 0.0);
 
     FS_CU(cudaStreamCreateWithFlags(&s->capture_stream, cudaStreamNonBlocking));
-    FS_CU(cudaMalloc(&s->a, sizeof(float) * cnt));
-    FS_CU(cudaMalloc(&s->b, sizeof(float) * cnt));
-    FS_CU(cudaMalloc(&s->x, sizeof(float) * cnt));
-    FS_CU(cudaMalloc(&s->y, sizeof(float) * cnt));
-    FS_CU(cudaMalloc(&s->rowdiff, sizeof(float) * cnt));
-    FS_CU(cudaMalloc(&s->coldiff, sizeof(float) * cnt));
-    FS_CU(cudaMalloc(&s->offsets_dev, sizeof(int64_t) * (c + 1)));
-    FS_CU(cudaMalloc(&s->block_err, sizeof(double) * 2 * c));
-    FS_CU(cudaMalloc(&s->err_out, sizeof(double) * 4 * nbatch));
-    FS_CU(cudaMalloc(&s->status, sizeof(FsDeviceStatus)));
+    FS_CU(fsk_malloc(&s->a, sizeof(float) * cnt));
+    FS_CU(fsk_malloc(&s->b, sizeof(float) * cnt));
+    FS_CU(fsk_malloc(&s->x, sizeof(float) * cnt));
+    FS_CU(fsk_malloc(&s->y, sizeof(float) * cnt));
+    FS_CU(fsk_malloc(&s->rowdiff, sizeof(float) * cnt));
+    FS_CU(fsk_malloc(&s->coldiff, sizeof(float) * cnt));
+    FS_CU(fsk_malloc(&s->offsets_dev, sizeof(int64_t) * (c + 1)));
+    FS_CU(fsk_malloc(&s->block_err, sizeof(double) * 2 * c));
+    FS_CU(fsk_malloc(&s->err_out, sizeof(double) * 4 * nbatch));
+    FS_CU(fsk_malloc(&s->status, sizeof(FsDeviceStatus)));
     s->trace_cap = kTraceCap;
-    FS_CU(cudaMalloc(&s->trace, sizeof(double) * 2 * s->trace_cap));
+    FS_CU(fsk_malloc(&s->trace, sizeof(double) * 2 * s->trace_cap));
     FS_CU(cudaMemcpyAsync(s->a, a_dev, sizeof(float) * cnt, cudaMemcpyDeviceToDevice, st));
     FS_CU(cudaMemcpyAsync(s->b, b_dev, sizeof(float) * cnt, cudaMemcpyDeviceToDevice, st));
     FS_CU(cudaMemcpyAsync(s->offsets_dev, s->offsets.data(), sizeof(int64_t) * (c + 1), cudaMemcpyHostToDevice, st));
@@ -398,16 +401,16 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
     FS_CU(cudaMemsetAsync(s->coldiff, 0, sizeof(float) * cnt, st));
 
     if (domain == FS_DOMAIN_LOG) {
-        FS_CU(cudaMalloc(&s->loga, sizeof(float) * cnt));
-        FS_CU(cudaMalloc(&s->logb, sizeof(float) * cnt));
-        FS_CU(cudaMalloc(&s->xs, sizeof(float) * cnt));
-        FS_CU(cudaMalloc(&s->ys, sizeof(float) * cnt));
+        FS_CU(fsk_malloc(&s->loga, sizeof(float) * cnt));
+        FS_CU(fsk_malloc(&s->logb, sizeof(float) * cnt));
+        FS_CU(fsk_malloc(&s->xs, sizeof(float) * cnt));
+        FS_CU(fsk_malloc(&s->ys, sizeof(float) * cnt));
         fsk_log(s->a, cnt, s->loga, st);
         fsk_log(s->b, cnt, s->logb, st);
         s->mat = M_dev, s->mat_ld = ld;
     } else if (matrix_kind == FS_MATRIX_COST) {
         // set-up step: materialise the Gibbs kernel once (Section 1, K = exp(-C/eps))
-        FS_CU(cudaMalloc(&s->K_owned, sizeof(float) * (size_t)n * (size_t)s->n_pad));
+        FS_CU(fsk_malloc(&s->K_owned, sizeof(float) * (size_t)n * (size_t)s->n_pad));
         fsk_materialize_kernel(M_dev, ld, n, n, (float)(-1.0 / eps), s->K_owned, s->n_pad, st);
         s->mat = s->K_owned, s->mat_ld = s->n_pad;
     } else {
@@ -423,15 +426,15 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
             const size_t planes = 1;
             const std::vector<FsRowTile> ft = build_tiles(s->offsets, s->fused.tile_rows);
             s->fused_ntiles = (int)ft.size();
-            FS_CU(cudaMalloc(&s->fused_tiles_dev, sizeof(FsRowTile) * ft.size()));
+            FS_CU(fsk_malloc(&s->fused_tiles_dev, sizeof(FsRowTile) * ft.size()));
             FS_CU(cudaMemcpy(s->fused_tiles_dev, ft.data(), sizeof(FsRowTile) * ft.size(), cudaMemcpyHostToDevice));
             const size_t pbytes = sizeof(float) * planes * (size_t)s->fused.nclusters * (size_t)n;
-            FS_CU(cudaMalloc(&s->fused_partials, pbytes));
+            FS_CU(fsk_malloc(&s->fused_partials, pbytes));
             FS_CU(cudaMemsetAsync(s->fused_partials, 0, pbytes, st));
-            if (domain == FS_DOMAIN_SCALING) FS_CU(cudaMalloc(&s->fused_u_prev, sizeof(float) * (size_t)n));
+            if (domain == FS_DOMAIN_SCALING) FS_CU(fsk_malloc(&s->fused_u_prev, sizeof(float) * (size_t)n));
             if (domain == FS_DOMAIN_LOG) {
                 const size_t tbytes = 64; // stage 2's count of finished CTAs
-                FS_CU(cudaMalloc(&s->fused_log_tmp, tbytes));
+                FS_CU(fsk_malloc(&s->fused_log_tmp, tbytes));
                 FS_CU(cudaMemsetAsync(s->fused_log_tmp, 0, tbytes, st));
             }
         }
@@ -439,7 +442,7 @@ int fs_create(fs_solver **out, int64_t n, int32_t c, const int64_t *row_offsets,
     if (domain == FS_DOMAIN_SCALING && nbatch == 1) s->resident = fsk_resident_plan(n);
     if (domain == FS_DOMAIN_SCALING && nbatch == 1 && !s->resident.enabled) {
         s->persistent = fsk_persistent_plan(n, vec);
-        if (s->persistent.enabled) FS_CU(cudaMalloc(&s->persistent_scratch, fsk_persistent_scratch_bytes(s->persistent, n)));
+        if (s->persistent.enabled) FS_CU(fsk_malloc(&s->persistent_scratch, fsk_persistent_scratch_bytes(s->persistent, n)));
     }
     // batched problems: tensor-core engine when the batch is wide enough to fill its 128-problem tiles
     if (nbatch >= kTcMinBatch && n >= kTcMinN) s->tc = fsk_tc_create(s->mat, s->mat_ld, n, nbatch, st);
@@ -489,18 +492,18 @@ int fs_create_points(fs_solver **out, int64_t n, int32_t c, const int64_t *row_o
 
     const size_t vb = sizeof(float) * (size_t)s->vec_pad;
     FS_CU(cudaStreamCreateWithFlags(&s->capture_stream, cudaStreamNonBlocking));
-    FS_CU(cudaMalloc(&s->a, sizeof(float) * n));
-    FS_CU(cudaMalloc(&s->b, sizeof(float) * n));
-    FS_CU(cudaMalloc(&s->x, vb)); // zero beyond n: the pass reads whole 128-column tiles of its input vector
-    FS_CU(cudaMalloc(&s->y, vb));
-    FS_CU(cudaMalloc(&s->rowdiff, sizeof(float) * n));
-    FS_CU(cudaMalloc(&s->coldiff, sizeof(float) * n));
-    FS_CU(cudaMalloc(&s->offsets_dev, sizeof(int64_t) * (c + 1)));
-    FS_CU(cudaMalloc(&s->block_err, sizeof(double) * 2 * c));
-    FS_CU(cudaMalloc(&s->err_out, sizeof(double) * 4));
-    FS_CU(cudaMalloc(&s->status, sizeof(FsDeviceStatus)));
+    FS_CU(fsk_malloc(&s->a, sizeof(float) * n));
+    FS_CU(fsk_malloc(&s->b, sizeof(float) * n));
+    FS_CU(fsk_malloc(&s->x, vb)); // zero beyond n: the pass reads whole 128-column tiles of its input vector
+    FS_CU(fsk_malloc(&s->y, vb));
+    FS_CU(fsk_malloc(&s->rowdiff, sizeof(float) * n));
+    FS_CU(fsk_malloc(&s->coldiff, sizeof(float) * n));
+    FS_CU(fsk_malloc(&s->offsets_dev, sizeof(int64_t) * (c + 1)));
+    FS_CU(fsk_malloc(&s->block_err, sizeof(double) * 2 * c));
+    FS_CU(fsk_malloc(&s->err_out, sizeof(double) * 4));
+    FS_CU(fsk_malloc(&s->status, sizeof(FsDeviceStatus)));
     s->trace_cap = kTraceCap;
-    FS_CU(cudaMalloc(&s->trace, sizeof(double) * 2 * s->trace_cap));
+    FS_CU(fsk_malloc(&s->trace, sizeof(double) * 2 * s->trace_cap));
     FS_CU(cudaMemsetAsync(s->x, 0, vb, st));
     FS_CU(cudaMemsetAsync(s->y, 0, vb, st));
     FS_CU(cudaMemcpyAsync(s->a, a_dev, sizeof(float) * n, cudaMemcpyDeviceToDevice, st));
@@ -766,7 +769,7 @@ int fs_transport_cost(fs_solver *s, const float *C_dev, int64_t ldc, double *cos
         return FS_ERR_BAD_N;
     }
     const size_t cnt = (size_t)s->nbatch * (size_t)s->n;
-    if (!s->cost_scratch) FS_CU(cudaMalloc(&s->cost_scratch, sizeof(double) * (cnt + s->nbatch)));
+    if (!s->cost_scratch) FS_CU(fsk_malloc(&s->cost_scratch, sizeof(double) * (cnt + s->nbatch)));
     double *totals = s->cost_scratch + cnt;
     const bool logd = s->domain == FS_DOMAIN_LOG;
     fsk_transport_cost(s->domain, s->mat, s->mat_ld, C, ldC, s->n, s->nbatch, logd ? s->xs : s->x, logd ? s->ys : s->y,
@@ -852,11 +855,11 @@ int fs_solve_host(int64_t n, int32_t c, const int64_t *row_offsets, const float 
         }                                             \
     } while (0)
     FS_CU2(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
-    FS_CU2(cudaMalloc(&M, sizeof(float) * (size_t)n * (size_t)n));
-    FS_CU2(cudaMalloc(&a, vb));
-    FS_CU2(cudaMalloc(&b, vb));
-    FS_CU2(cudaMalloc(&u, vb));
-    FS_CU2(cudaMalloc(&v, vb));
+    FS_CU2(fsk_malloc(&M, sizeof(float) * (size_t)n * (size_t)n));
+    FS_CU2(fsk_malloc(&a, vb));
+    FS_CU2(fsk_malloc(&b, vb));
+    FS_CU2(fsk_malloc(&u, vb));
+    FS_CU2(fsk_malloc(&v, vb));
     FS_CU2(cudaMemcpy2DAsync(M, sizeof(float) * n, M_host, sizeof(float) * ld, sizeof(float) * n, n,
                              cudaMemcpyHostToDevice, st));
     FS_CU2(cudaMemcpyAsync(a, a_host, vb, cudaMemcpyHostToDevice, st));
@@ -892,12 +895,12 @@ int fs_solve_host_points(int64_t n, int32_t c, const int64_t *row_offsets, const
         if (st) cudaStreamDestroy(st);
     };
     FS_CU2(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
-    FS_CU2(cudaMalloc(&X, pb));
-    FS_CU2(cudaMalloc(&Y, pb));
-    FS_CU2(cudaMalloc(&a, vb));
-    FS_CU2(cudaMalloc(&b, vb));
-    FS_CU2(cudaMalloc(&u, vb));
-    FS_CU2(cudaMalloc(&v, vb));
+    FS_CU2(fsk_malloc(&X, pb));
+    FS_CU2(fsk_malloc(&Y, pb));
+    FS_CU2(fsk_malloc(&a, vb));
+    FS_CU2(fsk_malloc(&b, vb));
+    FS_CU2(fsk_malloc(&u, vb));
+    FS_CU2(fsk_malloc(&v, vb));
     FS_CU2(cudaMemcpyAsync(X, X_host, pb, cudaMemcpyHostToDevice, st));
     FS_CU2(cudaMemcpyAsync(Y, Y_host, pb, cudaMemcpyHostToDevice, st));
     FS_CU2(cudaMemcpyAsync(a, a_host, vb, cudaMemcpyHostToDevice, st));

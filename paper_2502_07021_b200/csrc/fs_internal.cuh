@@ -71,7 +71,39 @@ struct FsDeviceStatus {
     int timeout;     // a bounded device-side wait ran out (tensor-core engine)
     int range;       // fused log iteration: a marginal left the safe fp32 range and its row or column was redone
     int fallbacks;   // number of iterations in which that happened
+    int oob;         // checked build only: a kernel computed an index outside its buffer (the access was skipped)
 };
+
+// ---- device allocations and the checked build ------------------------------------------------
+// Every buffer the library owns comes from fsk_malloc and goes back through fsk_free.  In the ordinary build they
+// are cudaMalloc / cudaFree.  In the checked build (compiled with -DFS_DEBUG: python -m paper_2502_07021_b200.build
+// --debug) each allocation is followed by 256 canary bytes that fsk_free verifies, launchers verify their geometry
+// with FS_HOST_CHECK, and kernels guard their stores with FS_GUARD: an index outside its range raises the status
+// flag `oob` and the access is skipped -- nothing traps.  This stands in for a memory-checking tool.
+cudaError_t fsk_malloc_bytes(void **p, size_t bytes);
+cudaError_t fsk_free(void *p);
+template <typename T>
+inline cudaError_t fsk_malloc(T **p, size_t bytes) { return fsk_malloc_bytes(reinterpret_cast<void **>(p), bytes); }
+void fsk_debug_host_failure(const char *what, const char *file, int line);
+#ifdef FS_DEBUG
+#define FS_HOST_CHECK(cond)                                            \
+    do {                                                               \
+        if (!(cond)) fsk_debug_host_failure(#cond, __FILE__, __LINE__); \
+    } while (0)
+#define FS_GUARD(status, idx, limit)                                   \
+    if ((unsigned long long)(idx) >= (unsigned long long)(limit)) {    \
+        if (status) (status)->oob = 1;                                 \
+    } else
+// extra kernel parameters that only the checked build has: the true extent of the buffer a kernel writes partial
+// results into, and where to flag an index beyond it
+#define FS_DBG_PARAMS , long long dbg_limit, FsDeviceStatus *dbg_status
+#define FS_DBG_ARGS(limit, status) , (long long)(limit), (status)
+#else
+#define FS_HOST_CHECK(cond) ((void)0)
+#define FS_GUARD(status, idx, limit)
+#define FS_DBG_PARAMS
+#define FS_DBG_ARGS(limit, status)
+#endif
 
 struct fs_solver {
     int64_t n = 0, ld = 0;
@@ -147,13 +179,16 @@ struct fs_solver {
 void fsk_row_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t nrows, const float *v,
                   const float *a, float *u, float *rowdiff, int update, float eta, FsDeviceStatus *status,
                   cudaStream_t st);
+// partials_elems: number of floats the partials buffer really holds (checked build: stores beyond it are skipped and
+// flagged in `status`); -1 = not stated.
 void fsk_col_partial_sum(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
-                         int ntiles, const float *u, float *partials, float *r_out, cudaStream_t st);
+                         int ntiles, const float *u, float *partials, float *r_out, cudaStream_t st,
+                         int64_t partials_elems = -1, FsDeviceStatus *status = nullptr);
 FsPassPlan fsk_choose_plan(int64_t n, bool vec, int domain);
 // Column pass, scaling domain, two deterministic stages.
 void fsk_col_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
                   int ntiles, const float *u, const float *b, float *v, float *partials, float *coldiff,
-                  int update, float eta, FsDeviceStatus *status, cudaStream_t st);
+                  int update, float eta, FsDeviceStatus *status, cudaStream_t st, int64_t partials_elems = -1);
 // Log-domain row pass: L_i = LSE_l((g_l - C_il)/eps) streamed once with a running (max, sum).
 // ys = g * log2(e)/eps on input; writes f and xs = f * log2(e)/eps when update.
 void fsk_log_row_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n, double eps, const float *ys,
@@ -162,7 +197,7 @@ void fsk_log_row_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n
 void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n, int64_t n_pad, double eps,
                       const FsRowTile *tiles, int ntiles, const float *xs, const float *b, const float *logb,
                       float *g, float *ys, float *partials, float *coldiff, int update,
-                      FsDeviceStatus *status, cudaStream_t st);
+                      FsDeviceStatus *status, cudaStream_t st, int64_t partials_elems = -1);
 // Stage 2 of the column pass alone: r_l = sum over `ntiles` partial rows of pitch n_pad, residual, divide.
 void fsk_col_finish(int64_t n, int64_t n_pad, int ntiles, const float *partials, const float *b, float *v,
                     float *coldiff, int update, float eta, FsDeviceStatus *status, cudaStream_t st);

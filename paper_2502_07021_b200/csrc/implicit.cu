@@ -148,7 +148,7 @@ __global__ void __launch_bounds__(kImpThreads, 1)
 implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_constant__ CUtensorMap tmR_lo,
                      const __grid_constant__ CUtensorMap tmC_hi, const __grid_constant__ CUtensorMap tmC_lo,
                      const float *__restrict__ vin, float *__restrict__ partial, int64_t pitch, int nrows, int tiles,
-                     int T, int nsplit, int kd, FsDeviceStatus *status) {
+                     int T, int nsplit, int kd, long long partial_elems, FsDeviceStatus *status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bars = base + OFF_BARS;
@@ -297,7 +297,10 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
             bt0 += t1 - t0;
             if (ok) {
                 const int gi = rt * BM + row;
-                if (gi < nrows) partial[(int64_t)(cs * NACC + wg) * pitch + gi] = (acc0 + acc1) + (acc2 + acc3);
+                if (gi < nrows) {
+                    FS_GUARD(status, (int64_t)(cs * NACC + wg) * pitch + gi, partial_elems)
+                    partial[(int64_t)(cs * NACC + wg) * pitch + gi] = (acc0 + acc1) + (acc2 + acc3);
+                }
             }
             __syncwarp();
             if (lane == 0 && ok) mbar_arrive(item_free_epi + 8 * slot);
@@ -343,8 +346,8 @@ bool make_map(CUtensorMap *map, const __nv_bfloat16 *ptr, int64_t rows) {
 
 void implicit_free(ImplicitState *t) {
     if (!t) return;
-    for (auto p : t->buf) cudaFree(p);
-    cudaFree(t->partials);
+    for (auto p : t->buf) fsk_free(p);
+    fsk_free(t->partials);
     delete t;
 }
 
@@ -391,11 +394,11 @@ void *fsk_implicit_create(const float *X, const float *Y, int64_t n, int d, doub
     t->grid = (int)(items < sms ? items : sms);
     const size_t bytes = (size_t)t->n_pad * BK * 2;
     bool ok = true;
-    for (auto &p : t->buf) ok = ok && cudaMalloc(&p, bytes) == cudaSuccess && cudaMemsetAsync(p, 0, bytes, st) == cudaSuccess;
-    ok = ok && cudaMalloc(&t->partials, sizeof(float) * (size_t)t->nsplit * NACC * t->n_pad) == cudaSuccess;
+    for (auto &p : t->buf) ok = ok && fsk_malloc(&p, bytes) == cudaSuccess && cudaMemsetAsync(p, 0, bytes, st) == cudaSuccess;
+    ok = ok && fsk_malloc(&t->partials, sizeof(float) * (size_t)t->nsplit * NACC * t->n_pad) == cudaSuccess;
     double *mu = nullptr;
     unsigned int *maxsq = nullptr;
-    ok = ok && cudaMalloc(&mu, sizeof(double) * d) == cudaSuccess && cudaMalloc(&maxsq, 2 * sizeof(unsigned int)) == cudaSuccess &&
+    ok = ok && fsk_malloc(&mu, sizeof(double) * d) == cudaSuccess && fsk_malloc(&maxsq, 2 * sizeof(unsigned int)) == cudaSuccess &&
          cudaMemsetAsync(maxsq, 0, 2 * sizeof(unsigned int), st) == cudaSuccess;
     float hmax[2] = {0.f, 0.f};
     if (ok) {
@@ -408,7 +411,7 @@ void *fsk_implicit_create(const float *X, const float *Y, int64_t n, int d, doub
              cudaMemcpyAsync(hmax, maxsq, 2 * sizeof(float), cudaMemcpyDeviceToHost, st) == cudaSuccess &&
              cudaStreamSynchronize(st) == cudaSuccess;
     }
-    cudaFree(mu), cudaFree(maxsq);
+    fsk_free(mu), fsk_free(maxsq);
     for (int i = 0; i < 8 && ok; ++i) ok = make_map(&t->map[i], t->buf[i], t->n_pad);
     ok = ok && cudaFuncSetAttribute(implicit_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
     if (!ok) {
@@ -436,11 +439,13 @@ float *fsk_implicit_partials(void *h) { return static_cast<ImplicitState *>(h)->
 cudaError_t fsk_implicit_pass(void *h, int transposed, const float *in, FsDeviceStatus *status, cudaStream_t st) {
     ImplicitState *t = static_cast<ImplicitState *>(h);
     const int r = transposed ? 4 : 0, c = transposed ? 2 : 6; // row-side arrays of one cloud, column-side of the other
+    FS_HOST_CHECK(t->grid >= 1 && t->T >= 1 && t->T <= MAX_T && (int64_t)t->T * t->nsplit >= t->tiles &&
+                  t->tiles * (int64_t)BM == t->n_pad && t->kd >= 1 && t->kd <= BK / 16);
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)t->grid);
     cfg.blockDim = dim3(kImpThreads);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = st;
     return cudaLaunchKernelEx(&cfg, implicit_pass_kernel, t->map[r], t->map[r + 1], t->map[c], t->map[c + 1], in, t->partials,
-                              t->n_pad, (int)t->n, t->tiles, t->T, t->nsplit, t->kd, status);
+                              t->n_pad, (int)t->n, t->tiles, t->T, t->nsplit, t->kd, (long long)t->nsplit * NACC * t->n_pad, status);
 }

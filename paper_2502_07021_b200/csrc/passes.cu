@@ -285,7 +285,7 @@ __device__ __forceinline__ float4 ld_cols(const float *p, int valid) {
 template <int TX, int TY, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 col_partial_kernel(const float *__restrict__ K, int64_t ld, int n, int64_t n_pad, const FsRowTile *__restrict__ tiles,
-                   int nstrips, const float *__restrict__ u, float *__restrict__ partials) {
+                   int nstrips, const float *__restrict__ u, float *__restrict__ partials FS_DBG_PARAMS) {
     static_assert(TX * TY == kThreads, "CTA shape");
     constexpr int U = 8;
     __shared__ float u_s[kMaxTileRows];
@@ -336,8 +336,10 @@ col_partial_kernel(const float *__restrict__ K, int64_t ld, int n, int64_t n_pad
             }
         }
     }
-    if (ty == 0 && valid > 0)
+    if (ty == 0 && valid > 0) {
+        FS_GUARD(dbg_status, (int64_t)tile_idx * n_pad + col + 3, dbg_limit)
         *reinterpret_cast<float4 *>(partials + (int64_t)tile_idx * n_pad + col) = acc;
+    }
 }
 
 // Sum of the tile partials of the CTA's 32 columns: thread (c, k) of 32 x 8 adds the tiles k, k + 8, ... of
@@ -396,7 +398,7 @@ template <int TX, int TY, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 log_col_partial_kernel(const float *__restrict__ C, int64_t ld, int n, int64_t n_pad, float s2,
                        const FsRowTile *__restrict__ tiles, int ntiles, int nstrips, const float *__restrict__ xs,
-                       float *__restrict__ partials) {
+                       float *__restrict__ partials FS_DBG_PARAMS) {
     static_assert(TX * TY == kThreads, "CTA shape");
     constexpr int U = 8;
     __shared__ float x_s[kMaxTileRows];
@@ -469,8 +471,10 @@ log_col_partial_kernel(const float *__restrict__ C, int64_t ld, int n, int64_t n
         }
     }
     if (ty == 0 && valid > 0) {
-        *reinterpret_cast<float4 *>(partials + (int64_t)tile_idx * n_pad + col) = m4;
-        *reinterpret_cast<float4 *>(partials + ((int64_t)ntiles + tile_idx) * n_pad + col) = s4;
+        FS_GUARD(dbg_status, ((int64_t)ntiles + tile_idx) * n_pad + col + 3, dbg_limit) {
+            *reinterpret_cast<float4 *>(partials + (int64_t)tile_idx * n_pad + col) = m4;
+            *reinterpret_cast<float4 *>(partials + ((int64_t)ntiles + tile_idx) * n_pad + col) = s4;
+        }
     }
 }
 
@@ -539,13 +543,17 @@ log_col_finish_kernel(int n, int64_t n_pad, int ntiles, float s2, double eps, co
 void fsk_row_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t nrows, const float *v,
                   const float *a, float *u, float *rowdiff, int update, float eta, FsDeviceStatus *status,
                   cudaStream_t st) {
+    FS_HOST_CHECK(n >= 1 && nrows >= 1 && ld >= n && (!p.vec || ((ld & 3) == 0 && (reinterpret_cast<uintptr_t>(K) & 15) == 0)));
     FS_ROW_DISPATCH(row_pass_kernel, K, ld, (int)n, (int)nrows, v, a, u, rowdiff, update, eta, status);
 }
 
 void fsk_col_pass(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
                   int ntiles, const float *u, const float *b, float *v, float *partials, float *coldiff,
-                  int update, float eta, FsDeviceStatus *status, cudaStream_t st) {
-    FS_COL_DISPATCH(col_partial_kernel, K, ld, (int)n, n_pad, tiles, nstrips, u, partials);
+                  int update, float eta, FsDeviceStatus *status, cudaStream_t st, int64_t partials_elems) {
+    const long long plimit = partials_elems >= 0 ? partials_elems : (long long)ntiles * n_pad;
+    FS_HOST_CHECK(ntiles >= 1 && n_pad >= n && (n_pad & 3) == 0 && plimit >= (long long)ntiles * n_pad);
+    (void)plimit;
+    FS_COL_DISPATCH(col_partial_kernel, K, ld, (int)n, n_pad, tiles, nstrips, u, partials FS_DBG_ARGS(plimit, status));
     col_finish_kernel<<<(unsigned)((n + 31) / 32), kThreads, 0, st>>>(
         (int)n, n_pad, ntiles, partials, b, v, coldiff, update, eta, status);
 }
@@ -561,9 +569,12 @@ void fsk_log_row_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n
 void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n, int64_t n_pad, double eps,
                       const FsRowTile *tiles, int ntiles, const float *xs, const float *b, const float *logb,
                       float *g, float *ys, float *partials, float *coldiff, int update,
-                      FsDeviceStatus *status, cudaStream_t st) {
+                      FsDeviceStatus *status, cudaStream_t st, int64_t partials_elems) {
     const float s2 = (float)(1.4426950408889634 / eps);
-    FS_COL_DISPATCH(log_col_partial_kernel, C, ld, (int)n, n_pad, s2, tiles, ntiles, nstrips, xs, partials);
+    const long long plimit = partials_elems >= 0 ? partials_elems : 2LL * ntiles * n_pad;
+    FS_HOST_CHECK(ntiles >= 1 && n_pad >= n && (n_pad & 3) == 0 && plimit >= 2LL * ntiles * n_pad);
+    (void)plimit;
+    FS_COL_DISPATCH(log_col_partial_kernel, C, ld, (int)n, n_pad, s2, tiles, ntiles, nstrips, xs, partials FS_DBG_ARGS(plimit, status));
     log_col_finish_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, st>>>(
         (int)n, n_pad, ntiles, s2, eps, partials, b, logb, g, ys, coldiff, update, status);
 }
@@ -571,8 +582,13 @@ void fsk_log_col_pass(const FsPassPlan &p, const float *C, int64_t ld, int64_t n
 // Stage 1 followed by a plain sum of the tile partials: r_out[l] = sum over the given row tiles of
 // K_il u_i, without the divide (the shard's contribution to K^T u).
 void fsk_col_partial_sum(const FsPassPlan &p, const float *K, int64_t ld, int64_t n, int64_t n_pad, const FsRowTile *tiles,
-                         int ntiles, const float *u, float *partials, float *r_out, cudaStream_t st) {
-    FS_COL_DISPATCH(col_partial_kernel, K, ld, (int)n, n_pad, tiles, nstrips, u, partials);
+                         int ntiles, const float *u, float *partials, float *r_out, cudaStream_t st,
+                         int64_t partials_elems, FsDeviceStatus *status) {
+    const long long plimit = partials_elems >= 0 ? partials_elems : (long long)ntiles * n_pad;
+    FS_HOST_CHECK(ntiles >= 1 && n_pad >= n && (n_pad & 3) == 0 && plimit >= (long long)ntiles * n_pad);
+    (void)plimit;
+    (void)status;
+    FS_COL_DISPATCH(col_partial_kernel, K, ld, (int)n, n_pad, tiles, nstrips, u, partials FS_DBG_ARGS(plimit, status));
     sum_partials_kernel<<<(unsigned)((n + 31) / 32), kThreads, 0, st>>>((int)n, n_pad, ntiles, partials, r_out);
 }
 

@@ -242,18 +242,98 @@ void fsk_transport_cost(int domain, const float *mat, int64_t ld, const float *C
     sum_rows_kernel<<<nbatch, kThreads, 0, st>>>(rowsum_scratch, n, cost_dev);
 }
 
+// ---- allocations, canaries, checked-build counters ---------------------------------------------
+#ifdef FS_DEBUG
+#include <stdio.h>
+
+#include <mutex>
+#include <unordered_map>
+namespace {
+constexpr size_t kCanaryBytes = 256;
+constexpr unsigned char kCanaryByte = 0xC5;
+std::mutex g_dbg_mutex;
+std::unordered_map<void *, size_t> g_dbg_sizes; // allocation -> offset of its canary
+long long g_dbg_canary_failures = 0, g_dbg_host_failures = 0, g_dbg_allocations = 0;
+} // namespace
+
+cudaError_t fsk_malloc_bytes(void **p, size_t bytes) {
+    const size_t body = (bytes + 255) & ~size_t(255); // the canary starts on a 256-byte boundary after the buffer
+    cudaError_t e = cudaMalloc(p, body + kCanaryBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaMemset(static_cast<unsigned char *>(*p) + bytes, kCanaryByte, body - bytes + kCanaryBytes);
+    std::lock_guard<std::mutex> lock(g_dbg_mutex);
+    g_dbg_sizes[*p] = bytes;
+    ++g_dbg_allocations;
+    return e;
+}
+
+cudaError_t fsk_free(void *p) {
+    if (!p) return cudaSuccess;
+    size_t bytes = 0;
+    bool known = false;
+    {
+        std::lock_guard<std::mutex> lock(g_dbg_mutex);
+        auto it = g_dbg_sizes.find(p);
+        if (it != g_dbg_sizes.end()) known = true, bytes = it->second, g_dbg_sizes.erase(it);
+    }
+    if (known) {
+        const size_t body = (bytes + 255) & ~size_t(255), len = body - bytes + kCanaryBytes;
+        std::vector<unsigned char> h(len);
+        cudaDeviceSynchronize();
+        if (cudaMemcpy(h.data(), static_cast<unsigned char *>(p) + bytes, len, cudaMemcpyDeviceToHost) == cudaSuccess) {
+            for (size_t i = 0; i < len; ++i)
+                if (h[i] != kCanaryByte) {
+                    std::lock_guard<std::mutex> lock(g_dbg_mutex);
+                    ++g_dbg_canary_failures;
+                    fprintf(stderr, "fs debug: canary after a %zu-byte buffer overwritten at +%zu\n", bytes, i);
+                    break;
+                }
+        }
+    }
+    return cudaFree(p);
+}
+
+void fsk_debug_host_failure(const char *what, const char *file, int line) {
+    std::lock_guard<std::mutex> lock(g_dbg_mutex);
+    ++g_dbg_host_failures;
+    fprintf(stderr, "fs debug: launch check failed: %s (%s:%d)\n", what, file, line);
+}
+
+extern "C" int fs_debug_report(int32_t *checked_build, int64_t *canary_failures, int64_t *launch_check_failures,
+                               int64_t *allocations) {
+    std::lock_guard<std::mutex> lock(g_dbg_mutex);
+    if (checked_build) *checked_build = 1;
+    if (canary_failures) *canary_failures = g_dbg_canary_failures;
+    if (launch_check_failures) *launch_check_failures = g_dbg_host_failures;
+    if (allocations) *allocations = g_dbg_allocations;
+    return FS_OK;
+}
+#else
+cudaError_t fsk_malloc_bytes(void **p, size_t bytes) { return cudaMalloc(p, bytes); }
+cudaError_t fsk_free(void *p) { return cudaFree(p); }
+void fsk_debug_host_failure(const char *, const char *, int) {}
+extern "C" int fs_debug_report(int32_t *checked_build, int64_t *canary_failures, int64_t *launch_check_failures,
+                               int64_t *allocations) {
+    if (checked_build) *checked_build = 0;
+    if (canary_failures) *canary_failures = 0;
+    if (launch_check_failures) *launch_check_failures = 0;
+    if (allocations) *allocations = 0;
+    return FS_OK;
+}
+#endif
+
 extern "C" int fs_selftest_bounded_wait(int32_t poll_limit, int32_t arrive, int32_t *timed_out, void *stream) {
     if (!timed_out) return FS_ERR_NULL;
     if (poll_limit < 1 || poll_limit > (1 << 20)) return FS_ERR_BAD_N;
     cudaStream_t st = (cudaStream_t)stream;
     int *flag = nullptr;
-    if (cudaMalloc(&flag, sizeof(int)) != cudaSuccess) return FS_ERR_CUDA;
+    if (fsk_malloc(&flag, sizeof(int)) != cudaSuccess) return FS_ERR_CUDA;
     cudaMemsetAsync(flag, 0xff, sizeof(int), st);
     bounded_wait_probe_kernel<<<1, 64, 0, st>>>((uint32_t)poll_limit, arrive, flag);
     int h = -1;
     cudaError_t e = cudaMemcpyAsync(&h, flag, sizeof(int), cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    cudaFree(flag);
+    fsk_free(flag);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return FS_ERR_CUDA;
@@ -272,7 +352,7 @@ extern "C" int fs_selftest_ex2_rate(int32_t iters, double *ex2_per_second, void 
     const int blocks = sms * 8; // 2048 threads per SM: every scheduler has warps to issue from
     float *out = nullptr;
     cudaEvent_t e0 = nullptr, e1 = nullptr;
-    cudaError_t e = cudaMalloc(&out, sizeof(float) * 256 * (size_t)blocks);
+    cudaError_t e = fsk_malloc(&out, sizeof(float) * 256 * (size_t)blocks);
     if (e == cudaSuccess) e = cudaEventCreate(&e0);
     if (e == cudaSuccess) e = cudaEventCreate(&e1);
     float ms = 0.f;
@@ -286,7 +366,7 @@ extern "C" int fs_selftest_ex2_rate(int32_t iters, double *ex2_per_second, void 
     }
     if (e0) cudaEventDestroy(e0);
     if (e1) cudaEventDestroy(e1);
-    cudaFree(out);
+    fsk_free(out);
     if (e != cudaSuccess || !(ms > 0.f)) {
         cudaGetLastError();
         return FS_ERR_CUDA;

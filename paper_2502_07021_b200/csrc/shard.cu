@@ -50,8 +50,8 @@ namespace {
 
 void shard_free(fs_shard *s) {
     if (!s) return;
-    cudaFree(s->K_owned), cudaFree(s->a), cudaFree(s->b), cudaFree(s->u), cudaFree(s->v), cudaFree(s->rowdiff);
-    cudaFree(s->coldiff), cudaFree(s->partials), cudaFree(s->tiles_dev), cudaFree(s->err_dev), cudaFree(s->status);
+    fsk_free(s->K_owned), fsk_free(s->a), fsk_free(s->b), fsk_free(s->u), fsk_free(s->v), fsk_free(s->rowdiff);
+    fsk_free(s->coldiff), fsk_free(s->partials), fsk_free(s->tiles_dev), fsk_free(s->err_dev), fsk_free(s->status);
     delete s;
 }
 
@@ -72,13 +72,13 @@ int fs_shard_create(fs_shard **out, int64_t n, int64_t row_lo, int64_t m, const 
     // positivity of the local marginals (the equal-mass condition spans all shards and is the caller's)
     {
         double *scan = nullptr;
-        FS_SH(cudaMalloc(&scan, sizeof(double) * 4));
+        FS_SH(fsk_malloc(&scan, sizeof(double) * 4));
         fsk_min_sum(a_local_dev, m, 1, scan, st);
         fsk_min_sum(b_dev, n, 1, scan + 2, st);
         double h[4];
         cudaError_t e = cudaMemcpyAsync(h, scan, sizeof(h), cudaMemcpyDeviceToHost, st);
         if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-        cudaFree(scan);
+        fsk_free(scan);
         if (e != cudaSuccess) return FS_ERR_CUDA;
         if (!(h[0] > 0.0) || !(h[2] > 0.0) || !isfinite(h[1]) || !isfinite(h[3])) return FS_ERR_NONPOSITIVE_MARGINAL;
     }
@@ -90,14 +90,14 @@ int fs_shard_create(fs_shard **out, int64_t n, int64_t row_lo, int64_t m, const 
     } guard{s};
     s->n = n, s->m = m, s->row_lo = row_lo, s->ld = ld, s->eps = eps;
     s->n_pad = (n + 3) & ~int64_t(3);
-    FS_SH(cudaMalloc(&s->a, sizeof(float) * m));
-    FS_SH(cudaMalloc(&s->u, sizeof(float) * m));
-    FS_SH(cudaMalloc(&s->rowdiff, sizeof(float) * m));
-    FS_SH(cudaMalloc(&s->b, sizeof(float) * n));
-    FS_SH(cudaMalloc(&s->v, sizeof(float) * n));
-    FS_SH(cudaMalloc(&s->coldiff, sizeof(float) * n));
-    FS_SH(cudaMalloc(&s->err_dev, sizeof(double) * 2));
-    FS_SH(cudaMalloc(&s->status, sizeof(FsDeviceStatus)));
+    FS_SH(fsk_malloc(&s->a, sizeof(float) * m));
+    FS_SH(fsk_malloc(&s->u, sizeof(float) * m));
+    FS_SH(fsk_malloc(&s->rowdiff, sizeof(float) * m));
+    FS_SH(fsk_malloc(&s->b, sizeof(float) * n));
+    FS_SH(fsk_malloc(&s->v, sizeof(float) * n));
+    FS_SH(fsk_malloc(&s->coldiff, sizeof(float) * n));
+    FS_SH(fsk_malloc(&s->err_dev, sizeof(double) * 2));
+    FS_SH(fsk_malloc(&s->status, sizeof(FsDeviceStatus)));
     FS_SH(cudaMemsetAsync(s->status, 0, sizeof(FsDeviceStatus), st));
     FS_SH(cudaMemsetAsync(s->rowdiff, 0, sizeof(float) * m, st));
     FS_SH(cudaMemcpyAsync(s->a, a_local_dev, sizeof(float) * m, cudaMemcpyDeviceToDevice, st));
@@ -105,7 +105,7 @@ int fs_shard_create(fs_shard **out, int64_t n, int64_t row_lo, int64_t m, const 
     fsk_fill(s->u, m, 1.f, st);
     fsk_fill(s->v, n, 1.f, st);
     if (matrix_kind == FS_MATRIX_COST) {
-        FS_SH(cudaMalloc(&s->K_owned, sizeof(float) * (size_t)m * (size_t)s->n_pad));
+        FS_SH(fsk_malloc(&s->K_owned, sizeof(float) * (size_t)m * (size_t)s->n_pad));
         fsk_materialize_kernel(M_dev, ld, n, m, (float)(-1.0 / eps), s->K_owned, s->n_pad, st);
         s->mat = s->K_owned, s->mat_ld = s->n_pad;
     } else {
@@ -117,9 +117,9 @@ int fs_shard_create(fs_shard **out, int64_t n, int64_t row_lo, int64_t m, const 
     for (int64_t r = 0; r < m; r += s->plan.col_tile_rows)
         tiles.push_back(FsRowTile{(int32_t)r, (int32_t)(r + s->plan.col_tile_rows < m ? r + s->plan.col_tile_rows : m)});
     s->ntiles = (int)tiles.size();
-    FS_SH(cudaMalloc(&s->tiles_dev, sizeof(FsRowTile) * tiles.size()));
+    FS_SH(fsk_malloc(&s->tiles_dev, sizeof(FsRowTile) * tiles.size()));
     FS_SH(cudaMemcpyAsync(s->tiles_dev, tiles.data(), sizeof(FsRowTile) * tiles.size(), cudaMemcpyHostToDevice, st));
-    FS_SH(cudaMalloc(&s->partials, sizeof(float) * tiles.size() * (size_t)s->n_pad));
+    FS_SH(fsk_malloc(&s->partials, sizeof(float) * tiles.size() * (size_t)s->n_pad));
     FS_SH(cudaStreamSynchronize(st));
     FS_SH(cudaGetLastError());
     guard.s = nullptr;
@@ -138,7 +138,7 @@ int fs_shard_row_pass(fs_shard *s, void *stream) {
 int fs_shard_col_partial(fs_shard *s, float *r_dev_out, void *stream) {
     if (!s || !r_dev_out) return FS_ERR_NULL;
     fsk_col_partial_sum(s->plan, s->mat, s->mat_ld, s->n, s->n_pad, s->tiles_dev, s->ntiles, s->u, s->partials, r_dev_out,
-                        (cudaStream_t)stream);
+                        (cudaStream_t)stream, (int64_t)s->ntiles * s->n_pad, s->status);
     FS_SH(cudaGetLastError());
     return FS_OK;
 }

@@ -35,11 +35,11 @@ def test_every_declared_symbol_is_exported_and_bound(lib):
 
 def test_strerror_covers_all_codes(lib):
     seen = set()
-    for code in range(0, -13, -1):
+    for code in range(0, -14, -1):
         msg = lib.fs_strerror(code).decode()
         assert msg and msg != "unknown error code"
         seen.add(msg)
-    assert len(seen) == 13
+    assert len(seen) == 14
     assert lib.fs_strerror(-99).decode() == "unknown error code"
 
 
@@ -88,6 +88,20 @@ def test_host_side_validation_needs_no_device(lib):
     assert lib.fs_iterate(None, 1, None) == fs.FS_ERR_NULL
     assert lib.fs_destroy(None) == fs.FS_ERR_NULL
     assert lib.fs_iterations_done(None) == -1
+
+
+def test_checked_build_exports_the_same_interface_and_identifies_itself(lib):
+    """The checked build (-DFS_DEBUG: canaries, launch checks, guarded stores) is a second library with the same
+    C ABI; fs_debug_report tells the two apart without touching a device."""
+    path = fs_build.build(debug=True)
+    dbg = ctypes.CDLL(path)
+    for name in declared_functions():
+        assert hasattr(dbg, name), name
+    for handle, expect in ((dbg, 1), (lib, 0)):
+        flag = ctypes.c_int32(-1)
+        fails = ctypes.c_int64(-1)
+        assert handle.fs_debug_report(ctypes.byref(flag), ctypes.byref(fails), None, None) == fs.FS_OK
+        assert flag.value == expect and fails.value == 0
 
 
 def test_binding_refuses_missing_library(monkeypatch, tmp_path):
