@@ -52,8 +52,11 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (kernel name, n) -> bytes; a capture at n = 16384 is scaled by 4 for n = 32768 (traffic is proportional to n*n).
 TRAFFIC_BYTES_PER_LAUNCH = {
-    ("fused_iteration_kernel", 16384): 1.074000e9 + 3.67e6,
-    ("fused_iteration_kernel", 32768): 4 * (1.074000e9 + 3.67e6),
+    ("fused_iteration_kernel", 16384): 1.074029e9 + 1.96e6,
+    ("fused_iteration_kernel", 32768): 4 * (1.074029e9 + 1.96e6),
+    # the implicit pass reads only the operands of the two clouds from DRAM (n*d-sized, not n*n): captured at n = 16384
+    ("implicit_pass_kernel", 16384): 8.51e6,
+    ("implicit_pass_kernel", 32768): 2 * 8.51e6,
     ("log_row_pass_kernel", 16384): 1.074043e9 + 3.39e6,
     ("fused_log_iteration_kernel", 16384): 1.073997e9 + 4.36e6,
     ("batched_tc_kernel", 8192): 281.10e6 + 3.51e6,
@@ -407,7 +410,8 @@ def time_implicit(fs, torch, dev, stream, w, devidx, args, wp=None):
                         "nominal_peak_source": "16 ex2 per clock per SM x SM count x the median SM clock sampled in the "
                                                "timed region",
                         "frac_of_nominal": achieved / nominal,
-                        "algorithmic_ex2_per_launch": n2, "us_per_launch": pass_s * 1e6, "traffic": None}}
+                        "algorithmic_ex2_per_launch": n2, "us_per_launch": pass_s * 1e6,
+                        "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(("implicit_pass_kernel", wp.n))}}
     with_clock(out, ms * 1e-3 / its, clocks, "sm_cycles_per_iteration")
     if not args.no_e2e:
         pin = [torch.from_numpy(x).pin_memory() for x in (wp.X, wp.Y, wp.a, wp.b)]
