@@ -241,7 +241,8 @@ int fs_solve_host(int64_t n, int32_t c, const int64_t *row_offsets, const float 
  *   n, c, row_offsets, eps, a_dev, b_dev, stream   as for fs_create; one problem, scaling domain.
  *
  * The handle works with fs_iterate, fs_row_pass, fs_col_pass, fs_marginal_error, fs_scalings, fs_set_scalings,
- * fs_reset, fs_set_damping, the error trace and fs_block_errors; fs_transport_cost returns FS_ERR_UNSUPPORTED.
+ * fs_reset, fs_set_damping, the error trace, fs_block_errors and fs_transport_cost (which then ignores C_dev: the cost
+ * is cost_scale |x_i - y_l|^2 of the clouds themselves, accumulated by one more sweep of the implicit pass).
  * Memory is O(n d): nothing of size n^2 exists.  The squared distance is formed as a tensor-core contraction of
  * the translated, scaled points split into two bf16 terms each; the exponent -c|x - y|^2 log2(e)/eps then carries
  * an absolute error of at most about 2^-16 * max|z_x| * max|z_y| (z = sqrt(2 cost_scale log2(e) / eps) times the

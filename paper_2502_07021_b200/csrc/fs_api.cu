@@ -758,8 +758,19 @@ int fs_reset(fs_solver *s, void *stream) {
 
 int fs_transport_cost(fs_solver *s, const float *C_dev, int64_t ldc, double *cost_out, void *stream) {
     if (!s || !cost_out) return FS_ERR_NULL;
-    if (s->implicit) return FS_ERR_UNSUPPORTED; // no stored kernel to form P from
     cudaStream_t st = (cudaStream_t)stream;
+    if (s->implicit) {
+        // the cost is that of the point clouds the handle was created from (C_dev is ignored): one more sweep of the
+        // implicit pass accumulates K_il v_l C_il per row
+        if (!s->cost_scratch) FS_CU(fsk_malloc(&s->cost_scratch, sizeof(double) * ((size_t)s->n + 1)));
+        FS_CU(fsk_implicit_cost_rows(s->implicit, s->x, s->y, s->eps, s->cost_scratch, s->status, st));
+        fsk_sum_rows(s->cost_scratch, s->n, 1, s->cost_scratch + s->n, st);
+        s->launches += 3;
+        FS_CU(cudaGetLastError());
+        FS_CU(cudaMemcpyAsync(cost_out, s->cost_scratch + s->n, sizeof(double), cudaMemcpyDeviceToHost, st));
+        FS_CU(cudaStreamSynchronize(st));
+        return FS_OK;
+    }
     const float *C = C_dev;
     int64_t ldC = ldc;
     if (!C) {

@@ -260,6 +260,11 @@ int fsk_implicit_max_dim();
 int fsk_implicit_nsplit(const void *h);   // number of partial rows a pass writes
 float *fsk_implicit_partials(void *h);    // [partial rows][padded n] partial sums written by a pass
 cudaError_t fsk_implicit_pass(void *h, int transposed, const float *in, FsDeviceStatus *status, cudaStream_t st);
+// rowsum[i] = u_i sum_l K_il v_l C_il (n doubles); add them for <P,C>
+cudaError_t fsk_implicit_cost_rows(void *h, const float *u, const float *v, double eps, double *rowsum, FsDeviceStatus *status,
+                                   cudaStream_t st);
+// out[b] = sum of rowsum[b][0..n) in a fixed order (double)
+void fsk_sum_rows(const double *rowsum, int64_t n, int nbatch, double *out, cudaStream_t st);
 
 // ---- setup.cu ----------------------------------------------------------------------------
 // C and K are nrows x n.

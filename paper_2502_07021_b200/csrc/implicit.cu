@@ -125,6 +125,7 @@ prepare_points_kernel(const float *__restrict__ P, int n, int d, const double *_
 // 32 exponents of one row -> 32 kernel entries -> four running sums of K_il * in_l.  All 32 ex2 are issued before
 // the first multiply-add that needs one: with few epilogue warps per scheduler the special-function unit is only
 // kept busy if every warp has many independent ex2 in flight.
+template <bool COST>
 __device__ __forceinline__ void consume_chunk(const uint32_t *r, uint32_t vaddr, float &acc0, float &acc1, float &acc2,
                                               float &acc3) {
     float e[32];
@@ -133,17 +134,27 @@ __device__ __forceinline__ void consume_chunk(const uint32_t *r, uint32_t vaddr,
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
         const float4 v4 = lds4(vaddr + (uint32_t)q * 16u);
-        acc0 = fmaf(e[4 * q + 0], v4.x, acc0);
-        acc1 = fmaf(e[4 * q + 1], v4.y, acc1);
-        acc2 = fmaf(e[4 * q + 2], v4.z, acc2);
-        acc3 = fmaf(e[4 * q + 3], v4.w, acc3);
+        if (COST) { // sum of K_il in_l log2(K_il): the transport cost up to the factor -eps / log2(e)
+            acc0 = fmaf(e[4 * q + 0] * v4.x, __uint_as_float(r[4 * q + 0]), acc0);
+            acc1 = fmaf(e[4 * q + 1] * v4.y, __uint_as_float(r[4 * q + 1]), acc1);
+            acc2 = fmaf(e[4 * q + 2] * v4.z, __uint_as_float(r[4 * q + 2]), acc2);
+            acc3 = fmaf(e[4 * q + 3] * v4.w, __uint_as_float(r[4 * q + 3]), acc3);
+        } else {
+            acc0 = fmaf(e[4 * q + 0], v4.x, acc0);
+            acc1 = fmaf(e[4 * q + 1], v4.y, acc1);
+            acc2 = fmaf(e[4 * q + 2], v4.z, acc2);
+            acc3 = fmaf(e[4 * q + 3], v4.w, acc3);
+        }
     }
 }
 
 // ---- the pass kernel ----------------------------------------------------------------------
+// COST = false: the half-step.  COST = true: the same sweep accumulates 2^(t_il) * vin[l] * t_il instead, from which
+// the transport cost follows (C_il = -t_il * eps / log2(e)).
 // partial[(cs * 4 + g) * pitch + i] = sum over the columns l of the tiles that warpgroup g consumed of item (row tile
 // of i, column split cs) of 2^(t_il) * vin[l]; which tiles those are depends only on the launch geometry.
 // vin is padded with zeros up to tiles * 128 entries, so the padding columns of the last tile contribute nothing.
+template <bool COST>
 __global__ void __launch_bounds__(kImpThreads, 1)
 implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_constant__ CUtensorMap tmR_lo,
                      const __grid_constant__ CUtensorMap tmC_hi, const __grid_constant__ CUtensorMap tmC_lo,
@@ -281,18 +292,18 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
                 tmem_ld32_issue(lane_base, ra);
                 tmem_ld_wait32(ra);
                 tmem_ld32_issue(lane_base + 32, rb);
-                consume_chunk(ra, vaddr, acc0, acc1, acc2, acc3);
+                consume_chunk<COST>(ra, vaddr, acc0, acc1, acc2, acc3);
                 tmem_ld_wait32(rb);
                 tmem_ld32_issue(lane_base + 64, ra);
-                consume_chunk(rb, vaddr + 128u, acc0, acc1, acc2, acc3);
+                consume_chunk<COST>(rb, vaddr + 128u, acc0, acc1, acc2, acc3);
                 tmem_ld_wait32(ra);
                 tmem_ld32_issue(lane_base + 96, rb);
-                consume_chunk(ra, vaddr + 256u, acc0, acc1, acc2, acc3);
+                consume_chunk<COST>(ra, vaddr + 256u, acc0, acc1, acc2, acc3);
                 tmem_ld_wait32(rb);
                 fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(acc_empty + 8 * wg); // the whole tile has left tensor memory
-                consume_chunk(rb, vaddr + 384u, acc0, acc1, acc2, acc3);
+                consume_chunk<COST>(rb, vaddr + 384u, acc0, acc1, acc2, acc3);
             }
             bt0 += t1 - t0;
             if (ok) {
@@ -413,7 +424,8 @@ void *fsk_implicit_create(const float *X, const float *Y, int64_t n, int d, doub
     }
     fsk_free(mu), fsk_free(maxsq);
     for (int i = 0; i < 8 && ok; ++i) ok = make_map(&t->map[i], t->buf[i], t->n_pad);
-    ok = ok && cudaFuncSetAttribute(implicit_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
+    ok = ok && cudaFuncSetAttribute(implicit_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
+         cudaFuncSetAttribute(implicit_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         implicit_free(t);
@@ -436,8 +448,9 @@ float *fsk_implicit_partials(void *h) { return static_cast<ImplicitState *>(h)->
 
 // Stage 1 of one half-step: transposed = 0: partial sums of K in (rows = X, columns = Y); 1: of K^T in.
 // `in` holds n_pad floats, zero beyond n.  The caller runs the stage-2 kernel over the fsk_implicit_nsplit() partial rows.
-cudaError_t fsk_implicit_pass(void *h, int transposed, const float *in, FsDeviceStatus *status, cudaStream_t st) {
-    ImplicitState *t = static_cast<ImplicitState *>(h);
+namespace {
+template <bool COST>
+cudaError_t launch_pass(ImplicitState *t, int transposed, const float *in, FsDeviceStatus *status, cudaStream_t st) {
     const int r = transposed ? 4 : 0, c = transposed ? 2 : 6; // row-side arrays of one cloud, column-side of the other
     FS_HOST_CHECK(t->grid >= 1 && t->T >= 1 && t->T <= MAX_T && (int64_t)t->T * t->nsplit >= t->tiles &&
                   t->tiles * (int64_t)BM == t->n_pad && t->kd >= 1 && t->kd <= BK / 16);
@@ -446,6 +459,35 @@ cudaError_t fsk_implicit_pass(void *h, int transposed, const float *in, FsDevice
     cfg.blockDim = dim3(kImpThreads);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = st;
-    return cudaLaunchKernelEx(&cfg, implicit_pass_kernel, t->map[r], t->map[r + 1], t->map[c], t->map[c + 1], in, t->partials,
+    return cudaLaunchKernelEx(&cfg, implicit_pass_kernel<COST>, t->map[r], t->map[r + 1], t->map[c], t->map[c + 1], in, t->partials,
                               t->n_pad, (int)t->n, t->tiles, t->T, t->nsplit, t->kd, (long long)t->nsplit * NACC * t->n_pad, status);
+}
+
+// rowsum[i] = u_i * (sum of the partial rows of row i, in order) * scale, in double
+__global__ void __launch_bounds__(256)
+cost_rows_from_partials_kernel(const float *__restrict__ partials, int64_t pitch, int nparts, const float *__restrict__ u, int n,
+                               double scale, double *__restrict__ rowsum) {
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= n) return;
+    double s = 0.0;
+    for (int p = 0; p < nparts; ++p) s += (double)partials[(int64_t)p * pitch + i];
+    rowsum[i] = (double)u[i] * s * scale;
+}
+} // namespace
+
+cudaError_t fsk_implicit_pass(void *h, int transposed, const float *in, FsDeviceStatus *status, cudaStream_t st) {
+    return launch_pass<false>(static_cast<ImplicitState *>(h), transposed, in, status, st);
+}
+
+// Transport cost <P,C> = sum_il u_i K_il v_l C_il of the implicit plan, C_il = cost_scale |x_i - y_l|^2 = -t_il eps / log2(e):
+// one more sweep of the pass kernel that accumulates K_il v_l t_il per row, then rowsum[i] = -u_i (eps / log2 e) * that,
+// in double; the caller adds the n row sums in a fixed order.  rowsum: n doubles of scratch.
+cudaError_t fsk_implicit_cost_rows(void *h, const float *u, const float *v, double eps, double *rowsum, FsDeviceStatus *status,
+                                   cudaStream_t st) {
+    ImplicitState *t = static_cast<ImplicitState *>(h);
+    cudaError_t e = launch_pass<true>(t, 0, v, status, st);
+    if (e != cudaSuccess) return e;
+    cost_rows_from_partials_kernel<<<(unsigned)((t->n + 255) / 256), 256, 0, st>>>(t->partials, t->n_pad, t->nsplit * NACC, u, (int)t->n,
+                                                                                 -eps / 1.4426950408889634, rowsum);
+    return cudaGetLastError();
 }

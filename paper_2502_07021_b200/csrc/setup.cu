@@ -242,6 +242,10 @@ void fsk_transport_cost(int domain, const float *mat, int64_t ld, const float *C
     sum_rows_kernel<<<nbatch, kThreads, 0, st>>>(rowsum_scratch, n, cost_dev);
 }
 
+void fsk_sum_rows(const double *rowsum, int64_t n, int nbatch, double *out, cudaStream_t st) {
+    sum_rows_kernel<<<nbatch, kThreads, 0, st>>>(rowsum, n, out);
+}
+
 // ---- allocations, canaries, checked-build counters ---------------------------------------------
 #ifdef FS_DEBUG
 #include <stdio.h>

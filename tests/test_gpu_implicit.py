@@ -173,12 +173,23 @@ def test_implicit_refuses_what_it_cannot_do_accurately():
     with pytest.raises(fs.FsError) as ei:
         PointSolver(X, Y, 1.0, 10.0, a, b)
     assert ei.value.code == fs.FS_ERR_UNSUPPORTED
-    X, Y, a, b = random_clouds(64, 4, 4)
-    with PointSolver(X, Y, 1.0, 1.0, a, b) as g:
-        with pytest.raises(fs.FsError) as ei:
-            fs.fs_transport_cost(g.h, None, 0, 1, g.stream)
-        assert ei.value.code in (fs.FS_ERR_UNSUPPORTED, fs.FS_ERR_NULL)
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("cfg,n", [(2, 1500), (4, 4096), (5, 1024)])
+def test_implicit_transport_cost(cfg, n):
+    """<P,C> of the converged implicit plan, C_il = cost_scale |x_i - y_l|^2: one more sweep of the pass kernel
+    accumulates K_il v_l log2(K_il).  Reference: the checker's objective on the cost and kernel it forms from the same
+    points (rounded to fp32 for its interface: 6e-8), evaluated on the scalings the GPU returns; relative 1e-5."""
+    w = workloads.make(cfg, n=n, nbatch=1, fp32_points=True, want_cost=False, want_kernel=False)
+    with PointSolver(w.X, w.Y, w.cost_scale, w.eps, w.a, w.b, w.offsets) as g:
+        fs.fs_iterate(g.h, 200, g.stream)
+        x, y = g.scalings()
+        cost = fs.fs_transport_cost(g.h, None, 0, 1, g.stream)[0]
+    C = oracle.cost_from_points(w.X, w.Y, w.cost_scale)
+    C32 = C.astype(np.float32)
+    ref = oracle.objectives(C32, oracle.KIND_COST, w.eps, oracle.DOMAIN_SCALING, x, y, C32)["cost"]
+    assert abs(cost - ref) <= 1e-5 * abs(ref), (cost, ref)
 
 
 @pytest.mark.slow
