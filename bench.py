@@ -641,7 +641,7 @@ def run_ours(args, w, rank, local_rank, world):
                                  "achieved": burst_gbs, "frac": burst_gbs / peaks["hbm_gbs"],
                                  "us_per_launch": per_launch_burst_s * 1e6}, per_launch_burst_s, burst_clocks,
                                 "sm_cycles_per_launch"),
-            # BASELINE's accounting (every iteration streams 2 n^2 elements) applied to the timed region
+            # the metric's own accounting (every iteration streams 2 n^2 matrix elements) applied to the timed region
             "iteration_effective_gbs_2n2": 2 * n2 * its_region / (elapsed_ms * 1e-3) / 1e9}
     with_clock(roof, per_launch_sustained_s, clocks, "sm_cycles_per_launch")
 
