@@ -85,6 +85,8 @@ CHILD = textwrap.dedent("""
 
 
 def test_tiny_and_ragged_sizes_through_the_checked_build(tmp_path):
+    from paper_2502_07021_b200 import build as fs_build
+    fs_build.build(debug=True)                     # no-op when libfs_b200_debug.so is up to date
     script = tmp_path / "checked_child.py"
     script.write_text(CHILD % (ROOT, os.path.join(ROOT, "tests")))
     env = dict(os.environ, FS_B200_DEBUG="1")
