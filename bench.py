@@ -433,6 +433,58 @@ def time_implicit(fs, torch, dev, stream, w, devidx, args, wp=None):
     return out
 
 
+def run_shard_model(args):
+    """--multi model (one GPU): the local-compute term of the paper's per-iteration model (Section 4.1:
+    T_comp = 2 t_mv(m, n) + t_ew) measured for the row block a shard would own with G = 1, 2, 4, 8 shards of the
+    configuration: row pass + column partial + finish on an m x n block, m = n / G.  The exchange term cannot be
+    measured with one GPU; it is left out, not assumed."""
+    import torch
+    from paper_2502_07021_b200 import binding as fs
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.Stream(device=dev)
+    n = args.n or workloads._SPECS[args.config]["n"]
+    out = []
+    for G in (1, 2, 4, 8):
+        lo, hi = fsdist.row_range(n, 0, G)
+        w = workloads.make(args.config, n=args.n, nbatch=1, want_cost=False, rows=(lo, hi))
+        Kb = torch.from_numpy(w.K).to(dev)
+        a_loc = torch.from_numpy(w.a[lo:hi].copy()).to(dev)
+        b = torch.from_numpy(w.b).to(dev)
+        r_buf = torch.empty(w.n, dtype=torch.float32, device=dev)
+        torch.cuda.synchronize()
+        sh = fs.fs_shard_create(w.n, lo, hi - lo, Kb, w.n, fs.FS_MATRIX_KERNEL, w.eps, a_loc, b, stream)
+        iters = max(20, min(200, int(2e9 / ((hi - lo) * w.n * 8))))
+
+        def run(k):
+            for _ in range(k):
+                fs.fs_shard_row_pass(sh, stream)
+                fs.fs_shard_col_partial(sh, r_buf, stream)
+                fs.fs_shard_col_finish(sh, r_buf, stream)
+        run(5)
+        stream.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        run(iters)
+        e1.record(stream)
+        stream.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / iters
+        fs.fs_shard_destroy(sh)
+        del Kb
+        torch.cuda.empty_cache()
+        out.append({"shards": G, "rows_per_shard": hi - lo, "local_us_per_iteration": us,
+                    "local_gbs": 2 * (hi - lo) * w.n * 4 / (us * 1e-6) / 1e9,
+                    "exchange_bytes_per_iteration": w.n * 4})
+    line = {"metric": "shard_local_step_us", "unit": "us", "n_gpus": 1, "data": "synthetic", "dtype": "f32",
+            "config": {"workload": f"config {args.config}: n={n}, the row block of shard 0 of G"},
+            "model": out,
+            "note": "local operator time t_local(G) = 2 t_mv(n/G, n) + elementwise of one shard, measured on one GPU; "
+                    "an iteration on G GPUs costs max over shards of this plus one exchange of n floats (not measured here)"}
+    print(json.dumps(line), flush=True)
+
+
 def run_sharded(args, rank, local_rank, world):
     """Row-partitioned run (opt-in, --multi sharded): one shard of the SAME problem per GPU, one all-reduce
     of n floats per iteration over NCCL; total work is fixed, so scaling is strong."""
@@ -775,7 +827,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--ref-iters", type=int, default=1, help="--impl reference: iterations per step")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--multi", default="replicas", choices=["replicas", "sharded"],
+    ap.add_argument("--multi", default="replicas", choices=["replicas", "sharded", "model"],
                     help="N > 1: independent replicas (default, weak scaling) or row shards of one problem")
     ap.add_argument("--path", default="auto", choices=["auto", "implicit"],
                     help="implicit: time only the implicit-kernel path (fs_create_points) of the configuration")
@@ -798,6 +850,11 @@ def main():
         return 0
     if world > 1:
         fsdist.init()
+    if args.multi == "model":
+        if rank == 0:
+            run_shard_model(args)
+        fsdist.finalize()
+        return 0
     if args.multi == "sharded":
         try:
             run_sharded(args, rank, local_rank, world)
