@@ -457,24 +457,30 @@ def run_shard_model(args):
         sh = fs.fs_shard_create(w.n, lo, hi - lo, Kb, w.n, fs.FS_MATRIX_KERNEL, w.eps, a_loc, b, stream)
         iters = max(20, min(200, int(2e9 / ((hi - lo) * w.n * 8))))
 
-        def run(k):
+        def run(k, fused):
             for _ in range(k):
-                fs.fs_shard_row_pass(sh, stream)
-                fs.fs_shard_col_partial(sh, r_buf, stream)
+                if not (fused and fs.fs_shard_fused_step(sh, r_buf, stream, allow_unsupported=True)):
+                    fs.fs_shard_row_pass(sh, stream)
+                    fs.fs_shard_col_partial(sh, r_buf, stream)
                 fs.fs_shard_col_finish(sh, r_buf, stream)
-        run(5)
-        stream.synchronize()
-        e0 = torch.cuda.Event(enable_timing=True)
-        e1 = torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        run(iters)
-        e1.record(stream)
-        stream.synchronize()
-        us = e0.elapsed_time(e1) * 1e3 / iters
+
+        def timed_run(fused):
+            run(5, fused)
+            stream.synchronize()
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            run(iters, fused)
+            e1.record(stream)
+            stream.synchronize()
+            return e0.elapsed_time(e1) * 1e3 / iters
+        us = timed_run(False)
+        us_fused = timed_run(True)
         fs.fs_shard_destroy(sh)
         del Kb
         torch.cuda.empty_cache()
-        out.append({"shards": G, "rows_per_shard": hi - lo, "local_us_per_iteration": us,
+        out.append({"shards": G, "rows_per_shard": hi - lo, "local_us_per_iteration_single_read": us_fused,
+                    "local_us_per_iteration": us,
                     "local_gbs": 2 * (hi - lo) * w.n * 4 / (us * 1e-6) / 1e9,
                     "exchange_bytes_per_iteration": w.n * 4})
     line = {"metric": "shard_local_step_us", "unit": "us", "n_gpus": 1, "data": "synthetic", "dtype": "f32",

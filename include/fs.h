@@ -307,6 +307,12 @@ int fs_shard_create(fs_shard **out, int64_t n, int64_t row_lo, int64_t m, const 
                     int matrix_kind, double eps, const float *a_local_dev, const float *b_dev, void *stream);
 int fs_shard_row_pass(fs_shard *s, void *stream);
 int fs_shard_col_partial(fs_shard *s, float *r_dev_out, void *stream);
+/* The two local steps from ONE read of the shard's block: u_I = a_I ./ (K_{I,:} v) and p = (K_{I,:})^T u_I with the
+ * single-read fused kernel (Algorithm 1's first three statements on the local rows; a row is used for the column
+ * partial as soon as its own u_i is known).  Same results as fs_shard_row_pass + fs_shard_col_partial up to the
+ * grouping of the partial sums.  FS_ERR_UNSUPPORTED when the fused kernel does not apply (matrix not 16-byte aligned,
+ * n not a multiple of 4, n < 2048 or n > 65536) or a damping factor is set.  Asynchronous. */
+int fs_shard_fused_step(fs_shard *s, float *r_dev_out, void *stream);
 int fs_shard_col_finish(fs_shard *s, const float *r_total_dev, void *stream);
 /* Fixed reduction order for the column sums: the shards all-gather their partial vectors p^(g) (the caller's
  * collective) and every shard adds them itself, g = 0, 1, ..., G-1, before the divide.  parts_dev: DEVICE

@@ -58,6 +58,7 @@ _SIGNATURES = {
     "fs_shard_create": (_int, [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp, _i64, _int, _dbl, _vp, _vp, _vp]),
     "fs_shard_row_pass": (_int, [_vp, _vp]),
     "fs_shard_col_partial": (_int, [_vp, _vp, _vp]),
+    "fs_shard_fused_step": (_int, [_vp, _vp, _vp]),
     "fs_shard_col_finish": (_int, [_vp, _vp, _vp]),
     "fs_shard_col_finish_gathered": (_int, [_vp, _vp, _i32, _i64, _vp]),
     "fs_shard_col_block_pass": (_int, [_vp, _vp, _vp, _vp]),
@@ -265,6 +266,13 @@ def fs_shard_row_pass(s, stream=None):
 
 def fs_shard_col_partial(s, r_dev_out, stream=None):
     _check(lib().fs_shard_col_partial(s, _dev(r_dev_out), _stream(stream)), "fs_shard_col_partial")
+
+
+def fs_shard_fused_step(s, r_dev_out, stream=None, allow_unsupported=False):
+    """Row step and column partial from one read of the block; returns False when the fused kernel does not apply."""
+    rc = _check(lib().fs_shard_fused_step(s, _dev(r_dev_out), _stream(stream)), "fs_shard_fused_step",
+                allow=(FS_ERR_UNSUPPORTED,) if allow_unsupported else ())
+    return rc == FS_OK
 
 
 def fs_shard_col_finish(s, r_total_dev, stream=None):

@@ -204,6 +204,7 @@ void fsk_col_finish(int64_t n, int64_t n_pad, int ntiles, const float *partials,
 void fsk_log_col_finish(int64_t n, int64_t n_pad, int ntiles, double eps, const float *partials, const float *b,
                         const float *logb, float *g, float *ys, float *coldiff, int update, FsDeviceStatus *status,
                         cudaStream_t st);
+void fsk_sum_partials(int64_t n, int64_t n_pad, int nrows_partial, const float *partials, float *r_out, cudaStream_t st);
 int fsk_pass_launches_row();
 int fsk_pass_launches_col();
 

@@ -606,5 +606,10 @@ void fsk_log_col_finish(int64_t n, int64_t n_pad, int ntiles, double eps, const 
         (int)n, n_pad, ntiles, s2, eps, partials, b, logb, g, ys, coldiff, update, status);
 }
 
+// r_out[l] = sum over `nrows_partial` partial rows of pitch n_pad, in the fixed order of the stage-2 kernels.
+void fsk_sum_partials(int64_t n, int64_t n_pad, int nrows_partial, const float *partials, float *r_out, cudaStream_t st) {
+    sum_partials_kernel<<<(unsigned)((n + 31) / 32), kThreads, 0, st>>>((int)n, n_pad, nrows_partial, partials, r_out);
+}
+
 int fsk_pass_launches_row() { return 1; }
 int fsk_pass_launches_col() { return 2; }

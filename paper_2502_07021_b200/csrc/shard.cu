@@ -35,6 +35,11 @@ struct fs_shard {
     FsDeviceStatus *status = nullptr;
     FsPassPlan plan{};
     float eta = 1.f;
+    // single-read fused local step (fused.cu on the shard's row block): u_I and the column partial from ONE read
+    FsFusedPlan fused{};
+    FsRowTile *fused_tiles_dev = nullptr;
+    int fused_ntiles = 0;
+    float *fused_partials = nullptr;
 };
 
 namespace {
@@ -120,10 +125,44 @@ int fs_shard_create(fs_shard **out, int64_t n, int64_t row_lo, int64_t m, const 
     FS_SH(fsk_malloc(&s->tiles_dev, sizeof(FsRowTile) * tiles.size()));
     FS_SH(cudaMemcpyAsync(s->tiles_dev, tiles.data(), sizeof(FsRowTile) * tiles.size(), cudaMemcpyHostToDevice, st));
     FS_SH(fsk_malloc(&s->partials, sizeof(float) * tiles.size() * (size_t)s->n_pad));
+    s->fused = fsk_fused_plan(n, vec);
+    if (s->fused.enabled) {
+        // tile height for the block's m rows (the plan chose one for n rows): the one that gives the busiest cluster
+        // the fewest rows, a multiple of the kernel's rows per stage
+        int best = 32;
+        int64_t best_rows = ((m + 31) / 32 + s->fused.nclusters - 1) / s->fused.nclusters * 32;
+        for (int tr = 16; tr >= s->fused.R && tr >= 4; tr >>= 1) {
+            const int64_t nt = (m + tr - 1) / tr, rows = (nt + s->fused.nclusters - 1) / s->fused.nclusters * tr;
+            if (rows < best_rows) best_rows = rows, best = tr;
+        }
+        s->fused.tile_rows = best;
+        std::vector<FsRowTile> ft;
+        for (int64_t r = 0; r < m; r += s->fused.tile_rows)
+            ft.push_back(FsRowTile{(int32_t)r, (int32_t)(r + s->fused.tile_rows < m ? r + s->fused.tile_rows : m)});
+        s->fused_ntiles = (int)ft.size();
+        FS_SH(cudaMalloc(&s->fused_tiles_dev, sizeof(FsRowTile) * ft.size()));
+        FS_SH(cudaMemcpyAsync(s->fused_tiles_dev, ft.data(), sizeof(FsRowTile) * ft.size(), cudaMemcpyHostToDevice, st));
+        const size_t pbytes = sizeof(float) * (size_t)s->fused.nclusters * (size_t)n;
+        FS_SH(cudaMalloc(&s->fused_partials, pbytes));
+        FS_SH(cudaMemsetAsync(s->fused_partials, 0, pbytes, st));
+    }
     FS_SH(cudaStreamSynchronize(st));
     FS_SH(cudaGetLastError());
     guard.s = nullptr;
     *out = s;
+    return FS_OK;
+}
+
+int fs_shard_fused_step(fs_shard *s, float *r_dev_out, void *stream) {
+    if (!s || !r_dev_out) return FS_ERR_NULL;
+    if (!s->fused.enabled || s->eta != 1.f) return FS_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    // clusters without a row tile (short blocks) leave their partial rows untouched: they were cleared at creation
+    // and nothing else writes them
+    FS_SH(fsk_fused_iteration(s->fused, s->mat, s->mat_ld, s->n, s->fused_tiles_dev, s->fused_ntiles, s->v, s->a, s->u, s->u,
+                              s->rowdiff, s->fused_partials, 1.f, s->status, st));
+    fsk_sum_partials(s->n, s->n, s->fused.nclusters, s->fused_partials, r_dev_out, st);
+    FS_SH(cudaGetLastError());
     return FS_OK;
 }
 

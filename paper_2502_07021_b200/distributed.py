@@ -117,7 +117,7 @@ def gather_blocks(local_block, sizes, out_full, group=None):
 
 
 def sharded_iterate(api, shard, r_buf, k: int, stream=None, group=None, exchange: str = "allreduce", sizes=None,
-                    timed: bool = False):
+                    timed: bool = False, fused_local: bool = True):
     """k Sinkhorn iterations of a row-partitioned problem, one shard per process.
 
     exchange = "allreduce": Algorithm 1 with the column sums assembled by ONE sum all-reduce of the per-shard
@@ -131,7 +131,8 @@ def sharded_iterate(api, shard, r_buf, k: int, stream=None, group=None, exchange
 
     `api` provides the fs_shard_* steps (the ctypes binding on GPUs); `r_buf` is a length-n float32 tensor on the
     shard's device.  Collectives are torch.distributed's (NCCL on GPUs, gloo on CPU); with a CUDA `stream` all
-    steps are ordered on that stream.  With `timed` the time of the local steps and of the exchanges is
+    steps are ordered on that stream.  With `fused_local` the row step and the column partial of the "allreduce" and
+    "ordered" forms come from one read of the local block (fs_shard_fused_step) where that kernel applies.  With `timed` the time of the local steps and of the exchanges is
     accumulated separately (the paper's compute / communication split) and returned as a dict.
     """
     import contextlib
@@ -178,6 +179,10 @@ def sharded_iterate(api, shard, r_buf, k: int, stream=None, group=None, exchange
                 continue
 
             def local_partial():
+                # one read of the local block for both local steps where the fused kernel applies
+                step = getattr(api, "fs_shard_fused_step", None) if fused_local else None
+                if step is not None and step(shard, r_buf, stream, allow_unsupported=True):
+                    return
                 api.fs_shard_row_pass(shard, stream)
                 api.fs_shard_col_partial(shard, r_buf, stream)
             phase("local", local_partial)

@@ -176,3 +176,44 @@ def test_shards_add_gathered_partials_in_rank_order_reproducibly():
     off = [fsdist.row_range(n, r, G)[0] for r in range(G)] + [n]
     uo, vo = oracle.sinkhorn_rowpartition(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, off, 8)
     assert np.max(np.abs(runs[0][0] - uo) / uo) <= 1e-4 and np.max(np.abs(runs[0][1] - vo) / vo) <= 1e-4
+
+
+@pytest.mark.parametrize("n,G", [(4100, 2), (8192, 4)])
+def test_shards_single_read_local_step(n, G):
+    """fs_shard_fused_step (row step and column partial from ONE read of the block) against the two separate local
+    steps and the oracle's row-partition iterates; unequal blocks, ragged column segments."""
+    import torch
+    w = workloads.make(2, n=n)
+    dev = torch.device("cuda:0")
+    stream = torch.cuda.Stream(device=dev)
+    res = {}
+    for fused in (True, False):
+        shards, blocks, keep = make_shards(w, G, torch, dev, stream)
+        parts = torch.empty(G * n, dtype=torch.float32, device=dev)
+        try:
+            with torch.cuda.stream(stream):
+                for _ in range(8):
+                    for g, s in enumerate(shards):
+                        p = parts[g * n:(g + 1) * n]
+                        if fused:
+                            assert fs.fs_shard_fused_step(s, p, stream)
+                        else:
+                            fs.fs_shard_row_pass(s, stream)
+                            fs.fs_shard_col_partial(s, p, stream)
+                    for s in shards:
+                        fs.fs_shard_col_finish_gathered(s, parts, G, n, stream)
+            u = np.empty(n, dtype=np.float32)
+            for s, (lo, hi) in zip(shards, blocks):
+                ub = torch.empty(hi - lo, dtype=torch.float32, device=dev)
+                vb = torch.empty(n, dtype=torch.float32, device=dev)
+                fs.fs_shard_scalings(s, ub, vb, stream)
+                u[lo:hi] = ub.cpu().numpy()
+            res[fused] = (u, vb.cpu().numpy())
+        finally:
+            for s in shards:
+                fs.fs_shard_destroy(s)
+    off = [fsdist.row_range(n, r, G)[0] for r in range(G)] + [n]
+    uo, vo = oracle.sinkhorn_rowpartition(w.K, oracle.KIND_KERNEL, w.eps, w.a, w.b, off, 8)
+    for fused in (True, False):
+        assert np.max(np.abs(res[fused][0] - uo) / uo) <= 1e-4 and np.max(np.abs(res[fused][1] - vo) / vo) <= 1e-4
+    assert np.max(np.abs(res[True][0] - res[False][0]) / res[False][0]) < 1e-5
