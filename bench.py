@@ -518,6 +518,9 @@ def run_sharded(args, rank, local_rank, world):
     torch.cuda.synchronize()
     sh = fs.fs_shard_create(w.n, lo, hi - lo, Kb, w.n, fs.FS_MATRIX_KERNEL, w.eps, a_loc, b, stream)
 
+    # does the single-read local step apply (then the local block is read once per iteration, not twice)?
+    single_read = args.exchange != "alg1" and fs.fs_shard_fused_step(sh, r_buf, stream, allow_unsupported=True)
+    reads_per_iteration = 1 if single_read else 2
     sizes = [fsdist.row_range(n_total, r, world)[1] - fsdist.row_range(n_total, r, world)[0] for r in range(world)]
     split = {"local_ms": 0.0, "exchange_ms": 0.0}
 
@@ -572,9 +575,11 @@ def run_sharded(args, rank, local_rank, world):
                             "note": "CUDA events around every local step and every collective of one extra step, max over "
                                     "ranks; the paper reports the same split (local matvec time vs collective time)"},
             "gpu_launches": int(its * 5), "clocks": clocks, "e2e": None,
-            "roofline": {"bound": "hbm", "kernel": "row_pass_kernel + col_partial_kernel (per shard)",
-                         "achieved": 2 * per_pass_bytes * its / (t_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                         "unit": "GB/s", "frac": 2 * per_pass_bytes * its / (t_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "roofline": {"bound": "hbm", "kernel": "fused_iteration_kernel on the shard's block" if single_read
+                         else "row_pass_kernel + col_partial_kernel (per shard)",
+                         "achieved": reads_per_iteration * per_pass_bytes * its / (t_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s",
+                         "frac": reads_per_iteration * per_pass_bytes * its / (t_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                          "peak_source": f"of {peak_kind}", "traffic": None,
                          "note": "per-GPU rate over the whole iteration, collectives included"},
             "cpu_baseline": None, "row_marginal_l1_before_last_iteration": l1}
