@@ -196,6 +196,11 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
     fence_after();
     const uint32_t tmem = *tmem_slot_ptr;
     bool ok = true;
+    // The pass is launched with programmatic stream serialisation: it may become resident while the stage-2 kernel
+    // before it is still running.  The operands of the two clouds never change, so their tiles are requested and
+    // the first exponent tiles are formed at once; what that kernel produces (the input vector) or still reads (the
+    // partial sums of the previous pass) is touched only behind griddep_wait.
+    griddep_launch_dependents();
 
     if (warp == 0) {
         // ---------------- producer ----------------
@@ -211,6 +216,7 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
                 mbar_expect_tx(full, (uint32_t)PAIR_BYTES + (uint32_t)(t1 - t0) * BN * 4u);
                 tma_load_2d(&tmR_hi, base + OFF_A + slot * PAIR_BYTES, full, 0, rt * BM);
                 tma_load_2d(&tmR_lo, base + OFF_A + slot * PAIR_BYTES + TILE_BYTES, full, 0, rt * BM);
+                if (k == 0) griddep_wait(); // the input vector is the predecessor's output
                 bulk_load(base + OFF_V + slot * VSLOT_BYTES, vin + (int64_t)t0 * BN, (uint32_t)(t1 - t0) * BN * 4u, full);
                 ki = k + 1;
                 for (int j = t0; j < t1; ++j, ++bt) {
@@ -272,6 +278,7 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(wg * BN);
         int k = 0, bt0 = 0; // items begun; index in the CTA's tile stream of the item's first tile
+        griddep_wait();     // the partial sums this warp will overwrite may still be read by the predecessor
         for (int w = blockIdx.x; w < nitems; w += gridDim.x, ++k) {
             const int slot = k & 1;
             const int rt = w / nsplit, cs = w % nsplit;
@@ -459,6 +466,10 @@ cudaError_t launch_pass(ImplicitState *t, int transposed, const float *in, FsDev
     cfg.blockDim = dim3(kImpThreads);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr, cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, implicit_pass_kernel<COST>, t->map[r], t->map[r + 1], t->map[c], t->map[c + 1], in, t->partials,
                               t->n_pad, (int)t->n, t->tiles, t->T, t->nsplit, t->kd, (long long)t->nsplit * NACC * t->n_pad, status);
 }

@@ -94,6 +94,11 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
 __host__ __device__ constexpr uint32_t idesc_bf16_m128(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
+// Programmatic dependent launch.  launch_dependents: the next kernel in the stream, if it was launched with
+// programmatic stream serialisation, may begin once every CTA of this grid has executed this (or exited).
+// wait: returns when the preceding grid has completed and its writes are visible; a no-op otherwise.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ float4 lds4(uint32_t addr) {
     float4 r;
     asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(addr));
