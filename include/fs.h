@@ -236,7 +236,7 @@ int fs_solve_host(int64_t n, int32_t c, const int64_t *row_offsets, const float 
  *
  *   X_dev, Y_dev  DEVICE [n][d] fp32 row-major point clouds (Y_dev may equal X_dev: one cloud, symmetric cost).
  *                 Copied into the library's own operand layout; not needed after the call.
- *   d             coordinates per point, 1 <= d <= 58 (FS_ERR_UNSUPPORTED beyond).
+ *   d             coordinates per point, 1 <= d <= 122 (FS_ERR_UNSUPPORTED beyond).
  *   cost_scale    factor on the squared distance (e.g. 1 / largest squared distance), > 0.
  *   n, c, row_offsets, eps, a_dev, b_dev, stream   as for fs_create; one problem, scaling domain.
  *

@@ -40,25 +40,27 @@ using namespace fstc;
 constexpr int BM = 128, BN = 128, BK = 64;
 constexpr int TILE_BYTES = BM * BK * 2;      // one bf16 operand tile (hi or lo): 128 rows of 128 bytes
 constexpr int PAIR_BYTES = 2 * TILE_BYTES;   // hi + lo
-constexpr int B_STAGES = 3;
+constexpr int MAX_KB = 2;                    // 64-column k-blocks of the contraction: coordinates + 6 <= 128
+constexpr int MAX_B_STAGES = 3;              // ring of column-operand (tile, k-block) entries: 3 with one k-block, 2 with two
 constexpr int MAX_T = 32;                    // column tiles per work item (input slice of at most 16 KB)
 constexpr int VSLOT_BYTES = MAX_T * BN * 4;
 constexpr int EPI_WARPS = 16;                // four per scheduler: enough independent ex2 in flight to keep the unit busy
 constexpr int kImpThreads = 64 + 32 * EPI_WARPS; // TMA warp, MMA warp, sixteen epilogue warps
 constexpr int NACC = 4;                      // exponent tiles in flight between the tensor core and the epilogue
 constexpr int TMEM_COLS = NACC * BN;         // four 128-column fp32 accumulators: all of tensor memory
-constexpr int kMaxDim = BK - 6;              // coordinates + 3 norm terms + 3 ones fit one 64-column k-block
-// shared memory: A slots, B ring, input slots, barriers, TMEM slot
-constexpr int OFF_A = 0;
-constexpr int OFF_B = OFF_A + 2 * PAIR_BYTES;
-constexpr int OFF_V = OFF_B + B_STAGES * PAIR_BYTES;
-constexpr int OFF_BARS = OFF_V + 2 * VSLOT_BYTES;
-constexpr int NUM_BARS = 6 + 2 * B_STAGES + 2 * NACC; // item_full[2], item_free_mma[2], item_free_epi[2], b_full, b_empty, acc_full, acc_empty
-constexpr int SMEM_BYTES = OFF_BARS + 8 * NUM_BARS + 16 + 1024;
+constexpr int kMaxDim = MAX_KB * BK - 6;     // coordinates + 3 norm terms + 3 ones fit the k-blocks
+// shared memory (kb = number of k-blocks): two row-operand slots of kb pairs, the column-operand ring (3 entries with
+// kb = 1, 2 with kb = 2), two input slots, barriers, TMEM slot.  224 KB + barriers in both cases.
+__host__ __device__ constexpr int b_stages(int kb) { return kb == 1 ? 3 : 2; }
+__host__ __device__ constexpr int off_b(int kb) { return 2 * kb * PAIR_BYTES; }
+__host__ __device__ constexpr int off_v(int kb) { return off_b(kb) + b_stages(kb) * PAIR_BYTES; }
+__host__ __device__ constexpr int off_bars(int kb) { return off_v(kb) + 2 * VSLOT_BYTES; }
+constexpr int NUM_BARS = 6 + 2 * MAX_B_STAGES + 2 * NACC; // item_full[2], item_free_mma[2], item_free_epi[2], b_full, b_empty, acc_full, acc_empty
+__host__ __device__ constexpr int smem_bytes(int kb) { return off_bars(kb) + 8 * NUM_BARS + 16 + 1024; }
 
 struct ImplicitState {
     int64_t n = 0, n_pad = 0;
-    int d = 0, kd = 0;            // coordinates per point; 16-wide k-steps of the contraction
+    int d = 0, kd = 0, kblocks = 1; // coordinates per point; 16-wide k-steps of the LAST k-block; 64-column k-blocks
     int tiles = 0;                // 128-point tiles per cloud
     int T = 0, nsplit = 0;        // column tiles per item, items per row tile
     int grid = 0;
@@ -91,16 +93,16 @@ cloud_mean_kernel(const float *__restrict__ X, const float *__restrict__ Y, int 
 
 // One thread per point: z = sqrt(2c) (p - mu) rounded to fp32 and split into bf16 hi + lo; h = -|z|^2/2 (from the
 // rounded z, in double) split into three bf16 terms.  Row-side layout: [z | h1 h2 h3 | 1 1 1], column-side layout:
-// [z | 1 1 1 | h1 h2 h3]; rows of 64 bf16, the rest zero (the buffers are cleared before).  maxsq receives the
+// [z | 1 1 1 | h1 h2 h3]; rows of `pitch` bf16, the rest zero (the buffers are cleared before).  maxsq receives the
 // largest |z|^2 as the bit pattern of a non-negative float.
 __global__ void __launch_bounds__(256)
-prepare_points_kernel(const float *__restrict__ P, int n, int d, const double *__restrict__ mu, double sqrt2c,
+prepare_points_kernel(const float *__restrict__ P, int n, int d, int pitch, const double *__restrict__ mu, double sqrt2c,
                       __nv_bfloat16 *__restrict__ row_hi, __nv_bfloat16 *__restrict__ row_lo,
                       __nv_bfloat16 *__restrict__ col_hi, __nv_bfloat16 *__restrict__ col_lo, unsigned int *maxsq) {
     const int i = blockIdx.x * 256 + threadIdx.x;
     if (i >= n) return;
     double sq = 0.0;
-    const int64_t o = (int64_t)i * BK;
+    const int64_t o = (int64_t)i * pitch; // pitch = 64 * k-blocks bf16 per point
     for (int k = 0; k < d; ++k) {
         const float z = (float)(sqrt2c * ((double)P[(int64_t)i * d + k] - mu[k]));
         __nv_bfloat16 hi, lo;
@@ -154,18 +156,22 @@ __device__ __forceinline__ void consume_chunk(const uint32_t *r, uint32_t vaddr,
 // partial[(cs * 4 + g) * pitch + i] = sum over the columns l of the tiles that warpgroup g consumed of item (row tile
 // of i, column split cs) of 2^(t_il) * vin[l]; which tiles those are depends only on the launch geometry.
 // vin is padded with zeros up to tiles * 128 entries, so the padding columns of the last tile contribute nothing.
-template <bool COST>
+template <bool COST, int KB>
 __global__ void __launch_bounds__(kImpThreads, 1)
 implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_constant__ CUtensorMap tmR_lo,
                      const __grid_constant__ CUtensorMap tmC_hi, const __grid_constant__ CUtensorMap tmC_lo,
                      const float *__restrict__ vin, float *__restrict__ partial, int64_t pitch, int nrows, int tiles,
                      int T, int nsplit, int kd, long long partial_elems, FsDeviceStatus *status) {
+    constexpr int kblocks = KB; // 64-column k-blocks of the contraction (compile-time: the issuing threads' index
+                                // arithmetic sits on the critical path)
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bars = base + OFF_BARS;
+    constexpr int OFF_A = 0, OFF_B = off_b(kblocks), OFF_V = off_v(kblocks), B_STAGES = b_stages(kblocks);
+    constexpr int ASLOT = kblocks * PAIR_BYTES; // one row-operand slot: hi and lo tile of every k-block
+    const uint32_t bars = base + off_bars(kblocks);
     const uint32_t item_full = bars, item_free_mma = bars + 16, item_free_epi = bars + 32;
-    const uint32_t b_full = bars + 48, b_empty = b_full + 8 * B_STAGES;
-    const uint32_t acc_full = b_empty + 8 * B_STAGES, acc_empty = acc_full + 8 * NACC;
+    const uint32_t b_full = bars + 48, b_empty = b_full + 8 * MAX_B_STAGES;
+    const uint32_t acc_full = b_empty + 8 * MAX_B_STAGES, acc_empty = acc_full + 8 * NACC;
     const uint32_t tmem_slot = bars + 8 * NUM_BARS;
     uint32_t *tmem_slot_ptr = reinterpret_cast<uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -181,7 +187,7 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
             mbar_init(acc_full + 8 * s, 1);
             mbar_init(acc_empty + 8 * s, EPI_WARPS / NACC);
         }
-        for (int s = 0; s < B_STAGES; ++s) {
+        for (int s = 0; s < MAX_B_STAGES; ++s) {
             mbar_init(b_full + 8 * s, 1);
             mbar_init(b_empty + 8 * s, 1);
         }
@@ -205,7 +211,9 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
     if (warp == 0) {
         // ---------------- producer ----------------
         if (lane == 0) {
-            int k = 0, bt = 0, ki = 0; // items begun, column tiles issued, items whose loads were issued
+            int k = 0, bt = 0, ki = 0; // items begun, ring entries issued, items whose loads were issued
+            int ps = 0;                // ring position and its barrier phase, carried along
+            uint32_t pph = 0;
             for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x, ++k) {
                 const int slot = k & 1;
                 const uint32_t ph = (uint32_t)(k >> 1) & 1u;
@@ -213,19 +221,24 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
                 const int rt = w / nsplit, cs = w % nsplit;
                 const int t0 = cs * T, t1 = min(t0 + T, tiles);
                 const uint32_t full = item_full + 8 * slot;
-                mbar_expect_tx(full, (uint32_t)PAIR_BYTES + (uint32_t)(t1 - t0) * BN * 4u);
-                tma_load_2d(&tmR_hi, base + OFF_A + slot * PAIR_BYTES, full, 0, rt * BM);
-                tma_load_2d(&tmR_lo, base + OFF_A + slot * PAIR_BYTES + TILE_BYTES, full, 0, rt * BM);
+                mbar_expect_tx(full, (uint32_t)ASLOT + (uint32_t)(t1 - t0) * BN * 4u);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    tma_load_2d(&tmR_hi, base + OFF_A + slot * ASLOT + kb * PAIR_BYTES, full, kb * BK, rt * BM);
+                    tma_load_2d(&tmR_lo, base + OFF_A + slot * ASLOT + kb * PAIR_BYTES + TILE_BYTES, full, kb * BK, rt * BM);
+                }
                 if (k == 0) griddep_wait(); // the input vector is the predecessor's output
                 bulk_load(base + OFF_V + slot * VSLOT_BYTES, vin + (int64_t)t0 * BN, (uint32_t)(t1 - t0) * BN * 4u, full);
                 ki = k + 1;
-                for (int j = t0; j < t1; ++j, ++bt) {
-                    const int s = bt % B_STAGES;
-                    if (!mbar_wait(b_empty + 8 * s, ((uint32_t)(bt / B_STAGES) & 1u) ^ 1u)) { ok = false; break; }
-                    const uint32_t bf = b_full + 8 * s, dst = base + OFF_B + s * PAIR_BYTES;
-                    mbar_expect_tx(bf, PAIR_BYTES);
-                    tma_load_2d(&tmC_hi, dst, bf, 0, j * BN);
-                    tma_load_2d(&tmC_lo, dst + TILE_BYTES, bf, 0, j * BN);
+                for (int j = t0; j < t1 && ok; ++j) { // ring entries: (column tile, k-block)
+#pragma unroll
+                    for (int kb = 0; kb < kblocks; ++kb, ++bt) {
+                        if (!mbar_wait(b_empty + 8 * ps, pph ^ 1u)) { ok = false; break; }
+                        const uint32_t bf = b_full + 8 * ps, dst = base + OFF_B + ps * PAIR_BYTES;
+                        mbar_expect_tx(bf, PAIR_BYTES);
+                        tma_load_2d(&tmC_hi, dst, bf, kb * BK, j * BN);
+                        tma_load_2d(&tmC_lo, dst + TILE_BYTES, bf, kb * BK, j * BN);
+                        if (++ps == B_STAGES) ps = 0, pph ^= 1u;
+                    }
                 }
             }
             if (!ok) {
@@ -238,30 +251,42 @@ implicit_pass_kernel(const __grid_constant__ CUtensorMap tmR_hi, const __grid_co
         // ---------------- MMA issue ----------------
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16_m128(BN);
-            int k = 0, bt = 0;
+            // This thread's loop is on the critical path of every tile (a tile's MMAs are issued only after its
+            // bookkeeping), so ring positions, barrier phases and descriptors are carried along instead of being
+            // recomputed from counters.
+            int k = 0;
+            int s = 0, buf = 0;               // ring entry and accumulator in use
+            uint32_t sph = 0, aph = 0;        // their barrier phases
+            const uint64_t bdesc0 = make_desc(base + OFF_B);
             for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x, ++k) {
                 const int slot = k & 1;
                 if (!mbar_wait(item_full + 8 * slot, (uint32_t)(k >> 1) & 1u)) { ok = false; break; }
                 fence_after();
                 const int cs = w % nsplit;
-                const int t0 = cs * T, t1 = min(t0 + T, tiles);
-                const uint64_t a_hi = make_desc(base + OFF_A + slot * PAIR_BYTES), a_lo = make_desc(base + OFF_A + slot * PAIR_BYTES + TILE_BYTES);
-                for (int j = t0; j < t1; ++j, ++bt) {
-                    const int s = bt % B_STAGES, buf = bt % NACC;
-                    if (!mbar_wait(acc_empty + 8 * buf, ((uint32_t)(bt / NACC) & 1u) ^ 1u)) { ok = false; break; }
-                    if (!mbar_wait(b_full + 8 * s, (uint32_t)(bt / B_STAGES) & 1u)) { ok = false; break; }
-                    fence_after();
-                    const uint32_t st = base + OFF_B + s * PAIR_BYTES;
-                    const uint64_t b_hi = make_desc(st), b_lo = make_desc(st + TILE_BYTES);
+                const int ntile = min(cs * T + T, tiles) - cs * T;
+                const uint64_t adesc0 = make_desc(base + OFF_A + slot * ASLOT);
+                for (int j = 0; j < ntile && ok; ++j) {
+                    if (!mbar_wait(acc_empty + 8 * buf, aph ^ 1u)) { ok = false; break; }
                     const uint32_t acc = tmem + (uint32_t)(buf * BN);
-                    for (int kk = 0; kk < kd; ++kk) {
-                        const uint64_t adv = (uint64_t)(kk * 32 >> 4); // 16 bf16 = 32 bytes along the contraction
-                        mma_bf16(acc, a_lo + adv, b_hi + adv, idesc, kk > 0 ? 1u : 0u);
-                        mma_bf16(acc, a_hi + adv, b_lo + adv, idesc, 1u);
-                        mma_bf16(acc, a_hi + adv, b_hi + adv, idesc, 1u);
+#pragma unroll
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        if (!mbar_wait(b_full + 8 * s, sph)) { ok = false; break; }
+                        fence_after();
+                        // descriptors address shared memory in units of 16 bytes: a pair is hi tile, then lo tile
+                        const uint64_t a_hi = adesc0 + (uint64_t)(kb * (PAIR_BYTES >> 4)), a_lo = a_hi + (TILE_BYTES >> 4);
+                        const uint64_t b_hi = bdesc0 + (uint64_t)(s * (PAIR_BYTES >> 4)), b_lo = b_hi + (TILE_BYTES >> 4);
+                        const int steps = kb + 1 < kblocks ? BK / 16 : kd; // full k-blocks, then the k-steps of the last one
+                        for (int kk = 0; kk < steps; ++kk) {
+                            const uint64_t adv = (uint64_t)(kk * 2); // 16 bf16 = 32 bytes along the contraction
+                            mma_bf16(acc, a_lo + adv, b_hi + adv, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                            mma_bf16(acc, a_hi + adv, b_lo + adv, idesc, 1u);
+                            mma_bf16(acc, a_hi + adv, b_hi + adv, idesc, 1u);
+                        }
+                        commit(b_empty + 8 * s);  // ring entry free once these MMAs have read it
+                        if (++s == B_STAGES) s = 0, sph ^= 1u;
                     }
-                    commit(b_empty + 8 * s);      // ring slot free once these MMAs have read it
-                    commit(acc_full + 8 * buf);   // exponent tile complete
+                    if (ok) commit(acc_full + 8 * buf); // exponent tile complete
+                    if (++buf == NACC) buf = 0, aph ^= 1u;
                 }
                 if (ok) commit(item_free_mma + 8 * slot); // row operand slot free once every MMA of the item has read it
             }
@@ -349,12 +374,12 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// operand array of `rows` points x 64 bf16 (rows of 128 bytes); box = one 128-point tile, 128-byte swizzle
-bool make_map(CUtensorMap *map, const __nv_bfloat16 *ptr, int64_t rows) {
+// operand array of `rows` points x (64 * kblocks) bf16; box = one 128-point tile of one k-block, 128-byte swizzle
+bool make_map(CUtensorMap *map, const __nv_bfloat16 *ptr, int64_t rows, int kblocks) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)BK, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)BK * 2};
+    cuuint64_t dims[2] = {(cuuint64_t)BK * kblocks, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)BK * kblocks * 2};
     cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16 *>(ptr), dims, strides, box, estr,
@@ -404,13 +429,14 @@ void *fsk_implicit_create(const float *X, const float *Y, int64_t n, int d, doub
     t->n = n, t->d = d;
     t->n_pad = fsk_implicit_padded_n(n);
     t->tiles = (int)(t->n_pad / BM);
-    t->kd = (d + 6 + 15) / 16;
+    t->kblocks = (d + 6 + BK - 1) / BK;
+    t->kd = (d + 6 - (t->kblocks - 1) * BK + 15) / 16;
     int sms = 148, dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     choose_split(t->tiles, sms, &t->T, &t->nsplit);
     const int64_t items = (int64_t)t->tiles * t->nsplit;
     t->grid = (int)(items < sms ? items : sms);
-    const size_t bytes = (size_t)t->n_pad * BK * 2;
+    const size_t bytes = (size_t)t->n_pad * BK * t->kblocks * 2;
     bool ok = true;
     for (auto &p : t->buf) ok = ok && fsk_malloc(&p, bytes) == cudaSuccess && cudaMemsetAsync(p, 0, bytes, st) == cudaSuccess;
     ok = ok && fsk_malloc(&t->partials, sizeof(float) * (size_t)t->nsplit * NACC * t->n_pad) == cudaSuccess;
@@ -423,16 +449,18 @@ void *fsk_implicit_create(const float *X, const float *Y, int64_t n, int d, doub
         const double sqrt2c = sqrt(2.0 * cost_scale / eps * 1.4426950408889634);
         const unsigned grid = (unsigned)((n + 255) / 256);
         cloud_mean_kernel<<<d, 256, 0, st>>>(X, Y, (int)n, d, mu);
-        prepare_points_kernel<<<grid, 256, 0, st>>>(X, (int)n, d, mu, sqrt2c, t->buf[0], t->buf[1], t->buf[2], t->buf[3], maxsq);
-        prepare_points_kernel<<<grid, 256, 0, st>>>(Y, (int)n, d, mu, sqrt2c, t->buf[4], t->buf[5], t->buf[6], t->buf[7], maxsq + 1);
+        prepare_points_kernel<<<grid, 256, 0, st>>>(X, (int)n, d, BK * t->kblocks, mu, sqrt2c, t->buf[0], t->buf[1], t->buf[2], t->buf[3], maxsq);
+        prepare_points_kernel<<<grid, 256, 0, st>>>(Y, (int)n, d, BK * t->kblocks, mu, sqrt2c, t->buf[4], t->buf[5], t->buf[6], t->buf[7], maxsq + 1);
         ok = cudaGetLastError() == cudaSuccess &&
              cudaMemcpyAsync(hmax, maxsq, 2 * sizeof(float), cudaMemcpyDeviceToHost, st) == cudaSuccess &&
              cudaStreamSynchronize(st) == cudaSuccess;
     }
     fsk_free(mu), fsk_free(maxsq);
-    for (int i = 0; i < 8 && ok; ++i) ok = make_map(&t->map[i], t->buf[i], t->n_pad);
-    ok = ok && cudaFuncSetAttribute(implicit_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
-         cudaFuncSetAttribute(implicit_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
+    for (int i = 0; i < 8 && ok; ++i) ok = make_map(&t->map[i], t->buf[i], t->n_pad, t->kblocks);
+    ok = ok && cudaFuncSetAttribute(implicit_pass_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(1)) == cudaSuccess &&
+         cudaFuncSetAttribute(implicit_pass_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(1)) == cudaSuccess &&
+         cudaFuncSetAttribute(implicit_pass_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(2)) == cudaSuccess &&
+         cudaFuncSetAttribute(implicit_pass_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(2)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         implicit_free(t);
@@ -460,18 +488,23 @@ template <bool COST>
 cudaError_t launch_pass(ImplicitState *t, int transposed, const float *in, FsDeviceStatus *status, cudaStream_t st) {
     const int r = transposed ? 4 : 0, c = transposed ? 2 : 6; // row-side arrays of one cloud, column-side of the other
     FS_HOST_CHECK(t->grid >= 1 && t->T >= 1 && t->T <= MAX_T && (int64_t)t->T * t->nsplit >= t->tiles &&
-                  t->tiles * (int64_t)BM == t->n_pad && t->kd >= 1 && t->kd <= BK / 16);
+                  t->tiles * (int64_t)BM == t->n_pad && t->kd >= 1 && t->kd <= BK / 16 && t->kblocks >= 1 && t->kblocks <= MAX_KB);
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)t->grid);
     cfg.blockDim = dim3(kImpThreads);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.dynamicSmemBytes = smem_bytes(t->kblocks);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr, cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, implicit_pass_kernel<COST>, t->map[r], t->map[r + 1], t->map[c], t->map[c + 1], in, t->partials,
-                              t->n_pad, (int)t->n, t->tiles, t->T, t->nsplit, t->kd, (long long)t->nsplit * NACC * t->n_pad, status);
+    if (t->kblocks == 1)
+        return cudaLaunchKernelEx(&cfg, implicit_pass_kernel<COST, 1>, t->map[r], t->map[r + 1], t->map[c], t->map[c + 1], in,
+                                  t->partials, t->n_pad, (int)t->n, t->tiles, t->T, t->nsplit, t->kd,
+                                  (long long)t->nsplit * NACC * t->n_pad, status);
+    return cudaLaunchKernelEx(&cfg, implicit_pass_kernel<COST, 2>, t->map[r], t->map[r + 1], t->map[c], t->map[c + 1], in,
+                              t->partials, t->n_pad, (int)t->n, t->tiles, t->T, t->nsplit, t->kd,
+                              (long long)t->nsplit * NACC * t->n_pad, status);
 }
 
 // rowsum[i] = u_i * (sum of the partial rows of row i, in order) * scale, in double

@@ -64,10 +64,11 @@ def random_clouds(n, d, seed, spread=1.0):
     return X, Y, a, b
 
 
-@pytest.mark.parametrize("n,d", [(1, 3), (2, 1), (3, 2), (127, 5), (129, 16), (300, 58), (1000, 10), (1153, 27), (4100, 32)])
+@pytest.mark.parametrize("n,d", [(1, 3), (2, 1), (3, 2), (127, 5), (129, 16), (300, 58), (300, 59), (700, 64), (1030, 100), (513, 122), (1000, 10), (1153, 27), (4100, 32)])
 def test_implicit_single_passes(n, d):
     """Each half-step alone from a random state, element by element: ragged last tile, one tile, several
-    column splits, the smallest and the largest supported dimension."""
+    column splits, the smallest and the largest supported dimension, one and two k-blocks of the contraction
+    (d + 6 <= 64 and beyond), norm columns that straddle the k-block boundary (d = 59 .. 63)."""
     X, Y, a, b = random_clouds(n, d, 100 + n)
     scale, eps = 1.0 / d, 0.4
     rng = np.random.default_rng(n)
@@ -163,13 +164,13 @@ def test_implicit_damped_update_and_host_entry_point():
 
 def test_implicit_refuses_what_it_cannot_do_accurately():
     """Configuration 3 (eps = 0.01 on raw squared distances) is outside the accuracy range of the bf16-split
-    contraction: the set-up computes the exponent error bound and refuses; so is d > 58."""
+    contraction: the set-up computes the exponent error bound and refuses; so is d > 122."""
     import torch
     w = workloads.make(3, n=512, fp32_points=True, want_cost=False, want_kernel=False)
     with pytest.raises(fs.FsError) as ei:
         PointSolver(w.X, w.Y, w.cost_scale, w.eps, w.a, w.b)
     assert ei.value.code == fs.FS_ERR_UNSUPPORTED
-    X, Y, a, b = random_clouds(64, 59, 3)
+    X, Y, a, b = random_clouds(64, 123, 3)
     with pytest.raises(fs.FsError) as ei:
         PointSolver(X, Y, 1.0, 10.0, a, b)
     assert ei.value.code == fs.FS_ERR_UNSUPPORTED

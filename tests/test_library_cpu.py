@@ -79,7 +79,7 @@ def test_host_side_validation_needs_no_device(lib):
     assert create_points(b=None) == fs.FS_ERR_NULL
     assert create_points(n=0) == fs.FS_ERR_BAD_N
     assert create_points(d=0) == fs.FS_ERR_BAD_N
-    assert create_points(d=59) == fs.FS_ERR_UNSUPPORTED
+    assert create_points(d=123) == fs.FS_ERR_UNSUPPORTED
     assert create_points(c=9) == fs.FS_ERR_BAD_OFFSETS
     assert create_points(eps=0.0) == fs.FS_ERR_BAD_EPS
     assert create_points(scale=-1.0) == fs.FS_ERR_BAD_EPS
